@@ -1,0 +1,482 @@
+"""Pins for the CPU oracle: everything the paper and plain mathematics fix about
+the path, checked without a GPU.  Each test names the passage it rests on.
+
+The reference computations in this file are written independently of the oracle's
+formulas wherever possible: library softmax attention, brute-force duplication,
+the theorems' invariants, linear-domain closed forms, numpy sorting.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+
+RNG = np.random.default_rng
+
+
+def _rand_unit(rng, n, d, G=1, scale=1.0):
+    K = rng.standard_normal((n, d)) * scale
+    V = rng.standard_normal((n, d))
+    q = rng.standard_normal((G, d))
+    return q, K, V
+
+
+# --------------------------------------------------------------------- rounding
+
+def test_round_bf16_matches_torch_and_ties_to_even():
+    rng = RNG(1)
+    x = np.concatenate([rng.standard_normal(2000) * 10.0 ** rng.integers(-30, 30, 2000),
+                        [0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.3895313892515355e+38, 1e-40, -1e-45]])
+    x32 = x.astype(np.float32)
+    want = torch.from_numpy(x32).to(torch.bfloat16).to(torch.float64).numpy()
+    got = O.round_bf16(x32.astype(np.float64))
+    assert np.array_equal(got, want)
+    # 1 + 2^-8 is exactly half way between 1 and 1 + 2^-7: ties go to the even significand
+    assert O.round_bf16(1.0 + 2.0 ** -8) == 1.0
+    assert O.round_bf16(1.0 + 3 * 2.0 ** -8) == 1.0 + 2 * 2.0 ** -7
+    # directly from fp64 (no double rounding through fp32)
+    assert O.round_bf16(1.0 + 2.0 ** -8 + 2.0 ** -40) == 1.0 + 2.0 ** -7
+
+
+# ------------------------------------------------------- Eq. 3 / Eq. 6 attention
+
+@pytest.mark.parametrize("G,d,n", [(1, 8, 16), (4, 64, 200), (8, 128, 77)])
+def test_votes_one_is_library_softmax_attention(G, d, n):
+    """Eq. 6 with p = 1 is Eq. 3, i.e. textbook scaled-dot-product attention."""
+    rng = RNG(2)
+    q, K, V = _rand_unit(rng, n, d, G)
+    P = O.Params(G=G, d=d)
+    out, lse = O.decode(P, q, K, V, np.ones(n))
+    tq, tK, tV = (torch.from_numpy(a) for a in (q, K, V))
+    ref = torch.nn.functional.scaled_dot_product_attention(tq[None], tK[None], tV[None])[0].numpy()
+    assert np.allclose(out, ref, rtol=0, atol=1e-12)
+    ref_lse = torch.logsumexp(tq @ tK.T / math.sqrt(d), dim=-1).numpy()
+    assert np.allclose(lse, ref_lse, atol=1e-12)
+
+
+def test_votes_equal_duplicated_entries():
+    """Section 3.3.1: an entry with p votes acts as p identical independent copies."""
+    rng = RNG(3)
+    n, d, G = 9, 8, 2
+    q, K, V = _rand_unit(rng, n, d, G)
+    votes = rng.integers(1, 5, n).astype(np.float64)
+    P = O.Params(G=G, d=d)
+    out, lse = O.decode(P, q, K, V, votes)
+    rep = np.repeat(np.arange(n), votes.astype(int))
+    out2, lse2 = O.decode(P, q, K[rep], V[rep], np.ones(len(rep)))
+    assert np.allclose(out, out2, atol=1e-13)
+    assert np.allclose(lse, lse2, atol=1e-13)
+
+
+def test_decode_empty_and_single():
+    P = O.Params(G=2, d=4)
+    out, lse = O.decode(P, np.ones((2, 4)), np.zeros((0, 4)), np.zeros((0, 4)), np.zeros(0))
+    assert np.all(out == 0) and np.all(np.isneginf(lse))
+    V = np.arange(4.0)[None]
+    out, _ = O.decode(P, np.ones((2, 4)), np.ones((1, 4)), V, np.array([3.0]))
+    assert np.allclose(out, np.repeat(V, 2, 0))
+
+
+# ----------------------------------------------------------------- Eq. 8 (EMA)
+
+def test_ema_closed_forms():
+    """Eq. 8: alpha = 0 gives s_hat = s^t; a constant score sequence gives s_hat = s exactly;
+    in general S^n = alpha^(n-1) s^1 + (1-alpha) sum_k alpha^(n-k) s^k, evaluated here in the
+    linear domain, which the oracle never forms."""
+    rng = RNG(4)
+    n, d, G = 12, 8, 1
+    _, K, _ = _rand_unit(rng, n, d, G)
+    qs = rng.standard_normal((6, G, d))
+    s = np.stack([np.exp(qs[t, 0] @ K.T / math.sqrt(d)) for t in range(6)])   # [t, n]
+    # alpha = 0
+    P0 = O.Params(G=G, d=d, ema_alpha=0.0)
+    ls = np.full(n, -np.inf)
+    for t in range(3):
+        ls = O.score_update(P0, qs[t], K, ls)
+        assert np.allclose(np.exp(ls), s[t], rtol=1e-12)
+    # constant sequence
+    Pa = O.Params(G=G, d=d, ema_alpha=0.9)
+    ls = np.full(n, -np.inf)
+    for t in range(5):
+        ls = O.score_update(Pa, qs[0], K, ls)
+    assert np.allclose(np.exp(ls), s[0], rtol=1e-12)
+    # general closed form
+    a = 0.7
+    Pb = O.Params(G=G, d=d, ema_alpha=a)
+    ls = np.full(n, -np.inf)
+    for t in range(6):
+        ls = O.score_update(Pb, qs[t], K, ls)
+    S = a ** 5 * s[0] + (1 - a) * sum(a ** (5 - k) * s[k] for k in range(1, 6))
+    assert np.allclose(np.exp(ls), S, rtol=1e-12)
+
+
+def test_gqa_score_is_group_mean_of_exponentials():
+    rng = RNG(5)
+    n, d, G = 10, 8, 4
+    q, K, _ = _rand_unit(rng, n, d, G)
+    P = O.Params(G=G, d=d, ema_alpha=0.0)
+    ls = O.score_update(P, q, K, np.full(n, -np.inf))
+    s = np.exp(q @ K.T / math.sqrt(d)).mean(axis=0)
+    assert np.allclose(np.exp(ls), s, rtol=1e-12)
+
+
+# ------------------------------------------------------------------- selection
+
+def _select_numpy(kap, budget, n_sink, n_recent):
+    n = len(kap)
+    if budget >= n:
+        return np.arange(n)
+    n_sink = min(n_sink, budget)
+    n_recent = min(n_recent, budget - n_sink)
+    lo, hi = n_sink, n - n_recent
+    mid = np.arange(lo, hi)
+    order = np.lexsort((mid, -kap[mid].astype(np.float64)))   # by kappa descending, then index ascending
+    heavy = mid[order[:budget - n_sink - n_recent]]
+    return np.sort(np.concatenate([np.arange(lo), heavy, np.arange(hi, n)]))
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_selection_against_sorting_and_ties(seed):
+    rng = RNG(100 + seed)
+    n = int(rng.integers(5, 200))
+    kap = rng.standard_normal(n).astype(np.float32)
+    kap[rng.integers(0, n, n // 3)] = kap[rng.integers(0, n)]     # plant equal keys
+    if seed % 2:
+        kap[rng.integers(0, n, 3)] = -np.inf                         # never-scored entries
+    for budget in (0, 1, 3, n // 4, n // 2, n - 1, n, n + 5):
+        for n_sink, n_recent in ((0, 0), (4, 0), (4, 7), (2, n)):
+            want = _select_numpy(kap, budget, n_sink, n_recent)
+            got = O.select(kap, budget, n_sink, n_recent)
+            got2 = O.select(kap, budget, n_sink, n_recent, sorted_impl=True)
+            assert np.array_equal(got, want), (n, budget, n_sink, n_recent)
+            assert np.array_equal(got2, want)
+            assert len(got) == min(n, max(budget, 0))
+
+
+def test_selection_tie_keeps_lowest_index():
+    kap = np.array([0, 5, 5, 5, 1], dtype=np.float32)
+    assert list(O.select(kap, 2, 0, 0)) == [1, 2]
+    assert list(O.select(kap, 3, 1, 1)) == [0, 1, 4]
+
+
+def test_kappa_is_log_of_vote_weighted_score():
+    votes = np.array([1.0, 2.0, 7.0])
+    ls = np.array([0.25, -3.0, -np.inf])
+    k = O.kappa(votes, ls)
+    assert k.dtype == np.float32
+    assert k[0] == np.float32(0.25) and np.isneginf(k[2])
+    assert abs(float(k[1]) - (math.log(2.0) - 3.0)) < 1e-6
+
+
+# ------------------------------------------------- Algorithm 1 lines 4-5: match
+
+def test_match_agrees_with_fp64_cosine_away_from_ties():
+    rng = RNG(7)
+    n, d = 120, 32
+    K = O.round_bf16(rng.standard_normal((n, d)))
+    ret = np.sort(rng.choice(n, 30, replace=False)).astype(np.int32)
+    P = O.Params(G=1, d=d, merge_threshold=-np.inf)
+    target, umax, second = O.match(P, K, ret)
+    Kn = K / np.linalg.norm(K, axis=1, keepdims=True)
+    U = Kn @ Kn[ret].T
+    for e in range(n):
+        if e in ret:
+            assert target[e] == -2
+            continue
+        assert abs(umax[e] - U[e].max()) < 1e-5
+        srt = np.sort(U[e])
+        if srt[-1] - srt[-2] > 1e-5:
+            assert target[e] == int(np.argmax(U[e]))
+        assert 0 <= target[e] < len(ret)
+
+
+def test_match_threshold_and_tie_break_and_degenerate():
+    d = 8
+    e1 = np.eye(d)
+    K = np.stack([e1[0], e1[0], 2 * e1[0] + 0.01 * e1[1], e1[1], np.zeros(d)])
+    ret = np.array([0, 1, 3], dtype=np.int32)      # slots 0,1 hold identical keys
+    P = O.Params(G=1, d=d, merge_threshold=0.8)
+    target, umax, _ = O.match(P, K, ret)
+    assert list(target[:4]) == [-2, -2, 0, -2]     # equal cosine: lowest slot wins
+    assert target[4] == -1                         # zero key: cosine undefined, never merged
+    P2 = O.Params(G=1, d=d, merge_threshold=0.9999999)
+    t2, _, _ = O.match(P2, K, ret)
+    assert t2[2] == -1                             # below T -> evicted without merge
+    # the fixed fp32 recipe: cos(x, x) is exactly 1 for a power-of-two norm
+    assert O.cosine(2 * e1[0], 4 * e1[0]) == 1.0
+    # no retained entries at all
+    t3, u3, _ = O.match(P, K, np.zeros(0, dtype=np.int32))
+    assert np.all(t3 == -1) and np.all(np.isneginf(u3))
+
+
+# --------------------------------------------------------- Eq. 7 / (A.3): merge
+
+def _eq7_literal(pe, se, ke, ve, pc, sc, kc, vc):
+    """Eq. 7 exactly as printed (exponential domain)."""
+    we, wc = pe * se, pc * sc
+    kr = (we * ke + wc * kc) * math.log((we + wc) / (pe + pc)) / (we * math.log(se) + wc * math.log(sc))
+    vr = (we * ve + wc * vc) / (we + wc)
+    return kr, vr, pe + pc
+
+
+def test_pair_merge_equals_printed_equation_7():
+    rng = RNG(8)
+    d = 8
+    for _ in range(50):
+        K = rng.standard_normal((2, d)); V = rng.standard_normal((2, d))
+        p = rng.integers(1, 6, 2).astype(np.float64)
+        lam = rng.uniform(0.2, 3.0, 2) * rng.choice([-1, 1])      # same sign: denominator away from 0
+        m = O.merge_group(d, [0, 1], K, V, p, lam)
+        kr, vr, pr = _eq7_literal(p[0], math.exp(lam[0]), K[0], V[0], p[1], math.exp(lam[1]), K[1], V[1])
+        assert np.allclose(m["k_r"], kr, rtol=1e-11, atol=1e-13)
+        assert np.allclose(m["v_r"], vr, rtol=1e-12)
+        assert m["p_r"] == pr
+
+
+def test_golden_two_entry_values():
+    """Hand-evaluated instances of Eq. 7 (tests/golden/zip_merge_pairs.txt)."""
+    path = os.path.join(os.path.dirname(__file__), "golden", "zip_merge_pairs.txt")
+    rows = [l.split() for l in open(path) if l.strip() and not l.startswith("#")]
+    assert len(rows) >= 3
+    for r in rows:
+        l0, l1, p0, p1, L, lbar, gamma, om0 = map(float, r)
+        K = np.array([[1.0, 0.0], [0.0, 1.0]]); V = K.copy()
+        m = O.merge_group(2, [0, 1], K, V, [p0, p1], [l0, l1])
+        assert abs(m["lambda_r"] - L) < 2e-6
+        assert abs(m["lambda_bar"] - lbar) < 2e-6
+        assert abs(m["gamma"] - gamma) < 2e-6
+        assert abs(m["v_r"][0] - om0) < 2e-6       # v_r = omega_0 e_0 + omega_1 e_1
+        assert abs(m["k_r"][0] - gamma * om0) < 4e-6
+
+
+def _lossless_case(rng, n, d, budget, votes_max, guard=False, n_sink=0, n_recent=0):
+    q, K, V = _rand_unit(rng, n, d, 1)
+    votes = rng.integers(1, votes_max + 1, n).astype(np.float64)
+    P = O.Params(G=1, d=d, ema_alpha=0.0, merge_threshold=-np.inf, n_sink=n_sink, n_recent=n_recent,
+                 gamma_min=0.0 if guard else -np.inf, gamma_max=4.0 if guard else np.inf)
+    ls = O.score_update(P, q, K, np.full(n, -np.inf))       # s_hat = s^t
+    o0, lse0 = O.decode(P, q, K, V, votes)
+    c = O.compress(P, budget, K, V, votes, ls)
+    o1, lse1 = O.decode(P, q, c["K"], c["V"], c["votes"])
+    return P, q, K, V, votes, ls, c, (o0, lse0), (o1, lse1)
+
+
+@pytest.mark.parametrize("seed", range(20))
+def test_single_step_lossless_theorem_2(seed):
+    """Theorem 2 / Eq. (A.3): with s_hat = s^t, recomputing step t on the compressed cache
+    reproduces the output, for pair and many-to-one merges and any vote counts."""
+    rng = RNG(200 + seed)
+    n = int(rng.integers(3, 40)); d = int(rng.choice([4, 8, 16]))
+    budget = int(rng.integers(1, n))
+    P, q, K, V, votes, ls, c, (o0, lse0), (o1, lse1) = _lossless_case(rng, n, d, budget, 4, n_sink=seed % 3,
+                                                                      n_recent=seed % 4)
+    lbar_ok = np.all(np.isnan(c["gammas"]) | (np.abs(c["gammas"]) < 1e6))
+    if not lbar_ok:
+        pytest.skip("group with lambda_bar ~ 0: the printed formula is singular there")
+    assert c["stats"]["n_merged"] == n - budget          # T = -inf: every evicted entry merges
+    assert np.max(np.abs(o1 - o0)) < 1e-9                # north star asks 1e-5
+    assert abs(lse1[0] - lse0[0]) < 1e-9                 # the denominator is conserved too
+    # Electoral-Votes conservation: p_r = sum of members' votes
+    assert c["votes"].sum() == votes.sum()
+
+
+def test_conserved_sums_per_group():
+    """Eq. (A.2): sum_{K'_e} p_i s_i = p_r s_r and sum p_i s_i v_i = p_r s_r v_r for every group,
+    with s_r = exp(q.k_r/sqrt(d)) evaluated on the merged key."""
+    rng = RNG(9)
+    n, d = 30, 8
+    P, q, K, V, votes, ls, c, _, _ = _lossless_case(rng, n, d, 6, 3)
+    s = np.exp(q[0] @ K.T / math.sqrt(d))
+    for slot, ci in enumerate(c["ret_idx"]):
+        mem = [ci] + [e for e in range(n) if c["target"][e] == slot]
+        s_r = math.exp(q[0] @ c["K"][slot] / math.sqrt(d))
+        p_r = c["votes"][slot]
+        assert p_r == votes[mem].sum()
+        assert math.isclose(p_r * s_r, (votes[mem] * s[mem]).sum(), rel_tol=1e-9)
+        assert np.allclose(p_r * s_r * c["V"][slot], ((votes[mem] * s[mem])[:, None] * V[mem]).sum(0), rtol=1e-9)
+        # reading R8: the merged entry's score state carries ln(sum p s_hat / sum p)
+        assert math.isclose(c["lscore"][slot], math.log((votes[mem] * s[mem]).sum() / p_r), rel_tol=1e-9, abs_tol=1e-12)
+
+
+def test_softmax_probabilities_instead_of_exponentials_break_losslessness():
+    """Negative control for the reading s = exp(q.k/sqrt(d)) (Eq. 3): feeding normalised
+    attention weights into Eq. 7 does not preserve the output."""
+    rng = RNG(10)
+    n, d = 12, 8
+    q, K, V = _rand_unit(rng, n, d, 1)
+    P = O.Params(G=1, d=d, ema_alpha=0.0, merge_threshold=-np.inf, n_sink=0, gamma_min=-np.inf, gamma_max=np.inf)
+    ell = q[0] @ K.T / math.sqrt(d)
+    ls_prob = ell - np.log(np.exp(ell).sum())              # ln softmax probability
+    o0, _ = O.decode(P, q, K, V, np.ones(n))
+    c = O.compress(P, 4, K, V, np.ones(n), ls_prob)
+    o1, _ = O.decode(P, q, c["K"], c["V"], c["votes"])
+    assert np.max(np.abs(o1 - o0)) > 1e-3
+
+
+def test_identical_pair_lemma():
+    """Lemma 1: merging identical entries keeps (k, v), sets p = 2, and stays exact for every later query."""
+    rng = RNG(11)
+    d = 8
+    k = rng.standard_normal(d); v = rng.standard_normal(d)
+    lam = 0.7
+    m = O.merge_group(d, [0, 1], np.stack([k, k]), np.stack([v, v]), [1.0, 1.0], [lam, lam])
+    assert np.allclose(m["k_r"], k, atol=1e-14) and np.allclose(m["v_r"], v, atol=1e-14)
+    assert m["p_r"] == 2.0 and abs(m["gamma"] - 1.0) < 1e-14
+    K = np.vstack([rng.standard_normal((5, d)), k, k]); V = np.vstack([rng.standard_normal((5, d)), v, v])
+    P = O.Params(G=1, d=d)
+    for _ in range(5):
+        q = rng.standard_normal((1, d))
+        o0, _ = O.decode(P, q, K, V, np.ones(7))
+        o1, _ = O.decode(P, q, np.vstack([K[:5], m["k_r"]]), np.vstack([V[:5], m["v_r"]]), np.r_[np.ones(5), 2.0])
+        assert np.allclose(o0, o1, atol=1e-13)
+
+
+@pytest.mark.parametrize("seed", range(30))
+def test_multi_step_bound_theorem_3(seed):
+    """Theorem 3: with relative prediction error eps < 1 on every entry of the group and on the
+    merged entry, the perturbation at a later step is below 2 eps (1+eps) gamma / (1-eps)^2."""
+    rng = RNG(300 + seed)
+    n, d = 12, 8
+    K = rng.standard_normal((n, d)) * 0.5
+    V = rng.standard_normal((n, d))
+    votes = rng.integers(1, 3, n).astype(np.float64)
+    q2 = rng.standard_normal((1, d))                        # the later query (step t')
+    s2 = np.exp(q2[0] @ K.T / math.sqrt(d))                 # true scores at t'
+    group = [int(i) for i in rng.choice(n, int(rng.integers(2, 5)), replace=False)]
+    shat = s2 * (1.0 + rng.uniform(-0.3, 0.3, n))           # estimates used by the merge
+    m = O.merge_group(d, group, K, V, votes, np.log(shat))
+    rest = [i for i in range(n) if i not in group]
+    K1 = np.vstack([K[rest], m["k_r"]]); V1 = np.vstack([V[rest], m["v_r"]]); p1 = np.r_[votes[rest], m["p_r"]]
+    P = O.Params(G=1, d=d)
+    o_full, _ = O.decode(P, q2, K, V, votes)
+    o_cmp, _ = O.decode(P, q2, K1, V1, p1)
+    theta = np.linalg.norm(o_full - o_cmp)
+    s_r = math.exp(q2[0] @ m["k_r"] / math.sqrt(d)); shat_r = math.exp(m["lambda_r"])
+    eps = max(np.max(np.abs(1 - shat[group] / s2[group])), abs(1 - shat_r / s_r))
+    if eps >= 1.0:
+        pytest.skip("prediction error outside the theorem's range")
+    gam = max(np.linalg.norm(V[j] - V[i]) for j in group for i in range(n))
+    assert theta < 2 * eps * (1 + eps) * gam / (1 - eps) ** 2
+
+
+def test_eviction_identity_equation_4():
+    """Eq. 4 / (A.1): entries that find no target above T are dropped, and the output moves to
+    (o - sum_j A_j v_j) / (1 - sum_j A_j)."""
+    rng = RNG(12)
+    n, d = 20, 8
+    q, K, V = _rand_unit(rng, n, d, 1)
+    P = O.Params(G=1, d=d, ema_alpha=0.0, merge_threshold=np.inf, n_sink=0)
+    ls = O.score_update(P, q, K, np.full(n, -np.inf))
+    o0, _ = O.decode(P, q, K, V, np.ones(n))
+    c = O.compress(P, 7, K, V, np.ones(n), ls)
+    assert c["stats"]["n_merged"] == 0 and c["stats"]["n_below_T"] == n - 7
+    ev = [i for i in range(n) if i not in c["ret_idx"]]
+    A = np.exp(ls) / np.exp(ls).sum()
+    want = (o0[0] - (A[ev, None] * V[ev]).sum(0)) / (1 - A[ev].sum())
+    o1, _ = O.decode(P, q, c["K"], c["V"], c["votes"])
+    assert np.allclose(o1[0], want, atol=1e-12)
+    # retained rows are copied untouched, in ascending original index
+    assert np.array_equal(c["K"], K[c["ret_idx"]]) and np.all(np.diff(c["ret_idx"]) > 0)
+    # the kept set is the top-7 by score here (no sinks, no recent window)
+    assert set(c["ret_idx"]) == set(np.argsort(-ls)[:7])
+
+
+def test_attention_sag_of_convex_merging_theorem_1():
+    """Theorem 1 (negative control): a convex combination of two entries receives less attention
+    than the two did together, so the same check that passes for ZIP merging fails here."""
+    rng = RNG(13)
+    n, d = 10, 8
+    q, K, V = _rand_unit(rng, n, d, 1)
+    P = O.Params(G=1, d=d)
+    s = np.exp(q[0] @ K.T / math.sqrt(d)); A = s / s.sum()
+    e, c, w = 2, 5, 0.35
+    kr = w * K[e] + (1 - w) * K[c]; vr = w * V[e] + (1 - w) * V[c]
+    rest = [i for i in range(n) if i not in (e, c)]
+    s_r = math.exp(q[0] @ kr / math.sqrt(d))
+    A_r = s_r / (s[rest].sum() + s_r)
+    assert A_r < A[e] + A[c]
+    o0, _ = O.decode(P, q, K, V, np.ones(n))
+    o1, _ = O.decode(P, q, np.vstack([K[rest], kr]), np.vstack([V[rest], vr]), np.ones(n - 1))
+    assert np.linalg.norm(o0 - o1) > 1e-4
+
+
+def test_guard_on_rescale_factor():
+    """A group whose log-scores straddle zero makes the printed rescale factor negative; with the
+    guard on, its members are evicted and the target is left untouched."""
+    d = 4
+    K = np.eye(4)[:3] + 0.0; V = np.eye(4)[:3] + 1.0
+    K[1] = K[0] * 1.0001                                   # entry 1 will pick slot of entry 0
+    votes = np.ones(3); ls = np.array([0.5, -2.0, 3.0])
+    m = O.merge_group(d, [0, 1], K, V, votes, ls)
+    assert abs(m["gamma"] - (-0.368)) < 2e-3               # L = -0.114, lambda_bar = +0.310
+    P = O.Params(G=1, d=d, merge_threshold=-np.inf, n_sink=0)
+    c = O.compress(P, 2, K, V, votes, ls)
+    assert list(c["ret_idx"]) == [0, 2] and c["target"][1] == -1
+    assert c["stats"]["n_guard_groups"] == 1 and c["stats"]["n_merged"] == 0
+    assert np.array_equal(c["K"][0], K[0]) and c["votes"][0] == 1.0
+    Pu = O.Params(G=1, d=d, merge_threshold=-np.inf, n_sink=0, gamma_min=-np.inf, gamma_max=np.inf)
+    cu = O.compress(Pu, 2, K, V, votes, ls)
+    assert cu["target"][1] == 0 and cu["votes"][0] == 2.0
+
+
+def test_compress_is_ordered_copy_when_budget_not_exceeded():
+    rng = RNG(14)
+    n, d = 9, 4
+    q, K, V = _rand_unit(rng, n, d, 1)
+    P = O.Params(G=1, d=d)
+    c = O.compress(P, 9, K, V, np.ones(n), np.zeros(n))
+    assert np.array_equal(c["K"], K) and np.array_equal(c["V"], V) and len(c["ret_idx"]) == n
+    c = O.compress(P, 50, K, V, np.ones(n), np.zeros(n))
+    assert len(c["ret_idx"]) == n
+
+
+def test_storage_faithful_mode_rounds_every_write():
+    rng = RNG(15)
+    n, d = 24, 8
+    q, K, V = _rand_unit(rng, n, d, 1)
+    K = O.round_bf16(K); V = O.round_bf16(V)
+    P = O.Params(G=1, d=d, ema_alpha=0.0, merge_threshold=-np.inf, n_sink=0, storage_faithful=True,
+                 gamma_min=-np.inf, gamma_max=np.inf)
+    ls = O.score_update(P, q, K, np.full(n, -np.inf))
+    assert np.array_equal(ls, ls.astype(np.float32).astype(np.float64))
+    c = O.compress(P, 5, K, V, np.ones(n), ls)
+    assert np.array_equal(c["K"], O.round_bf16(c["K"])) and np.array_equal(c["V"], O.round_bf16(c["V"]))
+    # rounding the merged rows to bf16 costs accuracy but stays within bf16 resolution of lossless
+    o0, _ = O.decode(P, q, K, V, np.ones(n))
+    o1, _ = O.decode(P, q, c["K"], c["V"], c["votes"])
+    assert np.max(np.abs(o1 - o0)) < 5e-2
+
+
+def test_append_equation_2():
+    d = 4
+    K = np.zeros((5, d)); V = np.zeros((5, d)); votes = np.zeros(5); ls = np.zeros(5)
+    n = O.append(K, V, votes, ls, 2, np.arange(4.0), -np.arange(4.0))
+    assert n == 3 and np.array_equal(K[2], np.arange(4.0)) and np.array_equal(V[2], -np.arange(4.0))
+    assert votes[2] == 1.0 and np.isneginf(ls[2]) and np.all(K[3:] == 0)
+
+
+def test_batch_wrappers_match_per_unit():
+    rng = RNG(16)
+    U, n_cap, d, G = 3, 20, 8, 2
+    P = O.Params(G=G, d=d, merge_threshold=-np.inf, n_sink=1, n_recent=2)
+    K = rng.standard_normal((U, n_cap, d)); V = rng.standard_normal((U, n_cap, d))
+    votes = np.ones((U, n_cap)); ls = np.full((U, n_cap), -np.inf)
+    q = rng.standard_normal((U, G, d))
+    lens = np.array([20, 13, 0], dtype=np.int32)
+    out, lse = O.decode_batch(P, lens, q, K, V, votes, ls, True)
+    for u in range(U):
+        n = lens[u]
+        o, l = O.decode(P, q[u], K[u, :n], V[u, :n], votes[u, :n])
+        assert np.array_equal(out[u], o) and np.array_equal(lse[u], l)
+        assert np.array_equal(ls[u, :n], O.score_update(P, q[u], K[u, :n], np.full(n, -np.inf)))
+    r = O.compress_batch(P, lens, np.array([5, 5, 5], dtype=np.int32), K, V, votes, ls)
+    for u in range(U):
+        n = lens[u]
+        c = O.compress(P, 5, K[u, :n], V[u, :n], votes[u, :n], ls[u, :n])
+        m = r["new_lens"][u]
+        assert m == len(c["ret_idx"])
+        assert np.array_equal(r["K"][u, :m], c["K"]) and np.array_equal(r["votes"][u, :m], c["votes"])
+        assert np.array_equal(r["ret_idx"][u, :m], c["ret_idx"]) and np.array_equal(r["target"][u, :n], c["target"])
