@@ -1,0 +1,166 @@
+/*
+ * keepkv.h -- C ABI of the KeepKV hot path for NVIDIA B200 (sm_100a).
+ *
+ * KeepKV (arXiv 2504.09936) keeps a KV cache within a fixed budget by merging the
+ * entries it would otherwise evict into their most similar retained entries, in a
+ * way that leaves the current attention output unchanged (Theorem 2).  This
+ * library implements the three operations of its decode loop for one attention
+ * layer:
+ *
+ *   keepkv_append            K_t = [K_{t-1}, k_t], V_t = [V_{t-1}, v_t]          (Eq. 2)
+ *   keepkv_decode_attention  o = sum p_i s_i v_i / sum p_i s_i                   (Eq. 6)
+ *                            and the running score estimate of every entry       (Eq. 8)
+ *   keepkv_compress          Algorithm 1: select retained / evicted sets, match
+ *                            each evicted key to its most cosine-similar retained
+ *                            key, merge with the ZIP equations (Eq. 7, Eq. A.3).
+ *
+ * Conventions
+ *  - Every pointer is DEVICE memory owned by the caller unless its name ends in
+ *    `_host`.  The library allocates nothing, holds no state between calls and
+ *    never synchronises: each call validates its arguments on the host, enqueues
+ *    kernels on `stream` (a cudaStream_t passed as void*) and returns at once.
+ *  - Return value: KEEPKV_OK or a negative keepkv_status.  Nothing is enqueued
+ *    when a negative value is returned, except for KEEPKV_ERR_CUDA (a launch
+ *    failed part-way; keepkv_last_cuda_error() gives the cudaError_t).
+ *  - Problems only the device can see (append into a full cache) are reported by
+ *    OR-ing a KEEPKV_DEV_* bit into *status_dev, an int32 the caller zeroes and
+ *    reads back when it likes; the offending work item is skipped, never faulted.
+ *  - Layouts are dense row-major with the last index fastest.  bf16 is the
+ *    storage type of keys, values, queries and outputs; all accumulation is fp32.
+ *  - A "unit" is one (sequence b, kv head h) pair, u = b * H_kv + h.  Query head
+ *    g of unit u is head h * G + g, G = H_q / H_kv.
+ */
+#ifndef KEEPKV_H_
+#define KEEPKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum keepkv_status {
+  KEEPKV_OK = 0,
+  KEEPKV_ERR_INVALID_ARG = -1,     /* null pointer, non-positive size, misaligned pointer      */
+  KEEPKV_ERR_UNSUPPORTED = -2,     /* d not in {64,128}, G not in {1,2,4,8}, N_cap % 64 != 0 ...  */
+  KEEPKV_ERR_CAPACITY = -3,        /* budget + period exceeds N_cap, budget > N_cap             */
+  KEEPKV_ERR_WORKSPACE = -4,       /* workspace smaller than keepkv_workspace_bytes             */
+  KEEPKV_ERR_CUDA = -5             /* a CUDA runtime/driver call failed                         */
+} keepkv_status;
+
+/* bits OR-ed into *status_dev by kernels */
+#define KEEPKV_DEV_APPEND_FULL 1   /* keepkv_append: seq_len == N_cap, the token was dropped    */
+#define KEEPKV_DEV_TIMEOUT 2       /* a bounded wait inside a kernel ran out                    */
+
+typedef struct keepkv_params {
+  int32_t B;                /* sequences                                                       */
+  int32_t H_q;              /* query heads                                                     */
+  int32_t H_kv;             /* kv heads; G = H_q / H_kv in {1,2,4,8}                           */
+  int32_t d;                /* head dimension, 64 or 128                                       */
+  int32_t N_cap;            /* allocated entries per unit (stride of the entry axis), % 64 == 0 */
+  int32_t period;           /* compression period P, used only to check N_cap >= budget + P    */
+  int32_t n_sink;           /* entries always kept at the front (App. B.3: 4)                  */
+  int32_t n_recent;         /* entries always kept at the back  (App. B.3: recent window)      */
+  float sm_scale;           /* 1/sqrt(d) of Eq. 3                                              */
+  float ema_alpha;          /* alpha of Eq. 8, in [0,1); 0 makes the estimate the last score   */
+  float merge_threshold;    /* T of Algorithm 1 line 5 (paper: 0.8); -INFINITY merges always   */
+  float gamma_min;          /* a group is merged only if gamma_min < gamma <= gamma_max, gamma */
+  float gamma_max;          /* the key rescale factor of Eq. A.3; (-INF, +INF) = paper as is   */
+  int32_t reserved[3];      /* must be zero                                                    */
+} keepkv_params;
+
+/* One layer's cache.  Rows [seq_len[b], N_cap) of a unit are unspecified. */
+typedef struct keepkv_cache {
+  void *K;                  /* bf16 [B, H_kv, N_cap, d]  keys k_i              (16-byte aligned) */
+  void *V;                  /* bf16 [B, H_kv, N_cap, d]  values v_i            (16-byte aligned) */
+  float *votes;             /* fp32 [B, H_kv, N_cap]     Electoral Votes p_i, 1 for a fresh entry */
+  float *lscore;            /* fp32 [B, H_kv, N_cap]     ln of the EMA score estimate (Eq. 8);  */
+                            /*                           -INFINITY = never scored               */
+  int32_t *seq_len;         /* i32  [B]                  valid entries, shared by the kv heads  */
+} keepkv_cache;
+
+/* Per-unit counters written by keepkv_compress, [B * H_kv] of them. */
+typedef struct keepkv_stats {
+  int32_t n_retained;       /* entries kept (= new seq_len)                                    */
+  int32_t n_evicted;        /* entries not kept                                                */
+  int32_t n_merged;         /* evicted entries folded into a retained one                      */
+  int32_t n_below_T;        /* evicted entries whose best cosine did not exceed T              */
+  int32_t n_guard_groups;   /* groups rejected by the gamma guard (their members are dropped)  */
+  int32_t n_groups;         /* retained entries that had at least one candidate member         */
+  int32_t max_group;        /* largest number of members merged into one entry                 */
+  int32_t reserved;
+} keepkv_stats;
+
+/* Bytes of scratch the calls below need for this shape (a function of B, H_q, H_kv, d, N_cap
+ * only).  The same workspace serves decode and compress; calls that share one must not overlap
+ * in time.  It must be 256-byte aligned and set up once with keepkv_workspace_init. */
+int keepkv_workspace_bytes(const keepkv_params *p, size_t *bytes);
+
+/* Zeroes the arrival counters kept in the workspace (they return to zero after every call). */
+int keepkv_workspace_init(const keepkv_params *p, void *ws, size_t ws_bytes, void *stream);
+
+/* Eq. 2.  For every sequence b and kv head h, writes k_new[b,h,:], v_new[b,h,:] (bf16 [B,H_kv,d])
+ * to row seq_len[b], sets that entry's votes to 1 (Section 3.3.1: p initialised to 1) and its
+ * lscore to -INFINITY, then increments seq_len[b].  A sequence already at N_cap is left
+ * unchanged and KEEPKV_DEV_APPEND_FULL is raised in *status_dev. */
+int keepkv_append(const keepkv_params *p, const keepkv_cache *cache, const void *k_new, const void *v_new,
+                  int32_t *status_dev, void *stream);
+
+/* Eq. 6 (Electoral-Votes attention; Eq. 3 when all votes are 1).  For each query head,
+ *   l_i = sm_scale * q . k_i,   o = sum_i p_i e^{l_i} v_i / sum_i p_i e^{l_i},  i < seq_len[b].
+ * q, out: bf16 [B, H_q, d].  lse_or_null: fp32 [B, H_q], ln sum_i p_i e^{l_i} (-INF for an empty
+ * sequence, whose output is 0).
+ * update_scores != 0 also advances Eq. 8 for every entry read: the kv head's score at this step
+ * is the mean over its G query heads of e^{l_i}; lscore <- ln(alpha e^{lscore} + (1-alpha) score),
+ * or ln(score) for an entry never scored before (per-entry bias correction) or when alpha = 0.
+ * This is the "attention scores s^t" input of Algorithm 1, produced without materialising them. */
+int keepkv_decode_attention(const keepkv_params *p, const keepkv_cache *cache, const void *q, void *out,
+                            float *lse_or_null, int update_scores, void *ws, size_t ws_bytes, int32_t *status_dev,
+                            void *stream);
+
+/* Algorithm 1, out of place: reads `src` (unchanged), writes `dst` (distinct buffers of the same
+ * shape).  Per unit, with len = src.seq_len[b] and budget b_b (budget_dev[b] if given, else
+ * budget_scalar; likewise n_recent_dev[b] / p->n_recent):
+ *   1. key kappa_i = fp32(ln p_i + lscore_i); retained set = first n_sink, last n_recent and the
+ *      largest kappa among the rest, equal keys -> lower index; everything else is evicted
+ *      (Algorithm 1 lines 2-3; App. B.3).  If the budget is below n_sink + n_recent the recent
+ *      window shrinks first.  len <= budget: plain ordered copy.
+ *   2. each evicted key takes the retained key of highest cosine similarity as its target,
+ *      equal values -> lower slot, and is merged only if that cosine exceeds merge_threshold
+ *      (lines 4-5).  The cosine is the fp32 value dot/(sqrtf(n_e)*sqrtf(n_c)) with dot and the
+ *      squared norms accumulated by fused multiply-add from 0 over channels 0..d-1.
+ *   3. every retained entry with members is rewritten by Eq. A.3 using exp(lscore) as score
+ *      estimate: v_r, k_r, p_r = sum of votes, lscore_r = ln(sum p s / sum p) (lines 7-10).
+ *   4. dst holds the retained entries in ascending source order, dst.seq_len[b] = min(len, b_b).
+ * Optional outputs: retained_idx_or_null i32 [B, H_kv, N_cap] (first seq_len entries valid: source
+ * index of each dst row); target_or_null i32 [B, H_kv, N_cap] (per source entry: dst slot it was
+ * merged into, -1 dropped, -2 retained); stats_or_null [B * H_kv]. */
+int keepkv_compress(const keepkv_params *p, const keepkv_cache *src, const keepkv_cache *dst,
+                    const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
+                    int32_t *retained_idx_or_null, int32_t *target_or_null, keepkv_stats *stats_or_null, void *ws,
+                    size_t ws_bytes, int32_t *status_dev, void *stream);
+
+/* One decode step driven from HOST memory (the call a serving loop makes): copies q_host,
+ * k_new_host, v_new_host (pinned or pageable host memory, shapes as above) into the device
+ * staging buffers q_dev/k_new_dev/v_new_dev, runs keepkv_append and keepkv_decode_attention
+ * (update_scores as given) and copies the result from out_dev into out_host, all enqueued on
+ * `stream`; the caller synchronises the stream before reading out_host. */
+int keepkv_decode_step_host(const keepkv_params *p, const keepkv_cache *cache, const void *q_host,
+                            const void *k_new_host, const void *v_new_host, void *out_host, void *q_dev,
+                            void *k_new_dev, void *v_new_dev, void *out_dev, int update_scores, void *ws,
+                            size_t ws_bytes, int32_t *status_dev, void *stream);
+
+/* Human-readable name of a keepkv_status. */
+const char *keepkv_status_string(int status);
+
+/* cudaError_t of the most recent KEEPKV_ERR_CUDA on this thread (0 if none). */
+int keepkv_last_cuda_error(void);
+
+/* Number of kernels the most recent successful call on this thread enqueued. */
+int keepkv_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KEEPKV_H_ */

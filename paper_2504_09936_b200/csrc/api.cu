@@ -1,0 +1,212 @@
+// C ABI of libkeepkv: argument validation, workspace layout, and dispatch to the kernels.
+#include <math.h>
+#include <string.h>
+
+#include "common.cuh"
+
+namespace keepkv {
+
+static thread_local int g_last_cuda_error = 0;
+static thread_local int g_last_launches = 0;
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+WsLayout ws_layout(const keepkv_params &p) {
+  WsLayout L;
+  const size_t U = (size_t)p.B * p.H_kv, N = (size_t)p.N_cap, G = (size_t)(p.H_q / p.H_kv);
+  // Enough splits to put at least four waves of CTAs on 148 SMs, never more than the tiles of a unit.
+  size_t tiles = (N + kTile - 1) / kTile;
+  size_t want = (4 * 148 + U - 1) / U;
+  size_t S = want < 1 ? 1 : want;
+  if (S > tiles) S = tiles;
+  if (S > (size_t)kMaxSplits) S = kMaxSplits;
+  L.max_splits = (int)S;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  L.counters = take(U * 4);
+  L.part_ml = take(U * S * G * 2 * 4);
+  L.part_acc = take(U * S * G * (size_t)p.d * 4);
+  L.unit_info = take(U * 4 * 4);
+  L.ret_idx = take(U * N * 4);
+  L.target = take(U * N * 4);
+  L.ev_idx = take(U * N * 4);
+  L.dst_norm = take(U * N * 4);
+  L.umax = take(U * N * 4);
+  L.cand = take(U * N * 2 * 4);
+  L.grp_ptr = take(U * (N + 1) * 4);
+  L.grp_fill = take(U * N * 4);
+  L.grp_mem = take(U * N * 4);
+  L.stats = take(U * sizeof(keepkv_stats));
+  L.total = off;
+  return L;
+}
+
+int choose_splits(const keepkv_params &p, int max_splits) {
+  // Two resident CTAs per SM: aim at a whole number of waves of 296 CTAs.
+  const int U = p.B * p.H_kv;
+  int S = (2 * 148 + U - 1) / U;
+  if (S < 1) S = 1;
+  if (S > max_splits) S = max_splits;
+  return S;
+}
+
+static int validate(const keepkv_params *p) {
+  if (!p) return KEEPKV_ERR_INVALID_ARG;
+  if (p->B <= 0 || p->H_q <= 0 || p->H_kv <= 0 || p->N_cap <= 0) return KEEPKV_ERR_INVALID_ARG;
+  if (p->reserved[0] || p->reserved[1] || p->reserved[2]) return KEEPKV_ERR_INVALID_ARG;
+  if (p->H_q % p->H_kv) return KEEPKV_ERR_UNSUPPORTED;
+  const int G = p->H_q / p->H_kv;
+  if (!(G == 1 || G == 2 || G == 4 || G == 8)) return KEEPKV_ERR_UNSUPPORTED;
+  if (!(p->d == 64 || p->d == 128)) return KEEPKV_ERR_UNSUPPORTED;
+  if (p->N_cap % 64) return KEEPKV_ERR_UNSUPPORTED;
+  if (p->N_cap > 49152) return KEEPKV_ERR_UNSUPPORTED;  // selection keeps one key per entry in shared memory
+  if (p->n_sink < 0 || p->n_recent < 0 || p->period < 0) return KEEPKV_ERR_INVALID_ARG;
+  if (!(p->ema_alpha >= 0.0f && p->ema_alpha < 1.0f)) return KEEPKV_ERR_INVALID_ARG;
+  if (!(p->sm_scale > 0.0f) || isnan(p->merge_threshold) || isnan(p->gamma_min) || isnan(p->gamma_max))
+    return KEEPKV_ERR_INVALID_ARG;
+  return KEEPKV_OK;
+}
+
+static bool aligned(const void *ptr, size_t a) { return (reinterpret_cast<uintptr_t>(ptr) % a) == 0; }
+
+static int validate_cache(const keepkv_cache *c) {
+  if (!c || !c->K || !c->V || !c->votes || !c->lscore || !c->seq_len) return KEEPKV_ERR_INVALID_ARG;
+  if (!aligned(c->K, 16) || !aligned(c->V, 16) || !aligned(c->votes, 16) || !aligned(c->lscore, 16))
+    return KEEPKV_ERR_INVALID_ARG;
+  return KEEPKV_OK;
+}
+
+static int finish(LaunchCtx &ctx) {
+  g_last_launches = ctx.launches;
+  if (ctx.err != cudaSuccess) {
+    g_last_cuda_error = (int)ctx.err;
+    return KEEPKV_ERR_CUDA;
+  }
+  return KEEPKV_OK;
+}
+
+}  // namespace keepkv
+
+using namespace keepkv;
+
+extern "C" {
+
+int keepkv_workspace_bytes(const keepkv_params *p, size_t *bytes) {
+  int rc = validate(p);
+  if (rc) return rc;
+  if (!bytes) return KEEPKV_ERR_INVALID_ARG;
+  *bytes = ws_layout(*p).total;
+  return KEEPKV_OK;
+}
+
+int keepkv_workspace_init(const keepkv_params *p, void *ws, size_t ws_bytes, void *stream) {
+  int rc = validate(p);
+  if (rc) return rc;
+  if (!ws || !aligned(ws, 256)) return KEEPKV_ERR_INVALID_ARG;
+  WsLayout L = ws_layout(*p);
+  if (ws_bytes < L.total) return KEEPKV_ERR_WORKSPACE;
+  LaunchCtx ctx{(cudaStream_t)stream, 0, cudaSuccess};
+  ctx.err = cudaMemsetAsync((char *)ws + L.counters, 0, (size_t)p->B * p->H_kv * 4, ctx.stream);
+  return finish(ctx);
+}
+
+int keepkv_append(const keepkv_params *p, const keepkv_cache *cache, const void *k_new, const void *v_new,
+                  int32_t *status_dev, void *stream) {
+  int rc = validate(p);
+  if (rc) return rc;
+  if ((rc = validate_cache(cache))) return rc;
+  if (!k_new || !v_new || !status_dev || !aligned(k_new, 16) || !aligned(v_new, 16)) return KEEPKV_ERR_INVALID_ARG;
+  LaunchCtx ctx{(cudaStream_t)stream, 0, cudaSuccess};
+  launch_append(*p, *cache, k_new, v_new, status_dev, ctx);
+  return finish(ctx);
+}
+
+int keepkv_decode_attention(const keepkv_params *p, const keepkv_cache *cache, const void *q, void *out,
+                            float *lse_or_null, int update_scores, void *ws, size_t ws_bytes, int32_t *status_dev,
+                            void *stream) {
+  int rc = validate(p);
+  if (rc) return rc;
+  if ((rc = validate_cache(cache))) return rc;
+  if (!q || !out || !ws || !status_dev || !aligned(q, 16) || !aligned(out, 16) || !aligned(ws, 256))
+    return KEEPKV_ERR_INVALID_ARG;
+  WsLayout L = ws_layout(*p);
+  if (ws_bytes < L.total) return KEEPKV_ERR_WORKSPACE;
+  LaunchCtx ctx{(cudaStream_t)stream, 0, cudaSuccess};
+  launch_decode(*p, *cache, q, out, lse_or_null, update_scores, (char *)ws, L, status_dev, ctx);
+  return finish(ctx);
+}
+
+int keepkv_compress(const keepkv_params *p, const keepkv_cache *src, const keepkv_cache *dst,
+                    const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
+                    int32_t *retained_idx_or_null, int32_t *target_or_null, keepkv_stats *stats_or_null, void *ws,
+                    size_t ws_bytes, int32_t *status_dev, void *stream) {
+  int rc = validate(p);
+  if (rc) return rc;
+  if ((rc = validate_cache(src))) return rc;
+  if ((rc = validate_cache(dst))) return rc;
+  if (src->K == dst->K || src->V == dst->V || src->votes == dst->votes || src->lscore == dst->lscore ||
+      src->seq_len == dst->seq_len)
+    return KEEPKV_ERR_INVALID_ARG;
+  if (!ws || !status_dev || !aligned(ws, 256)) return KEEPKV_ERR_INVALID_ARG;
+  if (!budget_dev) {
+    if (budget_scalar < 0) return KEEPKV_ERR_INVALID_ARG;
+    if (budget_scalar > p->N_cap || (long long)budget_scalar + p->period > p->N_cap) return KEEPKV_ERR_CAPACITY;
+  }
+  WsLayout L = ws_layout(*p);
+  if (ws_bytes < L.total) return KEEPKV_ERR_WORKSPACE;
+  LaunchCtx ctx{(cudaStream_t)stream, 0, cudaSuccess};
+  char *w = (char *)ws;
+  launch_compress(*p, *src, *dst, budget_dev, budget_scalar, n_recent_dev,
+                  retained_idx_or_null ? retained_idx_or_null : (int32_t *)(w + L.ret_idx),
+                  target_or_null ? target_or_null : (int32_t *)(w + L.target),
+                  stats_or_null ? stats_or_null : (keepkv_stats *)(w + L.stats), w, L, status_dev, ctx);
+  return finish(ctx);
+}
+
+int keepkv_decode_step_host(const keepkv_params *p, const keepkv_cache *cache, const void *q_host,
+                            const void *k_new_host, const void *v_new_host, void *out_host, void *q_dev,
+                            void *k_new_dev, void *v_new_dev, void *out_dev, int update_scores, void *ws,
+                            size_t ws_bytes, int32_t *status_dev, void *stream) {
+  int rc = validate(p);
+  if (rc) return rc;
+  if ((rc = validate_cache(cache))) return rc;
+  if (!q_host || !k_new_host || !v_new_host || !out_host || !q_dev || !k_new_dev || !v_new_dev || !out_dev || !ws ||
+      !status_dev)
+    return KEEPKV_ERR_INVALID_ARG;
+  if (!aligned(q_dev, 16) || !aligned(k_new_dev, 16) || !aligned(v_new_dev, 16) || !aligned(out_dev, 16) ||
+      !aligned(ws, 256))
+    return KEEPKV_ERR_INVALID_ARG;
+  WsLayout L = ws_layout(*p);
+  if (ws_bytes < L.total) return KEEPKV_ERR_WORKSPACE;
+  LaunchCtx ctx{(cudaStream_t)stream, 0, cudaSuccess};
+  const size_t qb = (size_t)p->B * p->H_q * p->d * 2, kb = (size_t)p->B * p->H_kv * p->d * 2;
+  auto cp = [&](void *dstp, const void *srcp, size_t n, cudaMemcpyKind kind) {
+    cudaError_t e = cudaMemcpyAsync(dstp, srcp, n, kind, ctx.stream);
+    if (e != cudaSuccess && ctx.err == cudaSuccess) ctx.err = e;
+  };
+  cp(q_dev, q_host, qb, cudaMemcpyHostToDevice);
+  cp(k_new_dev, k_new_host, kb, cudaMemcpyHostToDevice);
+  cp(v_new_dev, v_new_host, kb, cudaMemcpyHostToDevice);
+  if (ctx.err == cudaSuccess) launch_append(*p, *cache, k_new_dev, v_new_dev, status_dev, ctx);
+  if (ctx.err == cudaSuccess)
+    launch_decode(*p, *cache, q_dev, out_dev, nullptr, update_scores, (char *)ws, L, status_dev, ctx);
+  if (ctx.err == cudaSuccess) cp(out_host, out_dev, qb, cudaMemcpyDeviceToHost);
+  return finish(ctx);
+}
+
+const char *keepkv_status_string(int status) {
+  switch (status) {
+    case KEEPKV_OK: return "KEEPKV_OK";
+    case KEEPKV_ERR_INVALID_ARG: return "KEEPKV_ERR_INVALID_ARG";
+    case KEEPKV_ERR_UNSUPPORTED: return "KEEPKV_ERR_UNSUPPORTED";
+    case KEEPKV_ERR_CAPACITY: return "KEEPKV_ERR_CAPACITY";
+    case KEEPKV_ERR_WORKSPACE: return "KEEPKV_ERR_WORKSPACE";
+    case KEEPKV_ERR_CUDA: return "KEEPKV_ERR_CUDA";
+    default: return "KEEPKV_UNKNOWN_STATUS";
+  }
+}
+
+int keepkv_last_cuda_error(void) { return g_last_cuda_error; }
+int keepkv_last_launch_count(void) { return g_last_launches; }
+
+}  // extern "C"

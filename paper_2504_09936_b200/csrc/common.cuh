@@ -1,0 +1,80 @@
+// Internal declarations shared by the translation units of libkeepkv (not installed).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+#include "keepkv.h"
+
+namespace keepkv {
+
+constexpr int kTile = 64;          // entries per K/V tile of the decode kernel
+constexpr int kMaxSplits = 64;     // upper bound on split-KV factor
+
+// Byte offsets of the arrays kept in the caller's workspace.  U = B*H_kv, N = N_cap.
+struct WsLayout {
+  size_t counters;    // i32 [U]            split-KV arrival counters (zero between calls)
+  size_t part_ml;     // f32 [U,S,G,2]      split-KV partial (max, sum)
+  size_t part_acc;    // f32 [U,S,G,d]      split-KV partial numerators
+  size_t unit_info;   // i32 [U,4]          len, n_ret, n_ev, budget of the running compression
+  size_t ret_idx;     // i32 [U,N]          source index of each retained slot, ascending
+  size_t target;      // i32 [U,N]          per source entry: slot, -1 dropped, -2 retained
+  size_t ev_idx;      // i32 [U,N]          source indices of evicted entries, ascending
+  size_t dst_norm;    // f32 [U,N]          sqrt of the fp32 chain norm of each retained key
+  size_t umax;        // f32 [U,N]          winning cosine of each evicted entry
+  size_t cand;        // i32 [U,N,2]        nominated slots of each evicted entry
+  size_t grp_ptr;     // i32 [U,N+1]        CSR offsets of the members of each slot
+  size_t grp_fill;    // i32 [U,N]          running fill positions
+  size_t grp_mem;     // i32 [U,N]          CSR members (source indices), ascending per slot
+  size_t stats;       // keepkv_stats [U]   used when the caller passes no stats array
+  size_t total;
+  int max_splits;
+};
+
+WsLayout ws_layout(const keepkv_params &p);
+int choose_splits(const keepkv_params &p, int max_splits);
+
+struct LaunchCtx {
+  cudaStream_t stream;
+  int launches;
+  cudaError_t err;
+};
+
+// launchers (each returns cudaSuccess or the launch error and bumps ctx.launches)
+void launch_append(const keepkv_params &p, const keepkv_cache &c, const void *k_new, const void *v_new,
+                   int32_t *status_dev, LaunchCtx &ctx);
+void launch_decode(const keepkv_params &p, const keepkv_cache &c, const void *q, void *out, float *lse,
+                   int update_scores, char *ws, const WsLayout &L, int32_t *status_dev, LaunchCtx &ctx);
+void launch_compress(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
+                     const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev, int32_t *ret_idx,
+                     int32_t *target, keepkv_stats *stats, char *ws, const WsLayout &L, int32_t *status_dev,
+                     LaunchCtx &ctx);
+
+#define KEEPKV_CHECK_LAUNCH(ctx)                        \
+  do {                                                  \
+    cudaError_t e__ = cudaGetLastError();               \
+    (ctx).launches++;                                   \
+    if (e__ != cudaSuccess && (ctx).err == cudaSuccess) \
+      (ctx).err = e__;                                  \
+  } while (0)
+
+// ---------------------------------------------------------------- device helpers
+__device__ __forceinline__ float bf16_lo(uint32_t x) { return __uint_as_float(x << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t x) { return __uint_as_float(x & 0xffff0000u); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t *>(&t);
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+}  // namespace keepkv

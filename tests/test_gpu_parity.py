@@ -1,0 +1,277 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded inputs.  Integer results (retained sets, merge targets, votes, lengths) must be identical;
+floating-point tensors obey the rules in tests/helpers.py."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from helpers import (HostCache, bits_to_dev, check_close, check_compress_unit, check_decode_unit, f32_to_dev_bf16,
+                     oracle_params, random_cache, to_f64, workload_cache, workload_params)
+from paper_2504_09936_b200 import binding as kb
+from paper_2504_09936_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+def _q(p, seed):
+    rng = np.random.default_rng(seed)
+    return f32_to_dev_bf16(rng.standard_normal((p.B, p.H_q, p.d)).astype(np.float32))
+
+
+def _run_decode(p, cache, q, update):
+    ws = kb.new_workspace(p)
+    st = kb.new_status()
+    out = torch.empty_like(q)
+    lse = torch.empty(p.B, p.H_q, dtype=torch.float32, device="cuda")
+    kb.keepkv_decode_attention(p, cache, q, out, lse, update, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    return out, lse
+
+
+@pytest.mark.parametrize("G,d", [(1, 64), (2, 64), (4, 64), (8, 64), (1, 128), (2, 128), (4, 128), (8, 128)])
+def test_decode_small_shapes_ragged(G, d):
+    """Eq. 6 + Eq. 8 on several tiles with ragged tails, votes > 1 and a mix of scored / unscored entries."""
+    H_kv, B = 2, 6
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=576, ema_alpha=0.9)
+    lens = [0, 1, 63, 64, 201, 576]
+    cache = random_cache(p, lens, seed=G * 100 + d, vote_max=5, scored_frac=0.7)
+    q = _q(p, 7)
+    hc = HostCache(cache)
+    out, lse = _run_decode(p, cache, q, True)
+    ls_after = to_f64(cache.lscore).reshape(B * H_kv, -1)
+    q64, o64, l64 = to_f64(q), to_f64(out), to_f64(lse)
+    for u in range(B * H_kv):
+        check_decode_unit(p, u, hc, q64, o64, l64, ls_after, what=f"G={G} d={d}")
+    # entries past seq_len are never touched
+    ls_before = hc.lscore
+    for u in range(B * H_kv):
+        n = lens[u // H_kv]
+        assert np.array_equal(ls_after[u, n:], ls_before[u, n:], equal_nan=True)
+
+
+def test_decode_without_score_update_leaves_lscore():
+    p = kb.make_params(B=2, H_q=8, H_kv=2, d=128, N_cap=256)
+    cache = random_cache(p, [256, 100], seed=3)
+    before = cache.lscore.clone()
+    _run_decode(p, cache, _q(p, 1), False)
+    assert torch.equal(before, cache.lscore)
+
+
+def test_decode_alpha_zero_and_votes_one_is_plain_attention():
+    """alpha = 0: the estimate is the last score; p = 1: Eq. 6 is Eq. 3 (library SDPA as reference)."""
+    p = kb.make_params(B=1, H_q=4, H_kv=4, d=128, N_cap=320, ema_alpha=0.0)
+    cache = random_cache(p, [300], seed=5)
+    q = _q(p, 2)
+    out, _ = _run_decode(p, cache, q, True)
+    K, V = cache.K.double().cpu()[:, :, :300], cache.V.double().cpu()[:, :, :300]
+    ref = torch.nn.functional.scaled_dot_product_attention(q.double().cpu()[:, :, None, :], K, V)[:, :, 0]
+    check_close(to_f64(out), O.round_bf16(ref.numpy()), "sdpa")
+    ell = (q.double().cpu()[:, :, None, :] @ K.transpose(-1, -2))[0, :, 0] / math.sqrt(128)
+    check_close(to_f64(cache.lscore)[0, :, :300], ell.numpy(), "lscore=logit", ulps=None, max_abs=1e-4, mean_rel=1e-5)
+
+
+def test_append_equation_2_and_full_cache_flag():
+    p = kb.make_params(B=3, H_q=4, H_kv=2, d=64, N_cap=64)
+    cache = random_cache(p, [0, 10, 64], seed=1)
+    before = HostCache(cache)
+    rng = np.random.default_rng(0)
+    kn = f32_to_dev_bf16(rng.standard_normal((3, 2, 64)).astype(np.float32))
+    vn = f32_to_dev_bf16(rng.standard_normal((3, 2, 64)).astype(np.float32))
+    st = kb.new_status()
+    kb.keepkv_append(p, cache, kn, vn, st)
+    torch.cuda.synchronize()
+    after = HostCache(cache)
+    assert list(after.seq_len) == [1, 11, 64]
+    assert int(st.item()) == 1                      # KEEPKV_DEV_APPEND_FULL for the third sequence
+    kn64, vn64 = to_f64(kn), to_f64(vn)
+    for b, pos in ((0, 0), (1, 10)):
+        for h in range(2):
+            u = b * 2 + h
+            Kc, Vc, vc, lc = before.K[u].copy(), before.V[u].copy(), before.votes[u].copy(), before.lscore[u].copy()
+            O.append(Kc, Vc, vc, lc, pos, kn64[b, h], vn64[b, h])
+            assert np.array_equal(after.K[u], Kc) and np.array_equal(after.V[u], Vc)
+            assert np.array_equal(after.votes[u], vc) and np.array_equal(after.lscore[u], lc)
+    for h in range(2):                              # the full sequence is untouched
+        assert np.array_equal(after.K[4 + h], before.K[4 + h]) and np.array_equal(after.votes[4 + h], before.votes[4 + h])
+
+
+def _run_compress(p, src, budget, n_recent_dev=None):
+    dst = kb.Cache.empty(p)
+    ws = kb.new_workspace(p)
+    st = kb.new_status()
+    U = p.B * p.H_kv
+    ret = torch.full((U, p.N_cap), -7, dtype=torch.int32, device="cuda")
+    tgt = torch.full((U, p.N_cap), -7, dtype=torch.int32, device="cuda")
+    stats = torch.zeros(U, 8, dtype=torch.int32, device="cuda")
+    kb.keepkv_compress(p, src, dst, budget, ws, st, n_recent_dev=n_recent_dev, retained_idx=ret, target=tgt,
+                       stats=stats)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    return dst, ret.cpu().numpy(), tgt.cpu().numpy(), stats.cpu().numpy()
+
+
+@pytest.mark.parametrize("d,G", [(64, 4), (128, 1), (128, 8)])
+@pytest.mark.parametrize("T,guard", [(0.8, True), (-math.inf, True), (-math.inf, False), (0.2, True)])
+def test_compress_staged_parity(d, G, T, guard):
+    """Algorithm 1 on ragged units with votes > 1: retained sets, targets, votes exact; K, V, lscore close."""
+    B, H_kv = 4, 2
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=768, period=64, n_sink=4, n_recent=20,
+                       merge_threshold=T, gamma_min=0.0 if guard else -math.inf, gamma_max=4.0 if guard else math.inf)
+    lens = [700, 333, 40, 130]
+    src = random_cache(p, lens, seed=d + G, vote_max=3, scored_frac=1.0)
+    # a few exactly equal scores so that the tie rule (lowest index) is exercised
+    src.lscore[:, :, 50:60] = src.lscore[:, :, 50:51]
+    budget = 70
+    dst, ret, tgt, stats = _run_compress(p, src, budget)
+    hs, hd = HostCache(src), HostCache(dst)
+    n_full = 0
+    for u in range(B * H_kv):
+        _, full = check_compress_unit(p, u, budget, p.n_recent, hs, hd, ret, tgt, stats, what=f"T={T}")
+        n_full += full
+    assert n_full >= B * H_kv - 1
+
+
+def test_compress_ragged_budgets_and_copy_through():
+    """Per-sequence budgets and recent windows; a sequence within its budget is copied in order."""
+    B, H_kv, G, d = 3, 2, 2, 128
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=512, period=0, n_sink=4, merge_threshold=-math.inf)
+    lens = [500, 90, 257]
+    src = random_cache(p, lens, seed=11, vote_max=2)
+    budgets = np.array([50, 100, 26], dtype=np.int32)
+    nrec = np.array([36, 70, 17], dtype=np.int32)
+    dst, ret, tgt, stats = _run_compress(p, src, torch.from_numpy(budgets).cuda(), torch.from_numpy(nrec).cuda())
+    hs, hd = HostCache(src), HostCache(dst)
+    assert list(hd.seq_len) == [50, 90, 26]
+    for u in range(B * H_kv):
+        b = u // H_kv
+        check_compress_unit(p, u, int(budgets[b]), int(nrec[b]), hs, hd, ret, tgt, stats, what="ragged")
+    for h in range(H_kv):
+        assert np.array_equal(hd.K[2 + h, :90], hs.K[2 + h, :90]) and np.array_equal(hd.votes[2 + h, :90], hs.votes[2 + h, :90])
+
+
+def test_compress_degenerate_budgets():
+    p = kb.make_params(B=2, H_q=2, H_kv=2, d=64, N_cap=128, period=0, n_sink=4, n_recent=8,
+                       merge_threshold=-math.inf)
+    src = random_cache(p, [100, 0], seed=2)
+    for budget in (0, 1, 3, 5, 12):
+        dst, ret, tgt, stats = _run_compress(p, src, budget)
+        hs, hd = HostCache(src), HostCache(dst)
+        assert list(hd.seq_len) == [budget, 0]
+        for u in range(4):
+            check_compress_unit(p, u, budget, p.n_recent, hs, hd, ret, tgt, stats, what=f"budget={budget}")
+
+
+def test_single_step_lossless_on_gpu():
+    """Theorem 2 through the library (G = 1, alpha = 0, T = -inf): decode, compress, decode again with
+    the same query.  The merged rows are stored in bf16, so equality holds to bf16 resolution."""
+    p = kb.make_params(B=2, H_q=4, H_kv=4, d=128, N_cap=1024, period=0, n_sink=0, n_recent=0, ema_alpha=0.0,
+                       merge_threshold=-math.inf, gamma_min=-math.inf, gamma_max=math.inf)
+    cache = random_cache(p, [1000, 600], seed=21, scored_frac=0.0, scale=0.3)
+    # a common positive offset and a constant query keep every logit near +1.4, away from the
+    # singular point of the rescale factor (scores straddling 1), so bf16 storage is the only error
+    cache.K.add_(0.5)
+    q = torch.full((p.B, p.H_q, p.d), 0.25, dtype=torch.bfloat16, device="cuda")
+    out0, lse0 = _run_decode(p, cache, q, True)
+    votes_before = to_f64(cache.votes)
+    dst, ret, tgt, stats = _run_compress(p, cache, 300)
+    out1, lse1 = _run_decode(p, dst, q, False)
+    assert np.all(stats[:, 2] == stats[:, 1])                       # every evicted entry merged
+    hd = HostCache(dst)
+    for u in range(8):
+        n0 = [1000, 600][u // 4]
+        assert hd.votes[u, :300].sum() == n0                        # Electoral Votes are conserved
+    check_close(to_f64(out1), to_f64(out0), "lossless out", ulps=None, max_abs=2e-2, mean_rel=2e-2)
+    check_close(to_f64(lse1), to_f64(lse0), "lossless lse", ulps=None, max_abs=2e-2, mean_rel=1e-3)
+
+
+def test_c1_protocol_free_running():
+    """Config C1 end to end: score the prompt, compress 512 -> 51, then 32 x (append, decode) on both
+    sides independently; final compression checked teacher-forced."""
+    w = W.CONFIGS["C1"]
+    p = workload_params(w, ema_alpha=0.9, merge_threshold=0.8)
+    P = oracle_params(p)
+    cache = workload_cache(w, n_cap=p.N_cap)
+    ws, st = kb.new_workspace(p), kb.new_status()
+    q_all, kn_all, vn_all = W.make_step_inputs(w, 0, 0, w.steps + 1)
+    out = torch.empty(w.B, w.H_q, w.d, dtype=torch.bfloat16, device="cuda")
+    # step 0: decode on the full prompt with score update, then the first compression
+    hc0 = HostCache(cache)
+    q0 = bits_to_dev(q_all[0])
+    kb.keepkv_decode_attention(p, cache, q0, out, None, True, ws, st)
+    torch.cuda.synchronize()
+    for u in range(w.U):
+        check_decode_unit(p, u, hc0, to_f64(q0), to_f64(out), None, to_f64(cache.lscore).reshape(w.U, -1), "C1 step0")
+    b = w.budget()
+    hs = HostCache(cache)
+    dst, ret, tgt, stats = _run_compress(p, cache, b)
+    hd = HostCache(dst)
+    orc = []
+    for u in range(w.U):
+        ref, _ = check_compress_unit(p, u, b, p.n_recent, hs, hd, ret, tgt, stats, what="C1 compress", sorted_select=False)
+        n_cap = p.N_cap
+        st_u = dict(K=np.zeros((n_cap, w.d)), V=np.zeros((n_cap, w.d)), votes=np.zeros(n_cap), ls=np.zeros(n_cap), n=b)
+        st_u["K"][:b], st_u["V"][:b], st_u["votes"][:b], st_u["ls"][:b] = ref["K"], ref["V"], ref["votes"], ref["lscore"]
+        orc.append(st_u)
+    # free-running decode: oracle continues from ITS compressed state, GPU from its own
+    cur = dst
+    for t in range(1, w.steps + 1):
+        q = bits_to_dev(q_all[t]); kn = bits_to_dev(kn_all[t]); vn = bits_to_dev(vn_all[t])
+        kb.keepkv_append(p, cur, kn, vn, st)
+        kb.keepkv_decode_attention(p, cur, q, out, None, True, ws, st)
+        torch.cuda.synchronize()
+        o64, q64, kn64, vn64 = to_f64(out), to_f64(q), to_f64(kn), to_f64(vn)
+        for u in range(w.U):
+            s = orc[u]
+            bb, h = divmod(u, w.H_kv)
+            s["n"] = O.append(s["K"], s["V"], s["votes"], s["ls"], s["n"], kn64[bb, h], vn64[bb, h])
+            n = s["n"]
+            qu = q64[bb, h * w.G:(h + 1) * w.G]
+            o_ref, _ = O.decode(P, qu, s["K"][:n], s["V"][:n], s["votes"][:n])
+            s["ls"][:n] = O.score_update(P, qu, s["K"][:n], s["ls"][:n])
+            check_close(o64[bb, h * w.G:(h + 1) * w.G], O.round_bf16(o_ref), f"C1 step {t} u={u}", ulps=2.0)
+    assert int(st.item()) == 0
+    assert int(cur.seq_len[0]) == b + w.steps
+    ls_gpu = to_f64(cur.lscore).reshape(w.U, -1)
+    for u in range(w.U):
+        check_close(ls_gpu[u, :orc[u]["n"]], orc[u]["ls"][:orc[u]["n"]], "C1 final lscore", ulps=None, max_abs=1e-3,
+                    mean_rel=1e-4)
+    # second compression (b + 32 -> b), teacher-forced on the GPU's state
+    hs = HostCache(cur)
+    dst2, ret, tgt, stats = _run_compress(p, cur, b)
+    hd = HostCache(dst2)
+    for u in range(w.U):
+        check_compress_unit(p, u, b, p.n_recent, hs, hd, ret, tgt, stats, what="C1 second compress", sorted_select=False)
+
+
+def test_decode_step_host_matches_separate_calls():
+    p = kb.make_params(B=2, H_q=8, H_kv=2, d=128, N_cap=256)
+    c1 = random_cache(p, [100, 200], seed=4)
+    c2 = kb.Cache(c1.K.clone(), c1.V.clone(), c1.votes.clone(), c1.lscore.clone(), c1.seq_len.clone())
+    ws, st = kb.new_workspace(p), kb.new_status()
+    rng = np.random.default_rng(5)
+    mk = lambda *s: torch.from_numpy(W.f32_to_bf16_bits(rng.standard_normal(s).astype(np.float32)).view(np.int16)).view(torch.bfloat16).pin_memory()
+    qh, kh, vh = mk(2, 8, 128), mk(2, 2, 128), mk(2, 2, 128)
+    oh = torch.empty(2, 8, 128, dtype=torch.bfloat16).pin_memory()
+    qd, kd, vd, od = (torch.empty_like(t, device="cuda") for t in (qh, kh, vh, oh))
+    kb.keepkv_decode_step_host(p, c1, qh, kh, vh, oh, qd, kd, vd, od, True, ws, st)
+    torch.cuda.synchronize()
+    out2 = torch.empty(2, 8, 128, dtype=torch.bfloat16, device="cuda")
+    kb.keepkv_append(p, c2, kh.cuda(), vh.cuda(), st)
+    kb.keepkv_decode_attention(p, c2, qh.cuda(), out2, None, True, ws, st)
+    torch.cuda.synchronize()
+    assert torch.equal(oh.cuda(), out2) and torch.equal(c1.lscore, c2.lscore) and torch.equal(c1.K, c2.K)
+    assert list(c1.seq_len.cpu()) == [101, 201]
+
+
+def test_decode_is_deterministic():
+    p = kb.make_params(B=2, H_q=8, H_kv=2, d=128, N_cap=2048)
+    cache = random_cache(p, [2048, 1500], seed=8, vote_max=3)
+    q = _q(p, 3)
+    a, la = _run_decode(p, cache, q, False)
+    for _ in range(3):
+        b2, lb = _run_decode(p, cache, q, False)
+        assert torch.equal(a, b2) and torch.equal(la, lb)
