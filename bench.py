@@ -1,0 +1,395 @@
+#!/usr/bin/env python
+"""Benchmark of the KeepKV hot path on B200.
+
+One "step" is one compression period of the steady-state decode loop of a workload
+(default C2, the Llama-3-8B-shaped layer): P x (append one token, decode attention with
+score update) followed by one compression (budget + P -> budget), for every one of
+`--layers` independent layer caches visited round-robin, so that no call finds its
+cache in L2.  value = decode tokens/s of one layer = B * P * layers / step time.
+
+  python bench.py [--gpus N --steps K --warmup W] [--impl reference]
+
+N > 1 (torchrun): every rank runs its own replica of the batch (the path shards by
+sequence with no collective); value is the sum over ranks over the slowest rank's time.
+`--impl reference` times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2504_09936_b200 import workloads as W  # noqa: E402
+
+METRIC = "decode tokens/s + compress GB/s, fraction of HBM roofline"
+UNIT = "tokens/s"
+
+
+def peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            m = json.load(f)
+        return float(m["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def decode_bytes(w, entries_total):
+    """Algorithmic bytes of one decode call: per entry K and V rows, votes, lscore read+write;
+    plus queries and outputs."""
+    return entries_total * (4 * w.d + 12) + 4 * w.B * w.H_q * w.d
+
+
+def compress_bytes(w, len_, b, m):
+    """Algorithmic bytes of one compression, all units: every key once, values of kept and merged
+    entries, votes+lscore of every entry, and the rows written."""
+    per_unit = len_ * 2 * w.d + (b + m) * 2 * w.d + len_ * 8 + b * (4 * w.d + 8)
+    return w.U * per_unit
+
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms",
+                                       "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1])); mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- CPU oracle legs
+
+_SAMPLE = {}
+
+
+def oracle_period_time(w, n_units, n_decode, seed_layer=0):
+    """Times the oracle, as it stands, on `n_units` units of the workload in its steady state:
+    `n_decode` decode steps (Eq. 6 + Eq. 8) at length b + P/2 and one compression b + P -> b.
+    Returns (seconds for a whole period of all U units extrapolated, threads, description, ...)."""
+    import oracle as O
+    b, P = w.budget(), w.period
+    n_cap = b + P
+    nu = min(n_units, w.U)
+    key = (w.name, nu, n_decode, seed_layer)
+    if key not in _SAMPLE:
+        K = np.zeros((nu, n_cap, w.d)); V = np.zeros((nu, n_cap, w.d))
+        for u in range(nu):
+            c = W.make_unit(w, seed_layer, u, n_cap)
+            K[u], V[u] = c["K"], c["V"]
+        q = np.stack([W.make_queries(w, seed_layer, u, 0, n_decode + 1) for u in range(nu)], axis=1).astype(np.float64)
+        _SAMPLE[key] = (K, V, q)
+    K, V, q = _SAMPLE[key]
+    votes = np.ones((nu, n_cap)); ls = np.full((nu, n_cap), -np.inf)
+    Pm = O.Params(G=w.G, d=w.d, n_sink=w.n_sink, n_recent=w.n_recent(), storage_faithful=True, ema_alpha=0.9)
+    lens_mid = np.full(nu, b + P // 2, dtype=np.int32)
+    O.decode_batch(Pm, np.full(nu, n_cap, dtype=np.int32), np.ascontiguousarray(q[0]), K, V, votes, ls, True)
+    t0 = time.perf_counter()
+    for t in range(n_decode):
+        O.decode_batch(Pm, lens_mid, np.ascontiguousarray(q[t + 1]), K, V, votes, ls, True)
+    t_dec = (time.perf_counter() - t0) / n_decode
+    t0 = time.perf_counter()
+    O.compress_batch(Pm, np.full(nu, n_cap, dtype=np.int32), np.full(nu, b, dtype=np.int32), K, V, votes, ls)
+    t_cmp = time.perf_counter() - t0
+    scale = w.U / nu
+    period_s = (P * t_dec + t_cmp) * scale
+    desc = (f"{nu} of {w.U} units; {n_decode} of {P} decode steps at len {b + P // 2} and one compression "
+            f"{b + P}->{b}, extrapolated to a whole period of all units")
+    return period_s, O.num_threads(), desc, t_dec * scale, t_cmp * scale
+
+
+def run_reference(args, w, rank):
+    if rank != 0:
+        return
+    t_all = []
+    for _ in range(min(args.warmup, 1)):
+        oracle_period_time(w, w.U, 8)
+    info = None
+    for _ in range(args.steps):
+        info = oracle_period_time(w, w.U, 8)
+        t_all.append(info[0])
+    period_s = float(np.mean(t_all))
+    val = w.B * w.period / period_s
+    cpu = {"value": val, "unit": UNIT, "cores": info[1], "kind": "oracle", "sample": info[2]}
+    print(json.dumps({"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": period_s * 1e3,
+                      "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+                      "data": "synthetic", "config": config_dict(w, args, "cpu"), "cpu_baseline": cpu,
+                      "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                      "gpu_launches": 0}))
+
+
+def config_dict(w, args, l2):
+    return {"workload": f"{w.name}: B={w.B}, {w.H_q}q/{w.H_kv}kv heads, d={w.d}, N={w.N}, budget {w.budget()} "
+                        f"({w.budget_ratio:.0%}), period {w.period}; steady-state compression period",
+            "layers_round_robin": args.layers, "l2": l2, "parallelism": f"replicas x{args.gpus}"}
+
+
+# --------------------------------------------------------------------------- GPU leg
+
+def run_ours(args, w, rank, world):
+    import torch
+    from paper_2504_09936_b200 import binding as kb
+
+    local = int(os.environ.get("LOCAL_RANK", 0))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    kb.lib()  # fails loudly when the CUDA library is missing
+    L, P, b = args.layers, w.period, w.budget()
+    n_cap = -(-(w.N + P) // 64) * 64
+    p = kb.make_params(B=w.B, H_q=w.H_q, H_kv=w.H_kv, d=w.d, N_cap=n_cap, period=P, n_sink=w.n_sink,
+                       n_recent=w.n_recent(), ema_alpha=0.9, merge_threshold=0.8)
+    dev = lambda bits: torch.from_numpy(bits.view(np.int16)).cuda().view(torch.bfloat16)
+
+    # inputs: one seeded prompt cache (per rank its own seed offset), replicated into L distinct buffers
+    Kb, Vb, lens = W.make_cache(w, layer=rank, n_cap=n_cap)
+    K0, V0 = dev(Kb).view(w.B, w.H_kv, n_cap, w.d), dev(Vb).view(w.B, w.H_kv, n_cap, w.d)
+    del Kb, Vb
+    A = [kb.Cache(K0.clone(), V0.clone(), torch.ones(w.B, w.H_kv, n_cap, device="cuda"),
+                  torch.full((w.B, w.H_kv, n_cap), -math.inf, device="cuda"), torch.from_numpy(lens).cuda())
+         for _ in range(L)]
+    Bc = [kb.Cache.empty(p) for _ in range(L)]
+    del K0, V0
+    qb, knb, vnb = W.make_step_inputs(w, rank, 0, P + 1)
+    q_all, kn_all, vn_all = dev(qb), dev(knb), dev(vnb)
+    ws, st = kb.new_workspace(p), kb.new_status()
+    out = torch.empty(w.B, w.H_q, w.d, dtype=torch.bfloat16, device="cuda")
+    stream = torch.cuda.Stream()
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    launches = 0
+
+    with torch.cuda.stream(stream):
+        # ---- phase 0: score the prompt on the full cache, then the first (full) compression
+        for l in range(L):   # warm
+            kb.keepkv_decode_attention(p, A[l], q_all[0], out, None, False, ws, st)
+        stream.synchronize()
+        e0, e1 = ev(), ev()
+        e0.record()
+        for l in range(L):
+            kb.keepkv_decode_attention(p, A[l], q_all[0], out, None, True, ws, st)
+        e1.record(); stream.synchronize()
+        t_full_decode = e0.elapsed_time(e1) * 1e-3 / L
+        stats = torch.zeros(L, w.U, 8, dtype=torch.int32, device="cuda")
+        e0.record()
+        for l in range(L):
+            kb.keepkv_compress(p, A[l], Bc[l], b, ws, st, stats=stats[l])
+        e1.record(); stream.synchronize()
+        t_full_compress = e0.elapsed_time(e1) * 1e-3 / L
+        m_full = float(stats[:, :, 2].sum().item()) / (L * w.U)
+        compress_launches = kb.last_launch_count()
+
+        # ---- one period as a CUDA graph, in both directions (src/dst swap after every compression)
+        def period(cur, oth, stats_t=None):
+            n = 0
+            for t in range(P):
+                for l in range(L):
+                    kb.keepkv_append(p, cur[l], kn_all[t + 1], vn_all[t + 1], st)
+                    kb.keepkv_decode_attention(p, cur[l], q_all[t + 1], out, None, True, ws, st)
+                    n += 2
+            for l in range(L):
+                kb.keepkv_compress(p, cur[l], oth[l], b, ws, st, stats=None if stats_t is None else stats_t[l])
+                n += compress_launches
+            return n
+
+        graphs = []
+        per_period = 0
+        period(Bc, A); period(A, Bc)          # eager warm-up of both directions (also loads every kernel)
+        stream.synchronize()
+        for cur, oth in ((Bc, A), (A, Bc)):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=stream):
+                per_period = period(cur, oth, stats)
+            graphs.append(g)
+        for k in range(args.warmup):
+            graphs[k % 2].replay()
+        stream.synchronize()
+        if dist is not None:
+            dist.barrier()
+        sampler = ClockSampler(local) if rank == 0 else None
+        torch.cuda.synchronize()
+        e0.record()
+        for k in range(args.steps):
+            graphs[(args.warmup + k) % 2].replay()
+        e1.record()
+        torch.cuda.synchronize()
+        t_steps = e0.elapsed_time(e1) * 1e-3
+        launches = per_period * args.steps
+        clocks = sampler.stop() if sampler else None
+        m_inc = float(stats[:, :, 2].sum().item()) / (L * w.U)
+        assert int(st.item()) == 0, "device status flag raised during the benchmark"
+
+        # ---- dominant kernel alone: decode over the round-robin layers at mid-period length
+        cur = (Bc, A)[(args.warmup + args.steps) % 2]
+        for l in range(L):
+            cur[l].seq_len.fill_(b + P // 2)
+        reps = 16
+        gd = torch.cuda.CUDAGraph()
+        for l in range(L):
+            kb.keepkv_decode_attention(p, cur[l], q_all[1], out, None, True, ws, st)
+        stream.synchronize()
+        with torch.cuda.graph(gd, stream=stream):
+            for _ in range(reps):
+                for l in range(L):
+                    kb.keepkv_decode_attention(p, cur[l], q_all[1], out, None, True, ws, st)
+        gd.replay(); stream.synchronize()
+        e0.record(); gd.replay(); e1.record(); stream.synchronize()
+        t_decode = e0.elapsed_time(e1) * 1e-3 / (reps * L)
+        # ---- compression alone (incremental, budget + P -> budget)
+        for l in range(L):
+            cur[l].seq_len.fill_(b + P)
+        oth = A if cur is Bc else Bc
+        e0.record()
+        for l in range(L):
+            kb.keepkv_compress(p, cur[l], oth[l], b, ws, st)
+        e1.record(); stream.synchronize()
+        t_inc_compress = e0.elapsed_time(e1) * 1e-3 / L
+
+        # ---- end to end through the host-buffer entry point: pinned inputs in, outputs back, every step
+        pin = lambda t: t.cpu().pin_memory()
+        qh, knh, vnh = pin(q_all), pin(kn_all), pin(vn_all)
+        oh = torch.empty(w.B, w.H_q, w.d, dtype=torch.bfloat16).pin_memory()
+        qd, kd, vd = torch.empty_like(q_all[0]), torch.empty_like(kn_all[0]), torch.empty_like(vn_all[0])
+        for l in range(L):
+            oth[l].seq_len.fill_(b)
+
+        def period_e2e(cur, oth):
+            for t in range(P):
+                for l in range(L):
+                    kb.keepkv_decode_step_host(p, cur[l], qh[t + 1], knh[t + 1], vnh[t + 1], oh, qd, kd, vd, out, True,
+                                               ws, st)
+                stream.synchronize()          # the next token's queries depend on this step's output
+            for l in range(L):
+                kb.keepkv_compress(p, cur[l], oth[l], b, ws, st)
+
+        pair = [(oth, cur), (cur, oth)]
+        period_e2e(*pair[0]); period_e2e(*pair[1])
+        stream.synchronize()
+        n_e2e = max(2, min(args.steps, 6))
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for k in range(n_e2e):
+            period_e2e(*pair[k % 2])
+        torch.cuda.synchronize()
+        t_e2e = (time.perf_counter() - t0) / n_e2e
+
+    # ---- reduce over ranks: slowest rank's time, summed tokens
+    if dist is not None:
+        tt = torch.tensor([t_steps, t_e2e], device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        t_steps, t_e2e = float(tt[0]), float(tt[1])
+    tokens_per_step = w.B * P * L * world
+    value = tokens_per_step * args.steps / t_steps
+    e2e_val = tokens_per_step / t_e2e
+    hbm, src = peaks()
+    entries = w.U * (b + P // 2)
+    ach = decode_bytes(w, entries) / t_decode / 1e9
+    full_dec_gbs = decode_bytes(w, int(lens.astype(np.int64).sum()) * w.H_kv) / t_full_decode / 1e9
+    inc_gbs = compress_bytes(w, b + P, b, m_inc) / t_inc_compress / 1e9
+    full_gbs = compress_bytes(w, w.N, b, m_full) / t_full_compress / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": t_steps / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 storage, fp32 accumulate", "data": "synthetic",
+        "config": config_dict(w, args, f"each call works on one of {L} distinct layer caches visited round-robin "
+                                       f"({L} x {decode_bytes(w, entries) / 1e6:.0f} MB > 126 MB L2)"),
+        "clocks": clocks, "gpu_launches": launches,
+        "e2e": {"value": e2e_val, "unit": UNIT,
+                "h2d_bytes_per_step": int(L * P * (q_all[0].numel() + 2 * kn_all[0].numel()) * 2),
+                "d2h_bytes_per_step": int(L * P * out.numel() * 2), "steps": n_e2e,
+                "note": "keepkv_decode_step_host per layer and step, stream sync after every decode step"},
+        "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": ach, "peak": hbm, "unit": "GB/s",
+                     "frac": ach / hbm, "peak_source": src, "traffic": None,
+                     "bytes_per_launch": decode_bytes(w, entries), "us_per_launch": t_decode * 1e6},
+        "phases": {
+            "decode_steady_us": t_decode * 1e6, "decode_steady_gbs": ach, "decode_steady_frac_hbm": ach / hbm,
+            "decode_full_cache_us": t_full_decode * 1e6, "decode_full_cache_gbs": full_dec_gbs,
+            "decode_full_cache_frac_hbm": full_dec_gbs / hbm,
+            "compress_incremental_us": t_inc_compress * 1e6, "compress_incremental_gbs": inc_gbs,
+            "compress_incremental_frac_hbm": inc_gbs / hbm, "merged_per_unit_incremental": m_inc,
+            "compress_full_us": t_full_compress * 1e6, "compress_full_gbs": full_gbs,
+            "compress_full_frac_hbm": full_gbs / hbm, "merged_per_unit_full": m_full,
+            "compress_full_gemm_tflops": 2.0 * (w.N - b) * b * w.d * w.U / t_full_compress / 1e12,
+        },
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            period_s, cores, desc, _, _ = oracle_period_time(w, w.U, 32)
+            line["cpu_baseline"] = {"value": w.B * P / period_s, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": desc}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=8)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C2", choices=sorted(W.CONFIGS))
+    ap.add_argument("--layers", type=int, default=8)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    rank = int(os.environ.get("RANK", 0))
+    world = int(os.environ.get("WORLD_SIZE", 1))
+    w = W.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w, rank)
+    else:
+        run_ours(args, w, rank, world)
+
+
+if __name__ == "__main__":
+    main()
