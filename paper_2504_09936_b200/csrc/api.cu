@@ -42,9 +42,9 @@ WsLayout ws_layout(const keepkv_params &p) {
 }
 
 int choose_splits(const keepkv_params &p, int max_splits) {
-  // Two resident CTAs per SM: aim at a whole number of waves of 296 CTAs.
+  // Two resident CTAs per SM: the largest split factor that still fits one wave of 296 CTAs.
   const int U = p.B * p.H_kv;
-  int S = (2 * 148 + U - 1) / U;
+  int S = (2 * 148) / U;
   if (S < 1) S = 1;
   if (S > max_splits) S = max_splits;
   return S;
