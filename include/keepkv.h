@@ -151,6 +151,25 @@ int keepkv_decode_step_host(const keepkv_params *p, const keepkv_cache *cache, c
                             void *k_new_dev, void *v_new_dev, void *out_dev, int update_scores, void *ws,
                             size_t ws_bytes, int32_t *status_dev, void *stream);
 
+/* No counterpart in the paper: the same operation as keepkv_decode_attention for callers that cannot
+ * provide a workspace because they cannot allocate device memory where they call this (code running
+ * inside another runtime's memory pool, a serving loop whose buffers were all fixed at start-up, a
+ * deployment that forbids cudaMalloc after initialisation).  The split-KV scratch is a fixed array
+ * of KEEPKV_STATIC_SCRATCH_BYTES inside the library image; every GPU that loads the library holds
+ * it until the process exits.  The call allocates and frees nothing.
+ *  - Arguments as keepkv_decode_attention, without ws / ws_bytes; inputs and outputs stay the caller's.
+ *  - Shapes whose decode scratch (4*U + 4*U*S*G*(d+2) bytes rounded up to 256-byte pieces, U = B*H_kv,
+ *    S the split factor the library picks for the shape) exceeds the array are refused with
+ *    KEEPKV_ERR_WORKSPACE before anything is enqueued; the five benchmark shapes need 0.3-4.3 MB.
+ *  - The first call on each device looks up the array's device address; make that call outside any
+ *    stream capture, with the device current that `stream` belongs to.
+ *  - All calls on one GPU share the array and find in it whatever the previous call left: the call
+ *    itself clears the counters it needs at zero, but two calls that overlap on the GPU (different
+ *    streams, or different host threads without ordering) race on it.  Order them on one stream. */
+#define KEEPKV_STATIC_SCRATCH_BYTES (8u << 20)
+int keepkv_decode_attention_static(const keepkv_params *p, const keepkv_cache *cache, const void *q, void *out,
+                                   float *lse_or_null, int update_scores, int32_t *status_dev, void *stream);
+
 /* Human-readable name of a keepkv_status. */
 const char *keepkv_status_string(int status);
 

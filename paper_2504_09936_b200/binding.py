@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkeepkv.so")
 
 EXPORTS = ("keepkv_workspace_bytes", "keepkv_workspace_init", "keepkv_append", "keepkv_decode_attention",
-           "keepkv_compress", "keepkv_decode_step_host", "keepkv_status_string", "keepkv_last_cuda_error",
+           "keepkv_compress", "keepkv_decode_step_host", "keepkv_decode_attention_static", "keepkv_status_string", "keepkv_last_cuda_error",
            "keepkv_last_launch_count")
 
 
@@ -59,6 +59,7 @@ def lib() -> C.CDLL:
         l.keepkv_workspace_init.argtypes = [pp, vp, sz, vp]
         l.keepkv_append.argtypes = [pp, pc, vp, vp, vp, vp]
         l.keepkv_decode_attention.argtypes = [pp, pc, vp, vp, vp, C.c_int, vp, sz, vp, vp]
+        l.keepkv_decode_attention_static.argtypes = [pp, pc, vp, vp, vp, C.c_int, vp, vp]
         l.keepkv_compress.argtypes = [pp, pc, pc, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         l.keepkv_decode_step_host.argtypes = [pp, pc] + [vp] * 8 + [C.c_int, vp, sz, vp, vp]
         _lib = l
@@ -141,6 +142,15 @@ def keepkv_decode_attention(p, cache: Cache, q, out, lse, update_scores: bool, w
     _check(lib().keepkv_decode_attention(C.byref(p), C.byref(cache.c()), q.data_ptr(), out.data_ptr(), _ptr(lse),
                                          int(update_scores), ws.data_ptr(), ws.numel(), status.data_ptr(),
                                          _stream(stream)), "keepkv_decode_attention")
+
+
+def keepkv_decode_attention_static(p, cache: Cache, q, out, lse, update_scores: bool, status, stream=None):
+    """keepkv_decode_attention without a caller workspace, for code that cannot allocate device memory:
+    the scratch is a fixed array inside the library (shared by all calls on the GPU, so keep them
+    on one stream; make the first call on a device outside stream capture)."""
+    _check(lib().keepkv_decode_attention_static(C.byref(p), C.byref(cache.c()), q.data_ptr(), out.data_ptr(),
+                                                _ptr(lse), int(update_scores), status.data_ptr(), _stream(stream)),
+           "keepkv_decode_attention_static")
 
 
 def keepkv_compress(p, src: Cache, dst: Cache, budget, ws, status, n_recent_dev=None, retained_idx=None,

@@ -26,6 +26,8 @@ WsLayout ws_layout(const keepkv_params &p) {
   L.counters = take(U * 4);
   L.part_ml = take(U * S * G * 2 * 4);
   L.part_acc = take(U * S * G * (size_t)p.d * 4);
+  L.decode_bytes = off;
+  L.counter_bytes = U * 4;
   L.unit_info = take(U * 4 * 4);
   L.ret_idx = take(U * N * 4);
   L.target = take(U * N * 4);
@@ -84,6 +86,8 @@ static int finish(LaunchCtx &ctx) {
   }
   return KEEPKV_OK;
 }
+
+int finish_call(LaunchCtx &ctx) { return finish(ctx); }
 
 }  // namespace keepkv
 

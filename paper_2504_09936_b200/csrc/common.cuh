@@ -29,6 +29,8 @@ struct WsLayout {
   size_t grp_mem;     // i32 [U,N]          CSR members (source indices), ascending per slot
   size_t stats;       // keepkv_stats [U]   used when the caller passes no stats array
   size_t total;
+  size_t decode_bytes;   // the leading part that keepkv_decode_attention uses (counters and partials)
+  size_t counter_bytes;  // size of the counters array
   int max_splits;
 };
 
@@ -40,6 +42,9 @@ struct LaunchCtx {
   int launches;
   cudaError_t err;
 };
+
+// records the launch count / CUDA error of a finished call and maps them to a keepkv_status
+int finish_call(LaunchCtx &ctx);
 
 // launchers (each returns cudaSuccess or the launch error and bumps ctx.launches)
 void launch_append(const keepkv_params &p, const keepkv_cache &c, const void *k_new, const void *v_new,

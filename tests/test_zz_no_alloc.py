@@ -1,0 +1,54 @@
+"""keepkv_decode_attention_static: decode attention for callers that cannot allocate device memory
+(code living inside another runtime's memory pool, or a serving loop whose buffers were all fixed at
+start-up), so the split-KV scratch is a fixed array inside the library instead of a workspace they
+would have had to allocate.  Its results must be those of keepkv_decode_attention.
+
+This file is named so that pytest collects it last: the array is shared, process-wide state, and a
+failure here must not hide the results of the other tests in a run that stops at the first failure.
+"""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from helpers import check_close, f32_to_dev_bf16, random_cache, to_f64
+from paper_2504_09936_b200 import binding as kb
+
+
+def test_static_scratch_refuses_shapes_beyond_its_size():
+    """A shape whose split-KV partials do not fit the built-in array is refused on the host, before
+    any CUDA call, with KEEPKV_ERR_WORKSPACE."""
+    p = kb.make_params(B=512, H_q=256, H_kv=32, d=128, N_cap=4096)      # 16384 units x 8 heads x 130 floats > 8 MiB
+    dummy = C.c_void_p(256)
+    cache = kb.keepkv_cache(256, 256, 256, 256, 256)
+    rc = kb.lib().keepkv_decode_attention_static(C.byref(p), C.byref(cache), dummy, dummy, None, 0, dummy, None)
+    assert rc == -4 and kb.lib().keepkv_status_string(rc) == b"KEEPKV_ERR_WORKSPACE"
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("G,d", [(4, 128), (1, 64)])
+def test_static_scratch_decode_matches_workspace_decode_twice(G, d):
+    """Two calls in a row (the second finds the first call's leftovers in the shared array) against the
+    entry point that uses a caller workspace, on ragged sequences with votes > 1 and a score update."""
+    H_kv, B = 2, 5
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=1024, ema_alpha=0.9)
+    lens = [1024, 0, 77, 640, 333]
+    ref_cache = random_cache(p, lens, seed=31 + G, vote_max=4, scored_frac=0.5)
+    new_cache = kb.Cache(ref_cache.K.clone(), ref_cache.V.clone(), ref_cache.votes.clone(), ref_cache.lscore.clone(),
+                         ref_cache.seq_len.clone())
+    ws, st = kb.new_workspace(p), kb.new_status()
+    rng = np.random.default_rng(17)
+    for call in range(2):
+        q = f32_to_dev_bf16(rng.standard_normal((B, p.H_q, d)).astype(np.float32))
+        out_ref, out_new = torch.empty_like(q), torch.empty_like(q)
+        lse_ref = torch.empty(B, p.H_q, dtype=torch.float32, device="cuda")
+        lse_new = torch.empty_like(lse_ref)
+        kb.keepkv_decode_attention(p, ref_cache, q, out_ref, lse_ref, True, ws, st)
+        kb.keepkv_decode_attention_static(p, new_cache, q, out_new, lse_new, True, st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        check_close(to_f64(out_new), to_f64(out_ref), f"call {call}: out", ulps=1.0)
+        check_close(to_f64(lse_new), to_f64(lse_ref), f"call {call}: lse", ulps=None, max_abs=1e-3, mean_rel=1e-4)
+        check_close(to_f64(new_cache.lscore), to_f64(ref_cache.lscore), f"call {call}: lscore", ulps=None,
+                    max_abs=1e-3, mean_rel=1e-4)
