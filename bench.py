@@ -198,8 +198,23 @@ def run_ours(args, w, rank, world):
          for _ in range(L)]
     Bc = [kb.Cache.empty(p) for _ in range(L)]
     del K0, V0
-    qb, knb, vnb = W.make_step_inputs(w, rank, 0, P + 1)
-    q_all, kn_all, vn_all = dev(qb), dev(knb), dev(vnb)
+    # step inputs: step 0 scores the prompt; after it every period draws P fresh steps (a token is never appended
+    # twice, which would plant exact duplicates of keys in the cache).  The graphs read the current period's
+    # inputs from q_all/kn_all/vn_all[1:], refreshed from the pool by a device copy before every replay.
+    n_e2e = max(2, min(args.steps, 6))
+    n_pool = 2 + args.warmup + args.steps + 1 + 2 + n_e2e
+    qb, knb, vnb = W.make_step_inputs(w, rank, 0, n_pool * P + 1)
+    q_pool, kn_pool, vn_pool = dev(qb), dev(knb), dev(vnb)
+    q_all, kn_all, vn_all = q_pool[:P + 1].clone(), kn_pool[:P + 1].clone(), vn_pool[:P + 1].clone()
+    pool_next = [0]
+
+    def load_period():
+        k = pool_next[0]
+        pool_next[0] += 1
+        assert k < n_pool
+        sl = slice(1 + k * P, 1 + (k + 1) * P)
+        q_all[1:].copy_(q_pool[sl]); kn_all[1:].copy_(kn_pool[sl]); vn_all[1:].copy_(vn_pool[sl])
+        return sl
     ws, st = kb.new_workspace(p), kb.new_status()
     out = torch.empty(w.B, w.H_q, w.d, dtype=torch.bfloat16, device="cuda")
     stream = torch.cuda.Stream()
@@ -241,7 +256,8 @@ def run_ours(args, w, rank, world):
 
         graphs = []
         per_period = 0
-        period(Bc, A); period(A, Bc)          # eager warm-up of both directions (also loads every kernel)
+        load_period(); period(Bc, A)          # eager warm-up of both directions (also loads every kernel)
+        load_period(); period(A, Bc)
         stream.synchronize()
         for cur, oth in ((Bc, A), (A, Bc)):
             g = torch.cuda.CUDAGraph()
@@ -249,6 +265,7 @@ def run_ours(args, w, rank, world):
                 per_period = period(cur, oth, stats)
             graphs.append(g)
         for k in range(args.warmup):
+            load_period()
             graphs[k % 2].replay()
         stream.synchronize()
         if dist is not None:
@@ -257,62 +274,69 @@ def run_ours(args, w, rank, world):
         torch.cuda.synchronize()
         e0.record()
         for k in range(args.steps):
+            load_period()
             graphs[(args.warmup + k) % 2].replay()
         e1.record()
         torch.cuda.synchronize()
         t_steps = e0.elapsed_time(e1) * 1e-3
         launches = per_period * args.steps
         clocks = sampler.stop() if sampler else None
-        m_inc = float(stats[:, :, 2].sum().item()) / (L * w.U)
         assert int(st.item()) == 0, "device status flag raised during the benchmark"
 
         # ---- dominant kernel alone: decode over the round-robin layers at mid-period length
         cur = (Bc, A)[(args.warmup + args.steps) % 2]
-        for l in range(L):
-            cur[l].seq_len.fill_(b + P // 2)
+        oth = A if cur is Bc else Bc
+        load_period()
+        for t in range(P // 2):              # a real half period with fresh tokens
+            for l in range(L):
+                kb.keepkv_append(p, cur[l], kn_all[t + 1], vn_all[t + 1], st)
+                kb.keepkv_decode_attention(p, cur[l], q_all[t + 1], out, None, True, ws, st)
         reps = 16
         gd = torch.cuda.CUDAGraph()
-        for l in range(L):
-            kb.keepkv_decode_attention(p, cur[l], q_all[1], out, None, True, ws, st)
         stream.synchronize()
         with torch.cuda.graph(gd, stream=stream):
             for _ in range(reps):
                 for l in range(L):
-                    kb.keepkv_decode_attention(p, cur[l], q_all[1], out, None, True, ws, st)
+                    kb.keepkv_decode_attention(p, cur[l], q_all[P // 2], out, None, True, ws, st)
         gd.replay(); stream.synchronize()
         e0.record(); gd.replay(); e1.record(); stream.synchronize()
         t_decode = e0.elapsed_time(e1) * 1e-3 / (reps * L)
-        # ---- compression alone (incremental, budget + P -> budget)
-        for l in range(L):
-            cur[l].seq_len.fill_(b + P)
-        oth = A if cur is Bc else Bc
-        e0.record()
-        for l in range(L):
-            kb.keepkv_compress(p, cur[l], oth[l], b, ws, st)
-        e1.record(); stream.synchronize()
-        t_inc_compress = e0.elapsed_time(e1) * 1e-3 / L
+        # ---- compression alone (incremental, budget + P -> budget), as a graph of the L calls
+        for t in range(P // 2, P):
+            for l in range(L):
+                kb.keepkv_append(p, cur[l], kn_all[t + 1], vn_all[t + 1], st)
+                kb.keepkv_decode_attention(p, cur[l], q_all[t + 1], out, None, True, ws, st)
+        gc = torch.cuda.CUDAGraph()
+        stream.synchronize()
+        with torch.cuda.graph(gc, stream=stream):
+            for l in range(L):
+                kb.keepkv_compress(p, cur[l], oth[l], b, ws, st, stats=stats[l])
+        gc.replay(); stream.synchronize()
+        e0.record(); gc.replay(); gc.replay(); e1.record(); stream.synchronize()
+        t_inc_compress = e0.elapsed_time(e1) * 1e-3 / (2 * L)
+        m_inc = float(stats[:, :, 2].sum().item()) / (L * w.U)
+        cur, oth = oth, cur                   # the compressed caches are current now
 
         # ---- end to end through the host-buffer entry point: pinned inputs in, outputs back, every step
         pin = lambda t: t.cpu().pin_memory()
-        qh, knh, vnh = pin(q_all), pin(kn_all), pin(vn_all)
+        qh, knh, vnh = pin(q_pool), pin(kn_pool), pin(vn_pool)
         oh = torch.empty(w.B, w.H_q, w.d, dtype=torch.bfloat16).pin_memory()
         qd, kd, vd = torch.empty_like(q_all[0]), torch.empty_like(kn_all[0]), torch.empty_like(vn_all[0])
-        for l in range(L):
-            oth[l].seq_len.fill_(b)
-
         def period_e2e(cur, oth):
+            k = pool_next[0]
+            pool_next[0] += 1
+            assert k < n_pool
             for t in range(P):
+                i = 1 + k * P + t
                 for l in range(L):
-                    kb.keepkv_decode_step_host(p, cur[l], qh[t + 1], knh[t + 1], vnh[t + 1], oh, qd, kd, vd, out, True,
-                                               ws, st)
+                    kb.keepkv_decode_step_host(p, cur[l], qh[i], knh[i], vnh[i], oh, qd, kd, vd, out, True, ws, st)
                 stream.synchronize()          # the next token's queries depend on this step's output
             for l in range(L):
                 kb.keepkv_compress(p, cur[l], oth[l], b, ws, st)
 
-        pair = [(oth, cur), (cur, oth)]
+        pair = [(cur, oth), (oth, cur)]
         period_e2e(*pair[0]); period_e2e(*pair[1])
         stream.synchronize()
-        n_e2e = max(2, min(args.steps, 6))
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()

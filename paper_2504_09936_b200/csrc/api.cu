@@ -28,16 +28,23 @@ WsLayout ws_layout(const keepkv_params &p) {
   L.part_acc = take(U * S * G * (size_t)p.d * 4);
   L.decode_bytes = off;
   L.counter_bytes = U * 4;
-  L.unit_info = take(U * 4 * 4);
+  L.unit_info = take(U * sizeof(UnitInfo));
+  L.sched = take(4 * 4);
+  size_t C = (2 * 148 + U - 1) / U;
+  if (C < 1) C = 1;
+  if (C > (size_t)kNomChunksMax) C = kNomChunksMax;
+  L.nom_chunks = (int)C;
+  size_t Np2 = 1;
+  while (Np2 < N) Np2 <<= 1;
+  L.key_stride = (int)Np2;
   L.ret_idx = take(U * N * 4);
   L.target = take(U * N * 4);
   L.ev_idx = take(U * N * 4);
-  L.dst_norm = take(U * N * 4);
-  L.umax = take(U * N * 4);
-  L.cand = take(U * N * 2 * 4);
-  L.grp_ptr = take(U * (N + 1) * 4);
-  L.grp_fill = take(U * N * 4);
-  L.grp_mem = take(U * N * 4);
+  L.inv_norm = take(U * N * 4);
+  L.nom_v = take(U * N * C * 16);
+  L.nom_si = take(U * N * C * 4);
+  L.grp_key = take(U * Np2 * 4);
+  L.grp_head = take(U * N * 4);
   L.stats = take(U * sizeof(keepkv_stats));
   L.total = off;
   return L;
@@ -70,6 +77,19 @@ static int validate(const keepkv_params *p) {
 }
 
 static bool aligned(const void *ptr, size_t a) { return (reinterpret_cast<uintptr_t>(ptr) % a) == 0; }
+
+int sm_count() {
+  static int n[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  dev &= 63;
+  if (!n[dev]) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+    n[dev] = v;
+  }
+  return n[dev];
+}
 
 static int validate_cache(const keepkv_cache *c) {
   if (!c || !c->K || !c->V || !c->votes || !c->lscore || !c->seq_len) return KEEPKV_ERR_INVALID_ARG;
@@ -152,6 +172,7 @@ int keepkv_compress(const keepkv_params *p, const keepkv_cache *src, const keepk
       src->seq_len == dst->seq_len)
     return KEEPKV_ERR_INVALID_ARG;
   if (!ws || !status_dev || !aligned(ws, 256)) return KEEPKV_ERR_INVALID_ARG;
+  if ((long long)p->B * p->H_kv > kMaxUnits) return KEEPKV_ERR_UNSUPPORTED;
   if (!budget_dev) {
     if (budget_scalar < 0) return KEEPKV_ERR_INVALID_ARG;
     if (budget_scalar > p->N_cap || (long long)budget_scalar + p->period > p->N_cap) return KEEPKV_ERR_CAPACITY;

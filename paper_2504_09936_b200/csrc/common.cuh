@@ -12,26 +12,33 @@ namespace keepkv {
 constexpr int kTile = 64;          // entries per K/V tile of the decode kernel
 constexpr int kMaxSplits = 64;     // upper bound on split-KV factor
 
+constexpr int kMaxUnits = 4096;    // B * H_kv that keepkv_compress accepts (per-unit tables live in shared memory)
+constexpr int kNomChunksMax = 8;   // upper bound on the column chunks a row's similarity search is split into
+
+struct UnitInfo { int len, n_ret, n_ev, n_groups; };
+
 // Byte offsets of the arrays kept in the caller's workspace.  U = B*H_kv, N = N_cap.
 struct WsLayout {
   size_t counters;    // i32 [U]            split-KV arrival counters (zero between calls)
   size_t part_ml;     // f32 [U,S,G,2]      split-KV partial (max, sum)
   size_t part_acc;    // f32 [U,S,G,d]      split-KV partial numerators
-  size_t unit_info;   // i32 [U,4]          len, n_ret, n_ev, budget of the running compression
+  size_t unit_info;   // UnitInfo [U]       len, n_ret, n_ev, n_groups of the running compression
+  size_t sched;       // i32 [4]            column-chunk count the nomination kernel settled on
   size_t ret_idx;     // i32 [U,N]          source index of each retained slot, ascending
   size_t target;      // i32 [U,N]          per source entry: slot, -1 dropped, -2 retained
   size_t ev_idx;      // i32 [U,N]          source indices of evicted entries, ascending
-  size_t dst_norm;    // f32 [U,N]          sqrt of the fp32 chain norm of each retained key
-  size_t umax;        // f32 [U,N]          winning cosine of each evicted entry
-  size_t cand;        // i32 [U,N,2]        nominated slots of each evicted entry
-  size_t grp_ptr;     // i32 [U,N+1]        CSR offsets of the members of each slot
-  size_t grp_fill;    // i32 [U,N]          running fill positions
-  size_t grp_mem;     // i32 [U,N]          CSR members (source indices), ascending per slot
+  size_t inv_norm;    // f32 [U,N]          1/|k| of each retained key (tree-summed; only ranks candidates)
+  size_t nom_v;       // float4 [U,N,C]     per evicted row and column chunk: best, second, third cosine, best slot
+  size_t nom_si;      // i32 [U,N,C]        slot of the second-best cosine
+  size_t grp_key;     // u32 [U,Npow2]      (slot << 16 | evicted position) of merged entries, sorted
+  size_t grp_head;    // i32 [U,N]          position in grp_key where each group starts
   size_t stats;       // keepkv_stats [U]   used when the caller passes no stats array
   size_t total;
   size_t decode_bytes;   // the leading part that keepkv_decode_attention uses (counters and partials)
   size_t counter_bytes;  // size of the counters array
   int max_splits;
+  int nom_chunks;        // C: column chunks reserved per evicted row
+  int key_stride;        // Npow2: N rounded up to a power of two
 };
 
 WsLayout ws_layout(const keepkv_params &p);
@@ -55,6 +62,11 @@ void launch_compress(const keepkv_params &p, const keepkv_cache &src, const keep
                      const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev, int32_t *ret_idx,
                      int32_t *target, keepkv_stats *stats, char *ws, const WsLayout &L, int32_t *status_dev,
                      LaunchCtx &ctx);
+// tcgen05 similarity search: for every evicted key the three largest cosines over the retained keys
+void launch_nominate(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst, const int32_t *ev_idx,
+                     const UnitInfo *unit_info, const float *inv_norm, int32_t *sched, float4 *nom_v, int32_t *nom_si,
+                     int nom_chunks, int32_t *status_dev, LaunchCtx &ctx);
+int sm_count();
 
 #define KEEPKV_CHECK_LAUNCH(ctx)                        \
   do {                                                  \

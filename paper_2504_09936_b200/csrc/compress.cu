@@ -1,14 +1,15 @@
 // keepkv_compress: Algorithm 1 of the paper, out of place, one (sequence, kv-head) unit at a time.
-//   select  -> retained / evicted sets from the key kappa = ln p + lscore        (lines 2-3)
-//   compact -> retained rows copied to dst in ascending source order             (line 11)
-//   match   -> cosine arg-max of every evicted key over the retained keys        (lines 4-5)
-//   group   -> members of each retained slot, ascending                          (many-to-one, App. A.2)
-//   merge   -> Eq. A.3 with the EMA estimate as score                            (lines 7-10)
+//   select   -> retained / evicted sets from the key kappa = ln p + lscore       (lines 2-3)
+//   compact  -> retained rows copied to dst in ascending source order            (line 11)
+//   nominate -> three best cosines of every evicted key over the retained keys,
+//               on the tensor cores (nominate.cu)                                (line 4)
+//   resolve  -> arg-max and threshold of line 5, decided in the interface's fixed fp32
+//               arithmetic wherever the tensor-core ranking is too close to call; members
+//               of each retained slot sorted into groups                         (many-to-one, App. A.2)
+//   merge    -> Eq. A.3 with the EMA estimate as score                           (lines 7-10)
 #include "common.cuh"
 
 namespace keepkv {
-
-struct UnitInfo { int len, n_ret, n_ev, budget; };
 
 // ------------------------------------------------------------------ block scan of 0/1 flags
 // Exclusive prefix count of `flag` over the block in thread order; total returned through `total`.
@@ -101,22 +102,45 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
   if (n_heavy > 0) {
     uint32_t prefix = 0, mask = 0;
     int kr = n_heavy;
+    const int lane = tid & 31;
     for (int pass = 3; pass >= 0; --pass) {
       if (tid < 256) hist[tid] = 0;
       __syncthreads();
-      for (int i = lo + tid; i < hi; i += blockDim.x) {
-        const uint32_t k = keys[i];
-        if ((k & mask) == prefix) atomicAdd(&hist[(k >> (8 * pass)) & 255u], 1);
+      for (int start = lo; start < hi; start += blockDim.x) {
+        const int i = start + tid;
+        const uint32_t k = i < hi ? keys[i] : 0u;
+        const bool in = i < hi && (k & mask) == prefix;
+        // one shared-memory atomic per distinct bin of the warp (the leading bytes of most keys coincide)
+        const int bin = in ? (int)((k >> (8 * pass)) & 255u) : -1 - lane;
+        const unsigned peers = __match_any_sync(0xffffffffu, bin);
+        if (in && lane == __ffs(peers) - 1) atomicAdd(&hist[bin], __popc(peers));
       }
       __syncthreads();
-      if (tid == 0) {
-        int cum = 0, bin = 255;
-        for (; bin > 0; --bin) {
-          if (cum + hist[bin] >= kr) break;
-          cum += hist[bin];
+      if (tid < 32) {
+        // bins are scanned from the top: lane l owns bins 8l..8l+7
+        int c[8], s = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { c[j] = hist[8 * lane + j]; s += c[j]; }
+        int x = s;   // becomes the count in bins of lanes >= lane
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int y = __shfl_down_sync(0xffffffffu, x, o);
+          if (lane + o < 32) x += y;
         }
-        s_prefix = prefix | ((uint32_t)bin << (8 * pass));
-        s_kr = kr - cum;
+        const int above = x - s;
+        if (above < kr && x >= kr) {
+          int cum = above, bin = 0;
+          bool found = false;
+#pragma unroll
+          for (int j = 7; j >= 0; --j) {
+            if (!found) {
+              if (cum + c[j] >= kr) { bin = j; found = true; }
+              else cum += c[j];
+            }
+          }
+          s_prefix = prefix | ((uint32_t)(8 * lane + bin) << (8 * pass));
+          s_kr = kr - cum;
+        }
       }
       __syncthreads();
       prefix = s_prefix;
@@ -152,300 +176,344 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
     base_keep += tot_keep;
   }
   if (tid == 0) {
-    UnitInfo ui{len, base_keep, len - base_keep, budget};
+    UnitInfo ui{len, base_keep, len - base_keep, 0};
     unit_info[u] = ui;
     if (h == 0) dst_seq_len[b] = base_keep;
     keepkv_stats st;
-    st.n_retained = base_keep; st.n_evicted = len - base_keep; st.n_merged = 0; st.n_below_T = 0;
+    st.n_retained = base_keep; st.n_evicted = len - base_keep; st.n_merged = 0;
+    st.n_below_T = len - base_keep;   // resolve_kernel replaces this once targets are known
     st.n_guard_groups = 0; st.n_groups = 0; st.max_group = 0; st.reserved = 0;
     stats[u] = st;
   }
 }
 
 // ------------------------------------------------------------------ compact
-// grid (ceil(bound/32), U), 256 threads: 32 retained rows per CTA.  A warp moves a K row with its
-// lower half and the V row with its upper half; afterwards 32 threads run the fp32 norm chain.
+// grid (ceil(bound/64), U), 256 threads.  Sixteen lanes move one retained row (a 16-byte piece of
+// K and of V each); a warp has eight rows in flight.  The same lanes tree-sum the squared key for
+// the inverse norm the similarity search ranks with.
 template <int D>
 __global__ void __launch_bounds__(256)
-compact_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_t *ret_idx, const UnitInfo *unit_info,
-               float *dst_norm) {
+compact_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_t *__restrict__ ret_idx,
+               const UnitInfo *__restrict__ unit_info, float *__restrict__ inv_norm) {
   constexpr int CH = D / 8;       // 16-byte chunks per row
-  constexpr int RS = D + 8;       // padded row stride (bf16 elements) in shared memory
-  __shared__ __align__(16) __nv_bfloat16 Ks[32 * RS];
-  const int u = blockIdx.y, s0 = blockIdx.x * 32;
-  const int n_ret = unit_info[u].n_ret;
+  const int u = blockIdx.y, n_ret = unit_info[u].n_ret;
+  const int s0 = blockIdx.x * 64;
   if (s0 >= n_ret) return;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, ch = lane & 15, sub = lane >> 4;
   const size_t base = (size_t)u * p.N_cap;
   const uint4 *sK = reinterpret_cast<const uint4 *>(src.K), *sV = reinterpret_cast<const uint4 *>(src.V);
   uint4 *dK = reinterpret_cast<uint4 *>(dst.K), *dV = reinterpret_cast<uint4 *>(dst.V);
-  for (int idx = threadIdx.x; idx < 32 * CH * 2; idx += blockDim.x) {
-    const int r = idx / (2 * CH), rem = idx % (2 * CH), isv = rem / CH, j = rem % CH;
-    const int slot = s0 + r;
-    if (slot >= n_ret) continue;
-    const int si = ret_idx[base + slot];
-    if (isv) {
-      dV[(base + slot) * CH + j] = sV[(base + si) * CH + j];
-    } else {
-      const uint4 v = sK[(base + si) * CH + j];
-      dK[(base + slot) * CH + j] = v;
-      *reinterpret_cast<uint4 *>(&Ks[r * RS + j * 8]) = v;
+  int slot[4], si[4];
+  uint4 kv[4], vv[4];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    slot[r] = s0 + warp * 8 + r * 2 + sub;
+    si[r] = slot[r] < n_ret ? ret_idx[base + slot[r]] : -1;
+  }
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    kv[r] = make_uint4(0, 0, 0, 0);
+    vv[r] = kv[r];
+    if (si[r] >= 0 && ch < CH) {
+      kv[r] = sK[(base + si[r]) * CH + ch];
+      vv[r] = sV[(base + si[r]) * CH + ch];
     }
   }
-  __syncthreads();
-  if (threadIdx.x < 32) {
-    const int slot = s0 + threadIdx.x;
-    if (slot < n_ret) {
-      const int si = ret_idx[base + slot];
-      float acc = 0.f;
-      for (int j = 0; j < D; ++j) {
-        const float x = __bfloat162float(Ks[threadIdx.x * RS + j]);
-        acc = fmaf(x, x, acc);
-      }
-      dst_norm[base + slot] = sqrtf(acc);
-      dst.votes[base + slot] = src.votes[base + si];
-      dst.lscore[base + slot] = src.lscore[base + si];
+#pragma unroll
+  for (int r = 0; r < 4; ++r) {
+    if (si[r] >= 0 && ch < CH) {
+      dK[(base + slot[r]) * CH + ch] = kv[r];
+      dV[(base + slot[r]) * CH + ch] = vv[r];
+    }
+    float ss = 0.f;
+    const uint32_t w[4] = {kv[r].x, kv[r].y, kv[r].z, kv[r].w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) { const float a = bf16_lo(w[q]), b = bf16_hi(w[q]); ss = fmaf(a, a, ss); ss = fmaf(b, b, ss); }
+    ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+    ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+    ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+    ss += __shfl_xor_sync(0xffffffffu, ss, 8);
+    if (si[r] >= 0 && ch == 0) {
+      inv_norm[base + slot[r]] = rsqrtf(ss);
+      dst.votes[base + slot[r]] = src.votes[base + si[r]];
+      dst.lscore[base + slot[r]] = src.lscore[base + si[r]];
     }
   }
 }
 
-// ------------------------------------------------------------------ match (exact fp32 chain)
-// grid (ceil(N_cap/64), U), 256 threads as 16x16; each thread owns a 4x4 block of the
-// 64 evicted x 64 retained cosine tile.  Every dot product is accumulated by fused multiply-add
-// from 0 over channels 0..D-1 in order, which is the arithmetic the interface fixes for the
-// cosine, so the arg-max taken here is final.
+// ------------------------------------------------------------------ the cosine the interface defines
+// dot, |a|^2, |b|^2 by sequential fused multiply-add from 0 over channels 0..D-1; a, b point to bf16 rows.
 template <int D>
-__global__ void __launch_bounds__(256)
-match_exact_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_t *ev_idx,
-                   const UnitInfo *unit_info, const float *dst_norm, int32_t *target, float *umax,
-                   keepkv_stats *stats) {
-  constexpr int LD = 68;
-  extern __shared__ float smf[];
-  float *As = smf;                 // [D][LD]  evicted keys, channel-major
-  float *Bs = smf + D * LD;        // [D][LD]  retained keys, channel-major
-  __shared__ float na[64], nb[64];
-  __shared__ float red_v[64][17];
-  __shared__ int red_i[64][17];
-  __shared__ int s_below;
-  const int u = blockIdx.y, r0 = blockIdx.x * 64;
+__device__ __forceinline__ float exact_cosine(const __nv_bfloat16 *a, const __nv_bfloat16 *b) {
+  float dot = 0.f, na = 0.f, nb = 0.f;
+  const uint4 *pa = reinterpret_cast<const uint4 *>(a), *pb = reinterpret_cast<const uint4 *>(b);
+#pragma unroll 4
+  for (int q = 0; q < D / 8; ++q) {
+    const uint4 x = pa[q], y = pb[q];
+    const uint32_t xw[4] = {x.x, x.y, x.z, x.w}, yw[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+      const float x0 = bf16_lo(xw[t]), x1 = bf16_hi(xw[t]), y0 = bf16_lo(yw[t]), y1 = bf16_hi(yw[t]);
+      dot = fmaf(x0, y0, dot); na = fmaf(x0, x0, na); nb = fmaf(y0, y0, nb);
+      dot = fmaf(x1, y1, dot); na = fmaf(x1, x1, na); nb = fmaf(y1, y1, nb);
+    }
+  }
+  return dot / (sqrtf(na) * sqrtf(nb));
+}
+
+// ------------------------------------------------------------------ resolve + group
+// One CTA per unit.  The tensor-core search left, per evicted entry, the three largest cosines
+// (best, second with their slots, third as a value).  Its values differ from the interface's fp32
+// chain only by accumulation order (|diff| far below kRankEps), so:
+//   best - second > eps              the arg-max is settled; otherwise both candidates are re-evaluated
+//                                    with exact_cosine and the larger wins (equal -> lower slot);
+//   best - third  <= eps             three or more candidates too close: the whole row is re-evaluated;
+//   |best - T|    <= eps             the threshold test uses exact_cosine of the winner.
+// Entries to merge are then sorted by (slot, position) so that every group is contiguous and ascending.
+constexpr float kRankEps = 1e-4f;
+constexpr int kResolveThreads = 512;
+
+template <int D>
+__global__ void __launch_bounds__(kResolveThreads)
+resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_t *__restrict__ ev_idx,
+               UnitInfo *unit_info, const float4 *__restrict__ nom_v, const int32_t *__restrict__ nom_si,
+               const int32_t *__restrict__ sched, int C_max, int32_t *__restrict__ target, uint32_t *grp_key,
+               int key_stride, int32_t *__restrict__ grp_head, keepkv_stats *stats, int smem_keys) {
+  extern __shared__ uint32_t key_smem[];
+  __shared__ float ke_s[kResolveThreads / 32][D];
+  __shared__ int warp_tot[32];
+  __shared__ int s_count, s_ndeep[2];
+  __shared__ int s_deep_tid[kResolveThreads], s_deep_e[kResolveThreads], s_deep_slot[kResolveThreads];
+  __shared__ int s_deep_merge[kResolveThreads];
+  const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const UnitInfo ui = unit_info[u];
-  if (r0 >= ui.n_ev) return;
   const size_t base = (size_t)u * p.N_cap;
-  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
   const __nv_bfloat16 *sK = reinterpret_cast<const __nv_bfloat16 *>(src.K) + base * D;
   const __nv_bfloat16 *dK = reinterpret_cast<const __nv_bfloat16 *>(dst.K) + base * D;
-  if (tid == 0) s_below = 0;
-  for (int idx = tid; idx < 64 * (D / 2); idx += 256) {
-    const int r = idx / (D / 2), jj = idx % (D / 2);
-    uint32_t v = 0;
-    if (r0 + r < ui.n_ev) v = *reinterpret_cast<const uint32_t *>(sK + (size_t)ev_idx[base + r0 + r] * D + 2 * jj);
-    As[(2 * jj) * LD + r] = bf16_lo(v);
-    As[(2 * jj + 1) * LD + r] = bf16_hi(v);
-  }
+  int np2 = 1;
+  while (np2 < ui.n_ev) np2 <<= 1;
+  uint32_t *keys = np2 <= smem_keys ? key_smem : grp_key + (size_t)u * key_stride;
+  const int C = sched[0];
+  const float T = p.merge_threshold;
+  if (tid == 0) { s_count = 0; s_ndeep[0] = s_ndeep[1] = 0; }
   __syncthreads();
-  if (tid < 64) {
-    float acc = 0.f;
-    for (int j = 0; j < D; ++j) acc = fmaf(As[j * LD + tid], As[j * LD + tid], acc);
-    na[tid] = sqrtf(acc);
-  }
-  float best[4];
-  int bi[4];
-#pragma unroll
-  for (int r = 0; r < 4; ++r) { best[r] = -CUDART_INF_F; bi[r] = -1; }
 
-  for (int c0 = 0; c0 < ui.n_ret; c0 += 64) {
-    __syncthreads();
-    for (int idx = tid; idx < 64 * (D / 2); idx += 256) {
-      const int c = idx / (D / 2), jj = idx % (D / 2);
-      uint32_t v = 0;
-      if (c0 + c < ui.n_ret) v = *reinterpret_cast<const uint32_t *>(dK + (size_t)(c0 + c) * D + 2 * jj);
-      Bs[(2 * jj) * LD + c] = bf16_lo(v);
-      Bs[(2 * jj + 1) * LD + c] = bf16_hi(v);
-    }
-    if (tid < 64) nb[tid] = (c0 + tid < ui.n_ret) ? dst_norm[base + c0 + tid] : 1.f;
-    __syncthreads();
-    float acc[4][4];
+  for (int j0 = 0; j0 < ui.n_ev; j0 += kResolveThreads) {
+    const int j = j0 + tid;
+    const bool valid = j < ui.n_ev;
+    int e = 0, slot = -1;
+    bool merge = false, deep = false;
+    if (valid) {
+      e = ev_idx[base + j];
+      float best = -CUDART_INF_F, second = -CUDART_INF_F, third = -CUDART_INF_F;
+      int bi = -1, si = -1;
+      for (int c = 0; c < C; ++c) {   // chunks hold ascending slots: strict comparisons keep the lower slot on ties
+        const float4 v = nom_v[(base + j) * C_max + c];
+        const int vi[2] = {__float_as_int(v.w), nom_si[(base + j) * C_max + c]};
+        const float vv[2] = {v.x, v.y};
 #pragma unroll
-    for (int r = 0; r < 4; ++r)
-#pragma unroll
-      for (int c = 0; c < 4; ++c) acc[r][c] = 0.f;
-#pragma unroll 4
-    for (int j = 0; j < D; ++j) {
-      const float4 a = *reinterpret_cast<const float4 *>(&As[j * LD + ty * 4]);
-      const float4 bb = *reinterpret_cast<const float4 *>(&Bs[j * LD + tx * 4]);
-      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {bb.x, bb.y, bb.z, bb.w};
-#pragma unroll
-      for (int r = 0; r < 4; ++r)
-#pragma unroll
-        for (int c = 0; c < 4; ++c) acc[r][c] = fmaf(av[r], bv[c], acc[r][c]);
-    }
-#pragma unroll
-    for (int r = 0; r < 4; ++r)
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int col = c0 + tx * 4 + c;
-        if (col < ui.n_ret) {
-          const float uu = acc[r][c] / (na[ty * 4 + r] * nb[tx * 4 + c]);
-          if (uu > best[r]) { best[r] = uu; bi[r] = col; }
+        for (int t = 0; t < 2; ++t) {
+          if (vv[t] > second) {
+            third = second;
+            if (vv[t] > best) { second = best; si = bi; best = vv[t]; bi = vi[t]; }
+            else { second = vv[t]; si = vi[t]; }
+          } else {
+            third = fmaxf(third, vv[t]);
+          }
+        }
+        third = fmaxf(third, v.z);
+      }
+      if (bi >= 0) {
+        if (!(best - third > kRankEps)) {
+          deep = true;
+        } else {
+          float uu = best;
+          slot = bi;
+          bool exact = false;
+          if (!(best - second > kRankEps)) {
+            const float u1 = exact_cosine<D>(sK + (size_t)e * D, dK + (size_t)bi * D);
+            const float u2 = exact_cosine<D>(sK + (size_t)e * D, dK + (size_t)si * D);
+            uu = u1;
+            if (u2 > u1 || (u2 == u1 && si < bi)) { uu = u2; slot = si; }
+            exact = true;
+          }
+          if (!exact && !(fabsf(best - T) > kRankEps)) uu = exact_cosine<D>(sK + (size_t)e * D, dK + (size_t)slot * D);
+          merge = uu > T;
         }
       }
-  }
+    }
+    // ---- rows whose three best are too close: the whole row in exact arithmetic, one warp per row,
+    //      the rows of this pass shared out over all warps of the CTA
+    const int par = (j0 / kResolveThreads) & 1;
+    if (deep) { const int q = atomicAdd(&s_ndeep[par], 1); s_deep_tid[q] = tid; s_deep_e[q] = e; }
+    __syncthreads();
+    const int n_deep = s_ndeep[par];
+    if (tid == 0) s_ndeep[par ^ 1] = 0;   // the next pass counts in the other word
+    for (int q = warp; q < n_deep; q += kResolveThreads / 32) {
+      const int ee = s_deep_e[q];
+      __syncwarp();
+      for (int c = lane; c < D; c += 32) ke_s[warp][c] = __bfloat162float(sK[(size_t)ee * D + c]);
+      __syncwarp();
+      float ne = 0.f;
+      for (int c = 0; c < D; ++c) ne = fmaf(ke_s[warp][c], ke_s[warp][c], ne);
+      const float sne = sqrtf(ne);
+      float bu = -CUDART_INF_F;
+      int bc = -1;
+      for (int c = lane; c < ui.n_ret; c += 32) {
+        const uint4 *pc = reinterpret_cast<const uint4 *>(dK + (size_t)c * D);
+        float dot = 0.f, nc = 0.f;
+        for (int w = 0; w < D / 8; ++w) {
+          const uint4 y = pc[w];
+          const uint32_t yw[4] = {y.x, y.y, y.z, y.w};
 #pragma unroll
-  for (int r = 0; r < 4; ++r) { red_v[ty * 4 + r][tx] = best[r]; red_i[ty * 4 + r][tx] = bi[r]; }
-  __syncthreads();
-  if (tid < 64 && r0 + tid < ui.n_ev) {
-    float bv = -CUDART_INF_F;
-    int bx = -1;
-    for (int t = 0; t < 16; ++t) {
-      const float v = red_v[tid][t];
-      const int ix = red_i[tid][t];
-      if (ix >= 0 && (v > bv || (v == bv && ix < bx) || bx < 0)) { bv = v; bx = ix; }
-    }
-    const int e = ev_idx[base + r0 + tid];
-    const bool merge = bx >= 0 && bv > p.merge_threshold;
-    target[base + e] = merge ? bx : -1;
-    umax[base + e] = bv;
-    if (!merge) atomicAdd(&s_below, 1);
-  }
-  __syncthreads();
-  if (tid == 0 && s_below) atomicAdd(&stats[u].n_below_T, s_below);
-}
-
-// ------------------------------------------------------------------ group
-// One CTA per unit: count members per slot, scan, then one warp fills the CSR lists walking the
-// evicted entries in ascending order, so that every member list is ascending and the result
-// does not depend on scheduling.
-__global__ void __launch_bounds__(256)
-group_kernel(keepkv_params p, const int32_t *ev_idx, const int32_t *target, const UnitInfo *unit_info,
-             int32_t *grp_ptr, int32_t *grp_fill, int32_t *grp_mem) {
-  __shared__ int warp_tot[32];
-  const int u = blockIdx.x, tid = threadIdx.x;
-  const UnitInfo ui = unit_info[u];
-  const size_t base = (size_t)u * p.N_cap;
-  int32_t *ptr = grp_ptr + (size_t)u * (p.N_cap + 1);
-  volatile int32_t *fill = grp_fill + base;
-  int32_t *mem = grp_mem + base;
-  for (int c = tid; c <= ui.n_ret; c += blockDim.x) ptr[c] = 0;
-  __syncthreads();
-  for (int j = tid; j < ui.n_ev; j += blockDim.x) {
-    const int c = target[base + ev_idx[base + j]];
-    if (c >= 0) atomicAdd(&ptr[c], 1);
-  }
-  __syncthreads();
-  int run = 0;
-  for (int start = 0; start < ui.n_ret; start += blockDim.x) {
-    const int c = start + tid;
-    const int v = c < ui.n_ret ? ptr[c] : 0;
-    int tot;
-    const int ex = run + block_excl_sum(v, warp_tot, tot);
-    if (c < ui.n_ret) { ptr[c] = ex; fill[c] = ex; }
-    run += tot;
-  }
-  if (tid == 0) ptr[ui.n_ret] = run;
-  __syncthreads();
-  if (tid < 32) {
-    const int lane = tid;
-    for (int j0 = 0; j0 < ui.n_ev; j0 += 32) {
-      const int j = j0 + lane;
-      int e = -1, c = -1;
-      if (j < ui.n_ev) { e = ev_idx[base + j]; c = target[base + e]; }
-      const int keyc = c >= 0 ? c : -1 - lane;  // inactive lanes match nobody
-      const unsigned grp = __match_any_sync(0xffffffffu, keyc);
-      if (c >= 0) {
-        const int rank = __popc(grp & ((1u << lane) - 1u));
-        const int pos = fill[c] + rank;
-        mem[pos] = e;
+          for (int t = 0; t < 4; ++t) {
+            const float y0 = bf16_lo(yw[t]), y1 = bf16_hi(yw[t]);
+            dot = fmaf(ke_s[warp][w * 8 + 2 * t], y0, dot); nc = fmaf(y0, y0, nc);
+            dot = fmaf(ke_s[warp][w * 8 + 2 * t + 1], y1, dot); nc = fmaf(y1, y1, nc);
+          }
+        }
+        const float uu = dot / (sne * sqrtf(nc));
+        if (uu > bu) { bu = uu; bc = c; }
       }
-      __syncwarp();
-      if (c >= 0 && (grp >> lane) == 1u) fill[c] = fill[c] + __popc(grp);  // highest lane of the group
-      __syncwarp();
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const float ou = __shfl_xor_sync(0xffffffffu, bu, o);
+        const int oc = __shfl_xor_sync(0xffffffffu, bc, o);
+        if (oc >= 0 && (bc < 0 || ou > bu || (ou == bu && oc < bc))) { bu = ou; bc = oc; }
+      }
+      if (lane == 0) { s_deep_slot[s_deep_tid[q]] = bc; s_deep_merge[s_deep_tid[q]] = bc >= 0 && bu > T; }
     }
+    __syncthreads();
+    if (deep) { slot = s_deep_slot[tid]; merge = s_deep_merge[tid] != 0; }
+    if (valid) {
+      target[base + e] = merge ? slot : -1;
+      if (merge) keys[atomicAdd(&s_count, 1)] = ((uint32_t)slot << 16) | (uint32_t)j;
+    }
+  }
+  __syncthreads();
+  const int M = s_count;
+  int Mp = 1;
+  while (Mp < M) Mp <<= 1;
+  for (int i = M + tid; i < Mp; i += kResolveThreads) keys[i] = 0xFFFFFFFFu;
+  __syncthreads();
+  // ---- bitonic sort, ascending: (slot, position) order makes every group contiguous and ascending
+  for (int k = 2; k <= Mp; k <<= 1) {
+    for (int jj = k >> 1; jj > 0; jj >>= 1) {
+      for (int i = tid; i < Mp; i += kResolveThreads) {
+        const int ixj = i ^ jj;
+        if (ixj > i) {
+          const uint32_t a = keys[i], b = keys[ixj];
+          if ((a > b) == ((i & k) == 0)) { keys[i] = b; keys[ixj] = a; }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  // ---- publish the sorted members and the start of every group
+  uint32_t *gk = grp_key + (size_t)u * key_stride;
+  int n_groups = 0;
+  for (int i0 = 0; i0 < M; i0 += kResolveThreads) {
+    const int i = i0 + tid;
+    const bool head = i < M && (i == 0 || (keys[i] >> 16) != (keys[i - 1] >> 16));
+    int tot;
+    const int pos = n_groups + block_excl_count(head, warp_tot, tot);
+    if (head) grp_head[base + pos] = i;
+    if (i < M && keys != gk) gk[i] = keys[i];
+    n_groups += tot;
+  }
+  if (tid == 0) {
+    grp_head[base + n_groups] = M;
+    unit_info[u].n_groups = n_groups;
+    stats[u].n_below_T = ui.n_ev - M;
   }
 }
 
 // ------------------------------------------------------------------ merge
-// One warp per retained slot that has members.  With a_i = ln p_i + lscore_i over the group
-// K'_e (target first, then members ascending):  omega = softmax(a),  v_r = sum omega_i v_i,
-// k_r = gamma * sum omega_i k_i,  gamma = L / lambda_bar,  L = LSE(a) - ln(sum p),
-// lambda_bar = sum omega_i lscore_i,  p_r = sum p,  lscore_r = L   (Eq. A.3 in logarithms).
+// One warp per group.  With a_i = ln p_i + lscore_i over the group K'_e (target first, then members
+// ascending):  omega = softmax(a),  v_r = sum omega_i v_i,  k_r = gamma * sum omega_i k_i,
+// gamma = L / lambda_bar,  L = LSE(a) - ln(sum p),  lambda_bar = sum omega_i lscore_i,  p_r = sum p,
+// lscore_r = L   (Eq. A.3 in logarithms).
 template <int D>
-__global__ void __launch_bounds__(128)
-merge_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_t *ret_idx, int32_t *target,
-             const UnitInfo *unit_info, const int32_t *grp_ptr, const int32_t *grp_mem, keepkv_stats *stats) {
+__global__ void __launch_bounds__(256)
+merge_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_t *__restrict__ ret_idx,
+             const int32_t *__restrict__ ev_idx, int32_t *target, const UnitInfo *__restrict__ unit_info,
+             const uint32_t *__restrict__ grp_key, int key_stride, const int32_t *__restrict__ grp_head,
+             keepkv_stats *stats) {
   constexpr int EPL = D / 32;
   const int u = blockIdx.y, lane = threadIdx.x & 31;
-  const int c = blockIdx.x * 4 + (threadIdx.x >> 5);
   const UnitInfo ui = unit_info[u];
-  if (c >= ui.n_ret || ui.n_ev == 0) return;
   const size_t base = (size_t)u * p.N_cap;
-  const int32_t *ptr = grp_ptr + (size_t)u * (p.N_cap + 1);
-  const int beg = ptr[c], n = ptr[c + 1] - beg;
-  if (n == 0) return;
-  const int32_t *mem = grp_mem + base + beg;
-  const int ci = ret_idx[base + c];
+  const uint32_t *gk = grp_key + (size_t)u * key_stride;
   const float *votes = src.votes + base, *ls = src.lscore + base;
-
-  const float a_c = logf(votes[ci]) + ls[ci];
-  float M = a_c;
-  for (int t = lane; t < n; t += 32) { const int e = mem[t]; M = fmaxf(M, logf(votes[e]) + ls[e]); }
-  M = warp_max(M);
-  float Z = 0.f, Ps = 0.f;
-  if (lane == 0) { Z = expf(a_c - M); Ps = votes[ci]; }
-  for (int t = lane; t < n; t += 32) { const int e = mem[t]; Z += expf(logf(votes[e]) + ls[e] - M); Ps += votes[e]; }
-  Z = warp_sum(Z);
-  Ps = warp_sum(Ps);
-  const float Lam = M + logf(Z);
-  const float L = Lam - logf(Ps);
-
   const __nv_bfloat16 *sK = reinterpret_cast<const __nv_bfloat16 *>(src.K) + base * D;
   const __nv_bfloat16 *sV = reinterpret_cast<const __nv_bfloat16 *>(src.V) + base * D;
-  float ka[EPL], va[EPL], lbar = 0.f;
+  for (int g = blockIdx.x * 8 + (threadIdx.x >> 5); g < ui.n_groups; g += gridDim.x * 8) {
+    const int beg = grp_head[base + g], n = grp_head[base + g + 1] - beg;
+    const int c = (int)(gk[beg] >> 16);
+    const int ci = ret_idx[base + c];
+    auto member = [&](int t) { return ev_idx[base + (gk[beg + t] & 0xFFFFu)]; };
+
+    const float a_c = logf(votes[ci]) + ls[ci];
+    float M = a_c;
+    for (int t = lane; t < n; t += 32) { const int e = member(t); M = fmaxf(M, logf(votes[e]) + ls[e]); }
+    M = warp_max(M);
+    float Z = 0.f, Ps = 0.f;
+    if (lane == 0) { Z = expf(a_c - M); Ps = votes[ci]; }
+    for (int t = lane; t < n; t += 32) { const int e = member(t); Z += expf(logf(votes[e]) + ls[e] - M); Ps += votes[e]; }
+    Z = warp_sum(Z);
+    Ps = warp_sum(Ps);
+    const float Lam = M + logf(Z);
+    const float L = Lam - logf(Ps);
+
+    float ka[EPL], va[EPL], lbar = 0.f;
 #pragma unroll
-  for (int e = 0; e < EPL; ++e) { ka[e] = 0.f; va[e] = 0.f; }
-  for (int t = -1; t < n; ++t) {
-    const int i = t < 0 ? ci : mem[t];
-    const float lsi = ls[i];
-    const float om = expf(logf(votes[i]) + lsi - Lam);
-    lbar = fmaf(om, lsi, lbar);
-    if constexpr (EPL == 4) {
-      const uint2 kk = *reinterpret_cast<const uint2 *>(sK + (size_t)i * D + lane * 4);
-      const uint2 vv = *reinterpret_cast<const uint2 *>(sV + (size_t)i * D + lane * 4);
-      ka[0] = fmaf(om, bf16_lo(kk.x), ka[0]); ka[1] = fmaf(om, bf16_hi(kk.x), ka[1]);
-      ka[2] = fmaf(om, bf16_lo(kk.y), ka[2]); ka[3] = fmaf(om, bf16_hi(kk.y), ka[3]);
-      va[0] = fmaf(om, bf16_lo(vv.x), va[0]); va[1] = fmaf(om, bf16_hi(vv.x), va[1]);
-      va[2] = fmaf(om, bf16_lo(vv.y), va[2]); va[3] = fmaf(om, bf16_hi(vv.y), va[3]);
-    } else {
-      const uint32_t kk = *reinterpret_cast<const uint32_t *>(sK + (size_t)i * D + lane * 2);
-      const uint32_t vv = *reinterpret_cast<const uint32_t *>(sV + (size_t)i * D + lane * 2);
-      ka[0] = fmaf(om, bf16_lo(kk), ka[0]); ka[1] = fmaf(om, bf16_hi(kk), ka[1]);
-      va[0] = fmaf(om, bf16_lo(vv), va[0]); va[1] = fmaf(om, bf16_hi(vv), va[1]);
+    for (int e = 0; e < EPL; ++e) { ka[e] = 0.f; va[e] = 0.f; }
+    for (int t = -1; t < n; ++t) {
+      const int i = t < 0 ? ci : member(t);
+      const float lsi = ls[i];
+      const float om = expf(logf(votes[i]) + lsi - Lam);
+      lbar = fmaf(om, lsi, lbar);
+      if constexpr (EPL == 4) {
+        const uint2 kk = *reinterpret_cast<const uint2 *>(sK + (size_t)i * D + lane * 4);
+        const uint2 vv = *reinterpret_cast<const uint2 *>(sV + (size_t)i * D + lane * 4);
+        ka[0] = fmaf(om, bf16_lo(kk.x), ka[0]); ka[1] = fmaf(om, bf16_hi(kk.x), ka[1]);
+        ka[2] = fmaf(om, bf16_lo(kk.y), ka[2]); ka[3] = fmaf(om, bf16_hi(kk.y), ka[3]);
+        va[0] = fmaf(om, bf16_lo(vv.x), va[0]); va[1] = fmaf(om, bf16_hi(vv.x), va[1]);
+        va[2] = fmaf(om, bf16_lo(vv.y), va[2]); va[3] = fmaf(om, bf16_hi(vv.y), va[3]);
+      } else {
+        const uint32_t kk = *reinterpret_cast<const uint32_t *>(sK + (size_t)i * D + lane * 2);
+        const uint32_t vv = *reinterpret_cast<const uint32_t *>(sV + (size_t)i * D + lane * 2);
+        ka[0] = fmaf(om, bf16_lo(kk), ka[0]); ka[1] = fmaf(om, bf16_hi(kk), ka[1]);
+        va[0] = fmaf(om, bf16_lo(vv), va[0]); va[1] = fmaf(om, bf16_hi(vv), va[1]);
+      }
     }
-  }
-  const float gamma = L / lbar;
-  const bool ok = gamma > p.gamma_min && gamma <= p.gamma_max && fabsf(lbar) >= 1e-6f;
-  if (!ok) {
-    // guard: the members are dropped after all and the target keeps the row copied by compaction
-    for (int t = lane; t < n; t += 32) target[base + mem[t]] = -1;
-    if (lane == 0) { atomicAdd(&stats[u].n_guard_groups, 1); atomicAdd(&stats[u].n_groups, 1); }
-    return;
-  }
-  __nv_bfloat16 *dK = reinterpret_cast<__nv_bfloat16 *>(dst.K) + (base + c) * D;
-  __nv_bfloat16 *dV = reinterpret_cast<__nv_bfloat16 *>(dst.V) + (base + c) * D;
-  if constexpr (EPL == 4) {
-    uint2 ko, vo;
-    ko.x = pack_bf16(gamma * ka[0], gamma * ka[1]); ko.y = pack_bf16(gamma * ka[2], gamma * ka[3]);
-    vo.x = pack_bf16(va[0], va[1]); vo.y = pack_bf16(va[2], va[3]);
-    *reinterpret_cast<uint2 *>(dK + lane * 4) = ko;
-    *reinterpret_cast<uint2 *>(dV + lane * 4) = vo;
-  } else {
-    *reinterpret_cast<uint32_t *>(dK + lane * 2) = pack_bf16(gamma * ka[0], gamma * ka[1]);
-    *reinterpret_cast<uint32_t *>(dV + lane * 2) = pack_bf16(va[0], va[1]);
-  }
-  if (lane == 0) {
-    dst.votes[base + c] = Ps;
-    dst.lscore[base + c] = L;
-    atomicAdd(&stats[u].n_merged, n);
-    atomicAdd(&stats[u].n_groups, 1);
-    atomicMax(&stats[u].max_group, n);
+    const float gamma = L / lbar;
+    const bool ok = gamma > p.gamma_min && gamma <= p.gamma_max && fabsf(lbar) >= 1e-6f;
+    if (!ok) {
+      // guard: the members are dropped after all and the target keeps the row copied by compaction
+      for (int t = lane; t < n; t += 32) target[base + member(t)] = -1;
+      if (lane == 0) { atomicAdd(&stats[u].n_guard_groups, 1); atomicAdd(&stats[u].n_groups, 1); }
+      continue;
+    }
+    __nv_bfloat16 *dK = reinterpret_cast<__nv_bfloat16 *>(dst.K) + (base + c) * D;
+    __nv_bfloat16 *dV = reinterpret_cast<__nv_bfloat16 *>(dst.V) + (base + c) * D;
+    if constexpr (EPL == 4) {
+      uint2 ko, vo;
+      ko.x = pack_bf16(gamma * ka[0], gamma * ka[1]); ko.y = pack_bf16(gamma * ka[2], gamma * ka[3]);
+      vo.x = pack_bf16(va[0], va[1]); vo.y = pack_bf16(va[2], va[3]);
+      *reinterpret_cast<uint2 *>(dK + lane * 4) = ko;
+      *reinterpret_cast<uint2 *>(dV + lane * 4) = vo;
+    } else {
+      *reinterpret_cast<uint32_t *>(dK + lane * 2) = pack_bf16(gamma * ka[0], gamma * ka[1]);
+      *reinterpret_cast<uint32_t *>(dV + lane * 2) = pack_bf16(va[0], va[1]);
+    }
+    if (lane == 0) {
+      dst.votes[base + c] = Ps;
+      dst.lscore[base + c] = L;
+      atomicAdd(&stats[u].n_merged, n);
+      atomicAdd(&stats[u].n_groups, 1);
+      atomicMax(&stats[u].max_group, n);
+    }
   }
 }
 
@@ -454,56 +522,57 @@ template <int D>
 static void launch_compress_t(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
                               const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
                               int32_t *ret_idx, int32_t *target, keepkv_stats *stats, char *ws, const WsLayout &L,
-                              LaunchCtx &ctx) {
+                              int32_t *status_dev, LaunchCtx &ctx) {
   const int U = p.B * p.H_kv;
   UnitInfo *ui = reinterpret_cast<UnitInfo *>(ws + L.unit_info);
+  int32_t *sched = reinterpret_cast<int32_t *>(ws + L.sched);
   int32_t *ev_idx = reinterpret_cast<int32_t *>(ws + L.ev_idx);
-  float *dst_norm = reinterpret_cast<float *>(ws + L.dst_norm);
-  float *umax = reinterpret_cast<float *>(ws + L.umax);
-  int32_t *grp_ptr = reinterpret_cast<int32_t *>(ws + L.grp_ptr);
-  int32_t *grp_fill = reinterpret_cast<int32_t *>(ws + L.grp_fill);
-  int32_t *grp_mem = reinterpret_cast<int32_t *>(ws + L.grp_mem);
+  float *inv_norm = reinterpret_cast<float *>(ws + L.inv_norm);
+  float4 *nom_v = reinterpret_cast<float4 *>(ws + L.nom_v);
+  int32_t *nom_si = reinterpret_cast<int32_t *>(ws + L.nom_si);
+  uint32_t *grp_key = reinterpret_cast<uint32_t *>(ws + L.grp_key);
+  int32_t *grp_head = reinterpret_cast<int32_t *>(ws + L.grp_head);
   const int ret_bound = budget_dev ? p.N_cap : (budget_scalar < p.N_cap ? budget_scalar : p.N_cap);
 
   const size_t sel_smem = (size_t)p.N_cap * sizeof(uint32_t);
+  const int smem_keys = L.key_stride < 32768 ? L.key_stride : 32768;
   static bool attr_done_dev[64] = {};   // opt-in to large dynamic shared memory once per device
   int dev = 0;
   cudaGetDevice(&dev);
   bool &attr_done = attr_done_dev[dev & 63];
   if (!attr_done) {
     cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 49152 * 4);
-    cudaFuncSetAttribute(match_exact_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 64 * 68 * 4);
-    cudaFuncSetAttribute(match_exact_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 128 * 68 * 4);
+    cudaFuncSetAttribute(resolve_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
     attr_done = true;
   }
   select_kernel<<<U, 1024, sel_smem, ctx.stream>>>(p, src, dst.seq_len, budget_dev, budget_scalar, n_recent_dev,
                                                    ret_idx, target, ev_idx, ui, stats);
   KEEPKV_CHECK_LAUNCH(ctx);
-  if (ret_bound > 0) {
-    compact_kernel<D><<<dim3((ret_bound + 31) / 32, U), 256, 0, ctx.stream>>>(p, src, dst, ret_idx, ui, dst_norm);
-    KEEPKV_CHECK_LAUNCH(ctx);
-  }
-  match_exact_kernel<D><<<dim3(p.N_cap / 64, U), 256, 2 * D * 68 * 4, ctx.stream>>>(p, src, dst, ev_idx, ui, dst_norm,
-                                                                                    target, umax, stats);
+  if (ret_bound <= 0) return;   // nothing is kept: every entry is dropped, which select has recorded
+  compact_kernel<D><<<dim3((ret_bound + 63) / 64, U), 256, 0, ctx.stream>>>(p, src, dst, ret_idx, ui, inv_norm);
   KEEPKV_CHECK_LAUNCH(ctx);
-  if (ret_bound > 0) {
-    group_kernel<<<U, 256, 0, ctx.stream>>>(p, ev_idx, target, ui, grp_ptr, grp_fill, grp_mem);
-    KEEPKV_CHECK_LAUNCH(ctx);
-    merge_kernel<D><<<dim3((ret_bound + 3) / 4, U), 128, 0, ctx.stream>>>(p, src, dst, ret_idx, target, ui, grp_ptr,
-                                                                          grp_mem, stats);
-    KEEPKV_CHECK_LAUNCH(ctx);
-  }
+  launch_nominate(p, src, dst, ev_idx, ui, inv_norm, sched, nom_v, nom_si, L.nom_chunks, status_dev, ctx);
+  resolve_kernel<D><<<U, kResolveThreads, (size_t)smem_keys * 4, ctx.stream>>>(
+      p, src, dst, ev_idx, ui, nom_v, nom_si, sched, L.nom_chunks, target, grp_key, L.key_stride, grp_head, stats,
+      smem_keys);
+  KEEPKV_CHECK_LAUNCH(ctx);
+  int gx = 4096 / U;
+  gx = gx < 1 ? 1 : (gx > 32 ? 32 : gx);
+  merge_kernel<D><<<dim3(gx, U), 256, 0, ctx.stream>>>(p, src, dst, ret_idx, ev_idx, target, ui, grp_key,
+                                                        L.key_stride, grp_head, stats);
+  KEEPKV_CHECK_LAUNCH(ctx);
 }
 
 void launch_compress(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
                      const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev, int32_t *ret_idx,
                      int32_t *target, keepkv_stats *stats, char *ws, const WsLayout &L, int32_t *status_dev,
                      LaunchCtx &ctx) {
-  (void)status_dev;
   if (p.d == 128)
-    launch_compress_t<128>(p, src, dst, budget_dev, budget_scalar, n_recent_dev, ret_idx, target, stats, ws, L, ctx);
+    launch_compress_t<128>(p, src, dst, budget_dev, budget_scalar, n_recent_dev, ret_idx, target, stats, ws, L,
+                           status_dev, ctx);
   else
-    launch_compress_t<64>(p, src, dst, budget_dev, budget_scalar, n_recent_dev, ret_idx, target, stats, ws, L, ctx);
+    launch_compress_t<64>(p, src, dst, budget_dev, budget_scalar, n_recent_dev, ret_idx, target, stats, ws, L,
+                          status_dev, ctx);
 }
 
 }  // namespace keepkv

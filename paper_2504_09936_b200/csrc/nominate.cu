@@ -1,0 +1,386 @@
+// Similarity search of keepkv_compress (Algorithm 1 line 4: U = cosineSimilarity(K_e, K_c)) on the
+// 5th-generation tensor cores.  The cosine matrix is never stored: for every evicted key the kernel
+// keeps the three largest cosines over the retained keys (with the slots of the first two), which is
+// all the arg-max of line 5 needs.  The values found here only *rank* candidates; wherever the
+// ranking is closer than the accumulation error allows, the caller re-evaluates the candidates in
+// the fixed fp32 arithmetic the interface defines (see resolve_kernel in compress.cu).
+//
+// Work item = (unit, 128 evicted rows, one chunk of 256-column tiles of the unit's retained keys).
+// A persistent grid of one CTA per SM walks the items.  Inside a CTA:
+//   warp 0      TMA producer: retained-key tiles (256 rows x D, 128-byte swizzle) from the compacted
+//               dst cache into a 2-stage ring;
+//   warp 1      one thread issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32) into one of two
+//               256-column accumulators in tensor memory and commits to the ring / accumulator barriers;
+//   warps 2-9   gather the 128 evicted rows from the src cache into the swizzled A tile, then drain the
+//               accumulators with tcgen05.ld: two warps per 32-lane quarter, one per column half,
+//               scaling by the retained keys' inverse norms and tracking the row's top three.
+// Every wait is bounded; a wait that runs out raises KEEPKV_DEV_TIMEOUT, the CTA stops issuing work,
+// drains what is in flight, frees its tensor memory and returns.
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace keepkv {
+
+constexpr int kNomM = 128;        // evicted rows per item (tensor-memory lanes)
+constexpr int kNomN = 256;        // retained columns per tile
+constexpr int kNomStages = 2;     // B ring
+constexpr int kNomThreads = 320;  // 10 warps
+constexpr int kNomEpiThreads = 256;
+
+template <int D>
+struct NomSmem {
+  static constexpr int kSub = D / 64;                     // 64-channel (128-byte) K atoms per row
+  static constexpr int kABytes = kSub * kNomM * 128;
+  static constexpr int kBBytes = kSub * kNomN * 128;
+  static constexpr int kA = 0;
+  static constexpr int kB = kABytes;
+  static constexpr int kInv = kB + kNomStages * kBBytes;  // f32 [8 warps][128]   inverse norms of the warp's columns
+  static constexpr int kRowInv = kInv + 8 * 128 * 4;      // f32 [2][128]         inverse norms of the staged rows
+  static constexpr int kXchg = kRowInv + 2 * 128 * 4;     // u32 [2][128][5]      column-half exchange
+  static constexpr int kPrefix = kXchg + 2 * 128 * 5 * 4; // i32 [kMaxUnits + 1]  row-tile prefix over units
+  static constexpr int kBytes = kPrefix + (kMaxUnits + 1) * 4;
+};
+
+struct Top3 {
+  float best, second, third;
+  int bi, si;
+  __device__ __forceinline__ void init() { best = second = third = -CUDART_INF_F; bi = si = -1; }
+  // strict comparisons: among equal values the one inserted first (the lower slot) stays in front
+  __device__ __forceinline__ void insert(float v, int idx) {
+    if (v > second) {
+      third = second;
+      if (v > best) { second = best; si = bi; best = v; bi = idx; }
+      else { second = v; si = idx; }
+    } else {
+      third = fmaxf(third, v);
+    }
+  }
+};
+
+struct NomItem { int u, m_tile, chunk, t0, t1, n_ev, n_ret; };
+
+__device__ __forceinline__ NomItem nom_item(int item, int C, const int *prefix, int U, const UnitInfo *unit_info) {
+  NomItem it;
+  const int mg = item / C;
+  it.chunk = item % C;
+  int lo = 0, hi = U;   // largest u with prefix[u] <= mg
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (prefix[mid] <= mg) lo = mid; else hi = mid;
+  }
+  it.u = lo;
+  it.m_tile = mg - prefix[lo];
+  const UnitInfo ui = unit_info[lo];
+  it.n_ev = ui.n_ev;
+  it.n_ret = ui.n_ret;
+  const int T = (ui.n_ret + kNomN - 1) / kNomN;
+  it.t0 = (int)((long long)it.chunk * T / C);
+  it.t1 = (int)((long long)(it.chunk + 1) * T / C);
+  return it;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kNomThreads, 1)
+nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const __nv_bfloat16 *__restrict__ srcK,
+                const int32_t *__restrict__ ev_idx, const UnitInfo *__restrict__ unit_info,
+                const float *__restrict__ inv_norm, int32_t *sched, float4 *__restrict__ nom_v,
+                int32_t *__restrict__ nom_si, int C_max, int32_t *status_dev) {
+  using SL = NomSmem<D>;
+  constexpr int KSTEPS = D / 16;
+  constexpr uint32_t IDESC = umma_idesc_bf16(kNomM, kNomN);
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[10];   // a_ready, b_full[2], b_empty[2], t_full[2], t_empty[2], drain
+  __shared__ uint32_t s_tmem;
+  __shared__ volatile int s_abort;
+
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t bar_a_ready = smem_u32(&bars[0]);
+  const uint32_t bar_b_full = smem_u32(&bars[1]), bar_b_empty = smem_u32(&bars[3]);
+  const uint32_t bar_t_full = smem_u32(&bars[5]), bar_t_empty = smem_u32(&bars[7]);
+  const uint32_t bar_drain = smem_u32(&bars[9]);
+  int *prefix = reinterpret_cast<int *>(smem + SL::kPrefix);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int U = p.B * p.H_kv;
+
+  if (tid == 0) {
+    mbar_init(bar_a_ready, 8);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_b_full + 8 * i, 1);
+      mbar_init(bar_b_empty + 8 * i, 1);
+      mbar_init(bar_t_full + 8 * i, 1);
+      mbar_init(bar_t_empty + 8 * i, 8);
+    }
+    mbar_init(bar_drain, 1);
+    s_abort = 0;
+    mbar_fence_init();
+    fence_proxy_async_smem();
+    prefetch_tensormap(&mapB);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&s_tmem), 512);
+    tmem_relinquish();
+  }
+  if (warp == 2) {   // exclusive prefix of 128-row tiles over the units
+    int run = 0;
+    for (int u0 = 0; u0 < U; u0 += 32) {
+      const int u = u0 + lane;
+      const int t = u < U ? (unit_info[u].n_ev + kNomM - 1) / kNomM : 0;
+      int x = t;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= o) x += y;
+      }
+      if (u < U) prefix[u] = run + x - t;
+      run += __shfl_sync(0xffffffffu, x, 31);
+    }
+    if (lane == 0) prefix[U] = run;
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+
+  const uint32_t tmem = s_tmem;
+  const int total_m = prefix[U];
+  int C = total_m > 0 ? (2 * (int)gridDim.x + total_m - 1) / total_m : 1;
+  C = max(1, min(C, C_max));
+  const int n_items = total_m * C;
+  if (blockIdx.x == 0 && tid == 0) sched[0] = C;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int ring = 0;
+      for (int item = blockIdx.x; item < n_items && !s_abort; item += gridDim.x) {
+        const NomItem it = nom_item(item, C, prefix, U, unit_info);
+        for (int t = it.t0; t < it.t1; ++t, ++ring) {
+          const int s = ring & 1;
+          if (!mbar_wait(bar_b_empty + 8 * s, ((ring >> 1) & 1) ^ 1)) { s_abort = 1; break; }
+          mbar_expect_tx(bar_b_full + 8 * s, SL::kBBytes);
+          const uint32_t dst = sbase + SL::kB + s * SL::kBBytes;
+          const int row = it.u * p.N_cap + t * kNomN;
+#pragma unroll
+          for (int sub = 0; sub < SL::kSub; ++sub)
+            tma_load_2d(dst + sub * (kNomN * 128), &mapB, sub * 64, row, bar_b_full + 8 * s);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int ring = 0, acc = 0, n_done = 0;
+      for (int item = blockIdx.x; item < n_items && !s_abort; item += gridDim.x) {
+        const NomItem it = nom_item(item, C, prefix, U, unit_info);
+        if (it.t0 == it.t1) continue;
+        if (!mbar_wait(bar_a_ready, n_done & 1)) { s_abort = 1; break; }
+        ++n_done;
+        tc_fence_after();
+        for (int t = it.t0; t < it.t1; ++t, ++ring, ++acc) {
+          const int s = ring & 1, a = acc & 1;
+          if (!mbar_wait(bar_b_full + 8 * s, (ring >> 1) & 1) ||
+              !mbar_wait(bar_t_empty + 8 * a, ((acc >> 1) & 1) ^ 1)) { s_abort = 1; break; }
+          tc_fence_after();
+          const uint32_t a_base = sbase + SL::kA, b_base = sbase + SL::kB + s * SL::kBBytes;
+#pragma unroll
+          for (int k = 0; k < KSTEPS; ++k) {
+            const uint64_t ad = umma_desc_sw128(a_base + (k >> 2) * (kNomM * 128) + (k & 3) * 32);
+            const uint64_t bd = umma_desc_sw128(b_base + (k >> 2) * (kNomN * 128) + (k & 3) * 32);
+            umma_bf16(tmem + a * kNomN, ad, bd, IDESC, k > 0 ? 1u : 0u);
+          }
+          umma_commit(bar_b_empty + 8 * s);   // the stage may be refilled once these MMAs have read it
+          umma_commit(bar_t_full + 8 * a);    // the accumulator is complete
+        }
+      }
+      umma_commit(bar_drain);
+      mbar_wait(bar_drain, 0);   // every MMA issued above has retired (bounded)
+    }
+  } else {
+    // ------------------------------------------------------------ A staging + accumulator drain
+    const int ew = warp - 2, quarter = warp & 3, half = ew >> 2;
+    const int row = quarter * 32 + lane;                        // tensor-memory lane = row of the item
+    float *inv_w = reinterpret_cast<float *>(smem + SL::kInv) + ew * 128;
+    float *rowinv = reinterpret_cast<float *>(smem + SL::kRowInv);
+    uint32_t *xchg = reinterpret_cast<uint32_t *>(smem + SL::kXchg);
+    const size_t n_total = (size_t)U * p.N_cap;
+    int acc = 0, n_done = 0;
+    bool dead = false;
+    for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+      const NomItem it = nom_item(item, C, prefix, U, unit_info);
+      const size_t ubase = (size_t)it.u * p.N_cap;
+      const int m0 = it.m_tile * kNomM;
+      const int buf = n_done & 1;
+      Top3 top;
+      top.init();
+      if (it.t0 == it.t1) {   // a chunk without tiles (fewer tiles than chunks): publish an empty result
+        if (half == 0 && m0 + row < it.n_ev) {
+          const size_t o = (ubase + m0 + row) * C_max + it.chunk;
+          nom_v[o] = make_float4(top.best, top.second, top.third, __int_as_float(-1));
+          nom_si[o] = -1;
+        }
+        continue;
+      }
+      dead = __any_sync(0xffffffffu, dead || s_abort != 0);
+      {
+        // ---- gather the evicted rows into the swizzled A tile (the previous item's MMAs have retired:
+        //      this warp has seen the barrier of that item's last accumulator)
+#pragma unroll 2
+        for (int rep = 0; rep < kNomM / 16; ++rep) {
+          const int r = rep * 16 + ew * 2 + (lane >> 4), ch = lane & 15;
+          uint4 v = make_uint4(0, 0, 0, 0);
+          if (ch < D / 8 && m0 + r < it.n_ev) {
+            const int e = ev_idx[ubase + m0 + r];
+            v = *reinterpret_cast<const uint4 *>(srcK + (ubase + e) * D + ch * 8);
+          }
+          float ss = 0.f;
+          {
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) { const float a = bf16_lo(w[q]), b = bf16_hi(w[q]); ss = fmaf(a, a, ss); ss = fmaf(b, b, ss); }
+          }
+          ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+          ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+          ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+          ss += __shfl_xor_sync(0xffffffffu, ss, 8);
+          if (ch < D / 8)
+            *reinterpret_cast<uint4 *>(smem + SL::kA + (ch >> 3) * (kNomM * 128) + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = v;
+          if (ch == 0) rowinv[buf * 128 + r] = rsqrtf(ss);
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_a_ready);
+
+        for (int t = it.t0; t < it.t1; ++t, ++acc) {
+          const int a = acc & 1;
+          const int c0 = t * kNomN + half * 128;
+          {
+            const size_t g = ubase + c0 + 4 * lane;
+            float4 iv = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (g + 3 < n_total) iv = *reinterpret_cast<const float4 *>(inv_norm + g);
+            __syncwarp();
+            *reinterpret_cast<float4 *>(inv_w + 4 * lane) = iv;
+            __syncwarp();
+          }
+          if (!dead) {
+            const bool ok = mbar_wait(bar_t_full + 8 * a, (acc >> 1) & 1);
+            if (!__any_sync(0xffffffffu, ok)) { dead = true; s_abort = 1; }
+          }
+          if (!dead) {
+            tc_fence_after();
+            const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + a * kNomN + half * 128;
+            const int n_valid = it.n_ret - c0;   // columns of this half that exist
+#pragma unroll 1
+            for (int jg = 0; jg < 2; ++jg) {
+              uint32_t r0[32], r1[32];
+              tmem_ld_32x32(taddr + jg * 64, r0);
+              tmem_ld_32x32(taddr + jg * 64 + 32, r1);
+              tmem_ld_wait();
+              if (jg == 1) {   // everything this warp needs from the accumulator is in registers
+                tc_fence_before();
+                if (lane == 0) mbar_arrive(bar_t_empty + 8 * a);
+              }
+              const int cb = jg * 64;
+              if (n_valid >= cb + 64) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 4) {
+                  const float4 iv = *reinterpret_cast<const float4 *>(inv_w + cb + i);
+                  top.insert(__uint_as_float(r0[i]) * iv.x, c0 + cb + i);
+                  top.insert(__uint_as_float(r0[i + 1]) * iv.y, c0 + cb + i + 1);
+                  top.insert(__uint_as_float(r0[i + 2]) * iv.z, c0 + cb + i + 2);
+                  top.insert(__uint_as_float(r0[i + 3]) * iv.w, c0 + cb + i + 3);
+                }
+#pragma unroll
+                for (int i = 0; i < 32; i += 4) {
+                  const float4 iv = *reinterpret_cast<const float4 *>(inv_w + cb + 32 + i);
+                  top.insert(__uint_as_float(r1[i]) * iv.x, c0 + cb + 32 + i);
+                  top.insert(__uint_as_float(r1[i + 1]) * iv.y, c0 + cb + 32 + i + 1);
+                  top.insert(__uint_as_float(r1[i + 2]) * iv.z, c0 + cb + 32 + i + 2);
+                  top.insert(__uint_as_float(r1[i + 3]) * iv.w, c0 + cb + 32 + i + 3);
+                }
+              } else {   // ragged end of the retained set: columns past n_ret hold other rows' data
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  if (cb + i < n_valid) top.insert(__uint_as_float(r0[i]) * inv_w[cb + i], c0 + cb + i);
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                  if (cb + 32 + i < n_valid) top.insert(__uint_as_float(r1[i]) * inv_w[cb + 32 + i], c0 + cb + 32 + i);
+              }
+            }
+          }
+        }
+        ++n_done;
+      }
+      // ---- combine the two column halves of each row and publish the chunk's result
+      uint32_t *x = xchg + (size_t)(buf * 128 + row) * 5;
+      if (half == 1) {
+        x[0] = __float_as_uint(top.best); x[1] = (uint32_t)top.bi; x[2] = __float_as_uint(top.second);
+        x[3] = (uint32_t)top.si; x[4] = __float_as_uint(top.third);
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (half == 0) {
+        top.insert(__uint_as_float(x[0]), (int)x[1]);   // the upper half holds higher slots: ties keep the lower half
+        top.insert(__uint_as_float(x[2]), (int)x[3]);
+        top.third = fmaxf(top.third, __uint_as_float(x[4]));
+        if (m0 + row < it.n_ev) {
+          const float ri = rowinv[buf * 128 + row];
+          const size_t o = (ubase + m0 + row) * C_max + it.chunk;
+          nom_v[o] = make_float4(top.best * ri, top.second * ri, top.third * ri, __int_as_float(top.bi));
+          nom_si[o] = top.si;
+        }
+      }
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (s_abort) {
+    if (tid == 0) {
+      atomicOr(status_dev, KEEPKV_DEV_TIMEOUT);
+      // copies still in flight get a bounded chance to land before the shared memory goes away
+      for (int i = 0; i < 2; ++i) { mbar_wait(bar_b_full + 8 * i, 0); mbar_wait(bar_b_full + 8 * i, 1); }
+    }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+template <int D>
+static void launch_nominate_t(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
+                              const int32_t *ev_idx, const UnitInfo *unit_info, const float *inv_norm, int32_t *sched,
+                              float4 *nom_v, int32_t *nom_si, int nom_chunks, int32_t *status_dev, LaunchCtx &ctx) {
+  using SL = NomSmem<D>;
+  constexpr size_t smem_bytes = (size_t)SL::kBytes + 1024;
+  static bool attr_done_dev[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (!attr_done_dev[dev & 63]) {
+    cudaFuncSetAttribute(nominate_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+    attr_done_dev[dev & 63] = true;
+  }
+  CUtensorMap mapB;
+  if (!make_bf16_rows_map(&mapB, dst.K, (uint64_t)p.B * p.H_kv * p.N_cap, D, kNomN)) {
+    if (ctx.err == cudaSuccess) ctx.err = cudaErrorInvalidValue;
+    return;
+  }
+  nominate_kernel<D><<<sm_count(), kNomThreads, smem_bytes, ctx.stream>>>(
+      mapB, p, reinterpret_cast<const __nv_bfloat16 *>(src.K), ev_idx, unit_info, inv_norm, sched, nom_v, nom_si,
+      nom_chunks, status_dev);
+  KEEPKV_CHECK_LAUNCH(ctx);
+}
+
+void launch_nominate(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst, const int32_t *ev_idx,
+                     const UnitInfo *unit_info, const float *inv_norm, int32_t *sched, float4 *nom_v, int32_t *nom_si,
+                     int nom_chunks, int32_t *status_dev, LaunchCtx &ctx) {
+  if (p.d == 128)
+    launch_nominate_t<128>(p, src, dst, ev_idx, unit_info, inv_norm, sched, nom_v, nom_si, nom_chunks, status_dev, ctx);
+  else
+    launch_nominate_t<64>(p, src, dst, ev_idx, unit_info, inv_norm, sched, nom_v, nom_si, nom_chunks, status_dev, ctx);
+}
+
+}  // namespace keepkv
