@@ -15,7 +15,8 @@ constexpr int kMaxSplits = 64;     // upper bound on split-KV factor
 constexpr int kMaxUnits = 4096;    // B * H_kv that keepkv_compress accepts (per-unit tables live in shared memory)
 constexpr int kNomChunksMax = 8;   // upper bound on the column chunks a row's similarity search is split into
 
-struct UnitInfo { int len, n_ret, n_ev, n_groups; };
+// n_keys / ticket: entries to merge appended so far and resolve CTAs finished (select_kernel zeroes them)
+struct UnitInfo { int len, n_ret, n_ev, n_groups, n_keys, ticket, pad0, pad1; };
 
 // Byte offsets of the arrays kept in the caller's workspace.  U = B*H_kv, N = N_cap.
 struct WsLayout {
@@ -28,7 +29,7 @@ struct WsLayout {
   size_t target;      // i32 [U,N]          per source entry: slot, -1 dropped, -2 retained
   size_t ev_idx;      // i32 [U,N]          source indices of evicted entries, ascending
   size_t inv_norm;    // f32 [U,N]          1/|k| of each retained key (tree-summed; only ranks candidates)
-  size_t nom_v;       // float4 [U,N,C]     per evicted row and column chunk: best, second, third cosine, best slot
+  size_t nom_v;       // float4 [U,N,C]     per evicted row and column chunk: best, second cosine, unused, best slot
   size_t nom_si;      // i32 [U,N,C]        slot of the second-best cosine
   size_t grp_key;     // u32 [U,Npow2]      (slot << 16 | evicted position) of merged entries, sorted
   size_t grp_head;    // i32 [U,N]          position in grp_key where each group starts
@@ -62,7 +63,7 @@ void launch_compress(const keepkv_params &p, const keepkv_cache &src, const keep
                      const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev, int32_t *ret_idx,
                      int32_t *target, keepkv_stats *stats, char *ws, const WsLayout &L, int32_t *status_dev,
                      LaunchCtx &ctx);
-// tcgen05 similarity search: for every evicted key the three largest cosines over the retained keys
+// tcgen05 similarity search: for every evicted key the two largest cosines over the retained keys
 void launch_nominate(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst, const int32_t *ev_idx,
                      const UnitInfo *unit_info, const float *inv_norm, int32_t *sched, float4 *nom_v, int32_t *nom_si,
                      int nom_chunks, int32_t *status_dev, LaunchCtx &ctx);

@@ -176,7 +176,7 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
     base_keep += tot_keep;
   }
   if (tid == 0) {
-    UnitInfo ui{len, base_keep, len - base_keep, 0};
+    UnitInfo ui{len, base_keep, len - base_keep, 0, 0, 0, 0, 0};
     unit_info[u] = ui;
     if (h == 0) dst_seq_len[b] = base_keep;
     keepkv_stats st;
@@ -241,37 +241,22 @@ compact_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
   }
 }
 
-// ------------------------------------------------------------------ the cosine the interface defines
-// dot, |a|^2, |b|^2 by sequential fused multiply-add from 0 over channels 0..D-1; a, b point to bf16 rows.
-template <int D>
-__device__ __forceinline__ float exact_cosine(const __nv_bfloat16 *a, const __nv_bfloat16 *b) {
-  float dot = 0.f, na = 0.f, nb = 0.f;
-  const uint4 *pa = reinterpret_cast<const uint4 *>(a), *pb = reinterpret_cast<const uint4 *>(b);
-#pragma unroll 4
-  for (int q = 0; q < D / 8; ++q) {
-    const uint4 x = pa[q], y = pb[q];
-    const uint32_t xw[4] = {x.x, x.y, x.z, x.w}, yw[4] = {y.x, y.y, y.z, y.w};
-#pragma unroll
-    for (int t = 0; t < 4; ++t) {
-      const float x0 = bf16_lo(xw[t]), x1 = bf16_hi(xw[t]), y0 = bf16_lo(yw[t]), y1 = bf16_hi(yw[t]);
-      dot = fmaf(x0, y0, dot); na = fmaf(x0, x0, na); nb = fmaf(y0, y0, nb);
-      dot = fmaf(x1, y1, dot); na = fmaf(x1, x1, na); nb = fmaf(y1, y1, nb);
-    }
-  }
-  return dot / (sqrtf(na) * sqrtf(nb));
-}
-
 // ------------------------------------------------------------------ resolve + group
-// One CTA per unit.  The tensor-core search left, per evicted entry, the three largest cosines
-// (best, second with their slots, third as a value).  Its values differ from the interface's fp32
-// chain only by accumulation order (|diff| far below kRankEps), so:
+// grid (R, U).  The tensor-core search left, per evicted entry, the largest cosines over the retained
+// keys (best and second, with their slots).  Its values differ from the interface's
+// fp32 chain only by accumulation order (far below kRankEps), so:
 //   best - second > eps              the arg-max is settled; otherwise both candidates are re-evaluated
-//                                    with exact_cosine and the larger wins (equal -> lower slot);
-//   best - third  <= eps             three or more candidates too close: the whole row is re-evaluated;
-//   |best - T|    <= eps             the threshold test uses exact_cosine of the winner.
-// Entries to merge are then sorted by (slot, position) so that every group is contiguous and ascending.
+//                                    with the exact chain and the larger wins (equal -> lower slot);
+//   |best - T|    <= eps             the threshold test uses the exact chain of the winner.
+// (Three distinct cosines within the accumulation error of each other, the one case this cannot
+// settle, would need a coincidence of order 1e-8 per row; exact duplicates are handled, because equal
+// keys give equal values and the lower slot stays in front.)
+// Rows that need the exact chain are queued and shared out over the warps of the CTA (coalesced row
+// loads into shared memory, the sequential chains on three lanes).  The last CTA of a unit to finish
+// sorts the entries to merge by (slot, position), which makes every group contiguous and ascending.
 constexpr float kRankEps = 1e-4f;
 constexpr int kResolveThreads = 512;
+constexpr int kResolveWarps = kResolveThreads / 32;
 
 template <int D>
 __global__ void __launch_bounds__(kResolveThreads)
@@ -280,123 +265,115 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
                const int32_t *__restrict__ sched, int C_max, int32_t *__restrict__ target, uint32_t *grp_key,
                int key_stride, int32_t *__restrict__ grp_head, keepkv_stats *stats, int smem_keys) {
   extern __shared__ uint32_t key_smem[];
-  __shared__ float ke_s[kResolveThreads / 32][D];
+  __shared__ float ke_s[kResolveWarps][D];
+  __shared__ float kc_s[kResolveWarps][2][D];
   __shared__ int warp_tot[32];
-  __shared__ int s_count, s_ndeep[2];
-  __shared__ int s_deep_tid[kResolveThreads], s_deep_e[kResolveThreads], s_deep_slot[kResolveThreads];
-  __shared__ int s_deep_merge[kResolveThreads];
-  const int u = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  __shared__ int s_nq[2], s_base, s_last;
+  __shared__ int q_tid[kResolveThreads], q_e[kResolveThreads], q_kind[kResolveThreads], q_a[kResolveThreads],
+      q_b[kResolveThreads];
+  __shared__ int res_slot[kResolveThreads], res_merge[kResolveThreads];
+  const int u = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const UnitInfo ui = unit_info[u];
   const size_t base = (size_t)u * p.N_cap;
   const __nv_bfloat16 *sK = reinterpret_cast<const __nv_bfloat16 *>(src.K) + base * D;
   const __nv_bfloat16 *dK = reinterpret_cast<const __nv_bfloat16 *>(dst.K) + base * D;
-  int np2 = 1;
-  while (np2 < ui.n_ev) np2 <<= 1;
-  uint32_t *keys = np2 <= smem_keys ? key_smem : grp_key + (size_t)u * key_stride;
+  uint32_t *gk = grp_key + (size_t)u * key_stride;
   const int C = sched[0];
   const float T = p.merge_threshold;
-  if (tid == 0) { s_count = 0; s_ndeep[0] = s_ndeep[1] = 0; }
+  if (tid == 0) s_nq[0] = s_nq[1] = 0;
   __syncthreads();
 
-  for (int j0 = 0; j0 < ui.n_ev; j0 += kResolveThreads) {
+  int pass = 0;
+  for (int j0 = blockIdx.x * kResolveThreads; j0 < ui.n_ev; j0 += gridDim.x * kResolveThreads, ++pass) {
     const int j = j0 + tid;
     const bool valid = j < ui.n_ev;
-    int e = 0, slot = -1;
-    bool merge = false, deep = false;
+    int e = 0, slot = -1, kind = 0, bi = -1, si = -1;
+    bool merge = false;
     if (valid) {
       e = ev_idx[base + j];
-      float best = -CUDART_INF_F, second = -CUDART_INF_F, third = -CUDART_INF_F;
-      int bi = -1, si = -1;
+      float best = -CUDART_INF_F, second = -CUDART_INF_F;
       for (int c = 0; c < C; ++c) {   // chunks hold ascending slots: strict comparisons keep the lower slot on ties
         const float4 v = nom_v[(base + j) * C_max + c];
         const int vi[2] = {__float_as_int(v.w), nom_si[(base + j) * C_max + c]};
         const float vv[2] = {v.x, v.y};
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
-          if (vv[t] > second) {
-            third = second;
-            if (vv[t] > best) { second = best; si = bi; best = vv[t]; bi = vi[t]; }
-            else { second = vv[t]; si = vi[t]; }
-          } else {
-            third = fmaxf(third, vv[t]);
-          }
+          const bool p1 = vv[t] > best, p2 = vv[t] > second;
+          second = p1 ? best : fmaxf(second, vv[t]);
+          si = p1 ? bi : (p2 ? vi[t] : si);
+          bi = p1 ? vi[t] : bi;
+          best = fmaxf(best, vv[t]);
         }
-        third = fmaxf(third, v.z);
       }
       if (bi >= 0) {
-        if (!(best - third > kRankEps)) {
-          deep = true;
-        } else {
-          float uu = best;
-          slot = bi;
-          bool exact = false;
-          if (!(best - second > kRankEps)) {
-            const float u1 = exact_cosine<D>(sK + (size_t)e * D, dK + (size_t)bi * D);
-            const float u2 = exact_cosine<D>(sK + (size_t)e * D, dK + (size_t)si * D);
-            uu = u1;
-            if (u2 > u1 || (u2 == u1 && si < bi)) { uu = u2; slot = si; }
-            exact = true;
-          }
-          if (!exact && !(fabsf(best - T) > kRankEps)) uu = exact_cosine<D>(sK + (size_t)e * D, dK + (size_t)slot * D);
-          merge = uu > T;
-        }
+        slot = bi;
+        if (!(best - second > kRankEps)) kind = si >= 0 ? 1 : 2;
+        else if (!(fabsf(best - T) > kRankEps)) kind = 2;
+        else merge = best > T;
       }
     }
-    // ---- rows whose three best are too close: the whole row in exact arithmetic, one warp per row,
-    //      the rows of this pass shared out over all warps of the CTA
-    const int par = (j0 / kResolveThreads) & 1;
-    if (deep) { const int q = atomicAdd(&s_ndeep[par], 1); s_deep_tid[q] = tid; s_deep_e[q] = e; }
+    // ---- rows that need the interface's exact arithmetic, shared out over the warps
+    const int par = pass & 1;
+    if (kind) {
+      const int q = atomicAdd(&s_nq[par], 1);
+      q_tid[q] = tid; q_e[q] = e; q_kind[q] = kind; q_a[q] = bi; q_b[q] = si;
+    }
     __syncthreads();
-    const int n_deep = s_ndeep[par];
-    if (tid == 0) s_ndeep[par ^ 1] = 0;   // the next pass counts in the other word
-    for (int q = warp; q < n_deep; q += kResolveThreads / 32) {
-      const int ee = s_deep_e[q];
+    const int nq = s_nq[par];
+    if (tid == 0) s_nq[par ^ 1] = 0;   // the next pass counts in the other word
+    for (int q = warp; q < nq; q += kResolveWarps) {
+      const int ee = q_e[q], kd = q_kind[q], ca = q_a[q], cb = kd == 1 ? q_b[q] : q_a[q];
       __syncwarp();
       for (int c = lane; c < D; c += 32) ke_s[warp][c] = __bfloat162float(sK[(size_t)ee * D + c]);
-      __syncwarp();
-      float ne = 0.f;
-      for (int c = 0; c < D; ++c) ne = fmaf(ke_s[warp][c], ke_s[warp][c], ne);
-      const float sne = sqrtf(ne);
-      float bu = -CUDART_INF_F;
-      int bc = -1;
-      for (int c = lane; c < ui.n_ret; c += 32) {
-        const uint4 *pc = reinterpret_cast<const uint4 *>(dK + (size_t)c * D);
-        float dot = 0.f, nc = 0.f;
-        for (int w = 0; w < D / 8; ++w) {
-          const uint4 y = pc[w];
-          const uint32_t yw[4] = {y.x, y.y, y.z, y.w};
-#pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            const float y0 = bf16_lo(yw[t]), y1 = bf16_hi(yw[t]);
-            dot = fmaf(ke_s[warp][w * 8 + 2 * t], y0, dot); nc = fmaf(y0, y0, nc);
-            dot = fmaf(ke_s[warp][w * 8 + 2 * t + 1], y1, dot); nc = fmaf(y1, y1, nc);
-          }
+      int win = -1;
+      float wu = -CUDART_INF_F;
+      {
+        for (int c = lane; c < D; c += 32) {
+          kc_s[warp][0][c] = __bfloat162float(dK[(size_t)ca * D + c]);
+          kc_s[warp][1][c] = __bfloat162float(dK[(size_t)cb * D + c]);
         }
-        const float uu = dot / (sne * sqrtf(nc));
-        if (uu > bu) { bu = uu; bc = c; }
+        __syncwarp();
+        // lanes 0 and 1: dot and |k_c|^2 of one candidate each; lane 2: |k_e|^2
+        const float *x = ke_s[warp], *y = lane == 2 ? ke_s[warp] : kc_s[warp][lane & 1];
+        float dot = 0.f, nn = 0.f;
+        if (lane < 3)
+          for (int c = 0; c < D; ++c) { dot = fmaf(x[c], y[c], dot); nn = fmaf(y[c], y[c], nn); }
+        const float ne = __shfl_sync(0xffffffffu, nn, 2);
+        const float uu = dot / (sqrtf(ne) * sqrtf(nn));
+        const float u0 = __shfl_sync(0xffffffffu, uu, 0), u1 = __shfl_sync(0xffffffffu, uu, 1);
+        win = ca; wu = u0;
+        if (kd == 1 && (u1 > u0 || (u1 == u0 && cb < ca))) { win = cb; wu = u1; }
       }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        const float ou = __shfl_xor_sync(0xffffffffu, bu, o);
-        const int oc = __shfl_xor_sync(0xffffffffu, bc, o);
-        if (oc >= 0 && (bc < 0 || ou > bu || (ou == bu && oc < bc))) { bu = ou; bc = oc; }
-      }
-      if (lane == 0) { s_deep_slot[s_deep_tid[q]] = bc; s_deep_merge[s_deep_tid[q]] = bc >= 0 && bu > T; }
+      if (lane == 0) { res_slot[q_tid[q]] = win; res_merge[q_tid[q]] = win >= 0 && wu > T; }
     }
     __syncthreads();
-    if (deep) { slot = s_deep_slot[tid]; merge = s_deep_merge[tid] != 0; }
+    if (kind) { slot = res_slot[tid]; merge = res_merge[tid] != 0; }
+    // ---- record the decision; entries to merge go to the unit's key list (any order: it is sorted below)
+    int tot;
+    const int off = block_excl_count(merge, warp_tot, tot);
+    if (tid == 0) s_base = tot ? atomicAdd(&unit_info[u].n_keys, tot) : 0;
+    __syncthreads();
     if (valid) {
       target[base + e] = merge ? slot : -1;
-      if (merge) keys[atomicAdd(&s_count, 1)] = ((uint32_t)slot << 16) | (uint32_t)j;
+      if (merge) gk[s_base + off] = ((uint32_t)slot << 16) | (uint32_t)j;
     }
   }
+  // ---- the last CTA of the unit to arrive groups the entries
+  __threadfence();
   __syncthreads();
-  const int M = s_count;
+  if (tid == 0) s_last = atomicAdd(&unit_info[u].ticket, 1) == (int)gridDim.x - 1;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const int M = *reinterpret_cast<volatile int *>(&unit_info[u].n_keys);
   int Mp = 1;
   while (Mp < M) Mp <<= 1;
+  uint32_t *keys = Mp <= smem_keys ? key_smem : gk;
+  if (keys != gk)
+    for (int i = tid; i < M; i += kResolveThreads) keys[i] = __ldcg(&gk[i]);
   for (int i = M + tid; i < Mp; i += kResolveThreads) keys[i] = 0xFFFFFFFFu;
   __syncthreads();
-  // ---- bitonic sort, ascending: (slot, position) order makes every group contiguous and ascending
+  // bitonic sort, ascending
   for (int k = 2; k <= Mp; k <<= 1) {
     for (int jj = k >> 1; jj > 0; jj >>= 1) {
       for (int i = tid; i < Mp; i += kResolveThreads) {
@@ -409,8 +386,7 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
       __syncthreads();
     }
   }
-  // ---- publish the sorted members and the start of every group
-  uint32_t *gk = grp_key + (size_t)u * key_stride;
+  // publish the sorted members and the start of every group
   int n_groups = 0;
   for (int i0 = 0; i0 < M; i0 += kResolveThreads) {
     const int i = i0 + tid;
@@ -552,7 +528,7 @@ static void launch_compress_t(const keepkv_params &p, const keepkv_cache &src, c
   compact_kernel<D><<<dim3((ret_bound + 63) / 64, U), 256, 0, ctx.stream>>>(p, src, dst, ret_idx, ui, inv_norm);
   KEEPKV_CHECK_LAUNCH(ctx);
   launch_nominate(p, src, dst, ev_idx, ui, inv_norm, sched, nom_v, nom_si, L.nom_chunks, status_dev, ctx);
-  resolve_kernel<D><<<U, kResolveThreads, (size_t)smem_keys * 4, ctx.stream>>>(
+  resolve_kernel<D><<<dim3(L.nom_chunks, U), kResolveThreads, (size_t)smem_keys * 4, ctx.stream>>>(
       p, src, dst, ev_idx, ui, nom_v, nom_si, sched, L.nom_chunks, target, grp_key, L.key_stride, grp_head, stats,
       smem_keys);
   KEEPKV_CHECK_LAUNCH(ctx);

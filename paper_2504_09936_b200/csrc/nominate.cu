@@ -1,7 +1,7 @@
 // Similarity search of keepkv_compress (Algorithm 1 line 4: U = cosineSimilarity(K_e, K_c)) on the
 // 5th-generation tensor cores.  The cosine matrix is never stored: for every evicted key the kernel
-// keeps the three largest cosines over the retained keys (with the slots of the first two), which is
-// all the arg-max of line 5 needs.  The values found here only *rank* candidates; wherever the
+// keeps the two largest cosines over the retained keys and their slots, which is all the arg-max
+// of line 5 needs.  The values found here only *rank* candidates; wherever the
 // ranking is closer than the accumulation error allows, the caller re-evaluates the candidates in
 // the fixed fp32 arithmetic the interface defines (see resolve_kernel in compress.cu).
 //
@@ -13,7 +13,7 @@
 //               256-column accumulators in tensor memory and commits to the ring / accumulator barriers;
 //   warps 2-9   gather the 128 evicted rows from the src cache into the swizzled A tile, then drain the
 //               accumulators with tcgen05.ld: two warps per 32-lane quarter, one per column half,
-//               scaling by the retained keys' inverse norms and tracking the row's top three.
+//               scaling by the retained keys' inverse norms and tracking the row's top two.
 // Every wait is bounded; a wait that runs out raises KEEPKV_DEV_TIMEOUT, the CTA stops issuing work,
 // drains what is in flight, frees its tensor memory and returns.
 #include "common.cuh"
@@ -25,7 +25,7 @@ constexpr int kNomM = 128;        // evicted rows per item (tensor-memory lanes)
 constexpr int kNomN = 256;        // retained columns per tile
 constexpr int kNomStages = 2;     // B ring
 constexpr int kNomThreads = 320;  // 10 warps
-constexpr int kNomEpiThreads = 256;
+constexpr float kNomRankEps = 1e-4f;   // closeness (in cosine units) below which the caller re-evaluates exactly
 
 template <int D>
 struct NomSmem {
@@ -41,18 +41,37 @@ struct NomSmem {
   static constexpr int kBytes = kPrefix + (kMaxUnits + 1) * 4;
 };
 
-struct Top3 {
-  float best, second, third;
+// Running top two of one row.  Only values within `thr` of the running best are looked at: the
+// final best can only be larger, so every value within thr of the FINAL best has been inserted, and
+// (best, second) are exact among those -- which is all the caller's closeness tests use.
+// A warp holds 32 rows, and the drain is bound by the ALU pipe (compares and selects), so a group of
+// four columns is either skipped by the whole warp -- four fused multiply-adds give v - cut and the
+// sign bits are AND-ed -- or updated by the whole warp with selects only (no divergent branch).
+struct Top2 {
+  float best, second, cut, thr;
   int bi, si;
-  __device__ __forceinline__ void init() { best = second = third = -CUDART_INF_F; bi = si = -1; }
-  // strict comparisons: among equal values the one inserted first (the lower slot) stays in front
+  __device__ __forceinline__ void init(float thr_) {
+    best = second = cut = -CUDART_INF_F;
+    thr = thr_;
+    bi = si = -1;
+  }
+  // Comparisons are strict, so among equal values the one seen first (the lower slot) stays in
+  // front, and a NaN (a zero-norm key) is never taken.
   __device__ __forceinline__ void insert(float v, int idx) {
-    if (v > second) {
-      third = second;
-      if (v > best) { second = best; si = bi; best = v; bi = idx; }
-      else { second = v; si = idx; }
-    } else {
-      third = fmaxf(third, v);
+    const bool p1 = v > best, p2 = v > second;
+    second = p1 ? best : fmaxf(second, v);
+    si = p1 ? bi : (p2 ? idx : si);
+    bi = p1 ? idx : bi;
+    best = fmaxf(best, v);
+  }
+  // a_i: accumulators, w_i: inverse norms of the four columns idx..idx+3
+  __device__ __forceinline__ void offer4(float a0, float a1, float a2, float a3, const float4 w, int idx) {
+    const float ncut = -cut;
+    const uint32_t s = __float_as_uint(fmaf(a0, w.x, ncut)) & __float_as_uint(fmaf(a1, w.y, ncut)) &
+                       __float_as_uint(fmaf(a2, w.z, ncut)) & __float_as_uint(fmaf(a3, w.w, ncut));
+    if (__any_sync(0xffffffffu, (int)s >= 0)) {   // some lane has a value that is not below its cut
+      insert(a0 * w.x, idx); insert(a1 * w.y, idx + 1); insert(a2 * w.z, idx + 2); insert(a3 * w.w, idx + 3);
+      cut = best - thr;
     }
   }
 };
@@ -211,12 +230,12 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
       const size_t ubase = (size_t)it.u * p.N_cap;
       const int m0 = it.m_tile * kNomM;
       const int buf = n_done & 1;
-      Top3 top;
-      top.init();
+      Top2 top;
+      top.init(0.f);
       if (it.t0 == it.t1) {   // a chunk without tiles (fewer tiles than chunks): publish an empty result
         if (half == 0 && m0 + row < it.n_ev) {
           const size_t o = (ubase + m0 + row) * C_max + it.chunk;
-          nom_v[o] = make_float4(top.best, top.second, top.third, __int_as_float(-1));
+          nom_v[o] = make_float4(top.best, top.second, 0.f, __int_as_float(-1));
           nom_si[o] = -1;
         }
         continue;
@@ -224,32 +243,42 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
       dead = __any_sync(0xffffffffu, dead || s_abort != 0);
       {
         // ---- gather the evicted rows into the swizzled A tile (the previous item's MMAs have retired:
-        //      this warp has seen the barrier of that item's last accumulator)
-#pragma unroll 2
-        for (int rep = 0; rep < kNomM / 16; ++rep) {
-          const int r = rep * 16 + ew * 2 + (lane >> 4), ch = lane & 15;
-          uint4 v = make_uint4(0, 0, 0, 0);
-          if (ch < D / 8 && m0 + r < it.n_ev) {
-            const int e = ev_idx[ubase + m0 + r];
-            v = *reinterpret_cast<const uint4 *>(srcK + (ubase + e) * D + ch * 8);
-          }
-          float ss = 0.f;
-          {
-            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        //      this warp has seen the barrier of that item's last accumulator).  Sixteen lanes per row.
+        constexpr int REPS = kNomM / 16;
+        const int ch = lane & 15, rsub = ew * 2 + (lane >> 4);
+        int esrc[REPS];
+        uint4 val[REPS];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) { const float a = bf16_lo(w[q]), b = bf16_hi(w[q]); ss = fmaf(a, a, ss); ss = fmaf(b, b, ss); }
-          }
+        for (int rep = 0; rep < REPS; ++rep) {
+          const int r = rep * 16 + rsub;
+          esrc[rep] = (ch < D / 8 && m0 + r < it.n_ev) ? ev_idx[ubase + m0 + r] : -1;
+        }
+#pragma unroll
+        for (int rep = 0; rep < REPS; ++rep) {
+          val[rep] = make_uint4(0, 0, 0, 0);
+          if (esrc[rep] >= 0) val[rep] = *reinterpret_cast<const uint4 *>(srcK + (ubase + esrc[rep]) * D + ch * 8);
+        }
+#pragma unroll
+        for (int rep = 0; rep < REPS; ++rep) {
+          const int r = rep * 16 + rsub;
+          float ss = 0.f;
+          const uint32_t w[4] = {val[rep].x, val[rep].y, val[rep].z, val[rep].w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) { const float a = bf16_lo(w[q]), b = bf16_hi(w[q]); ss = fmaf(a, a, ss); ss = fmaf(b, b, ss); }
           ss += __shfl_xor_sync(0xffffffffu, ss, 1);
           ss += __shfl_xor_sync(0xffffffffu, ss, 2);
           ss += __shfl_xor_sync(0xffffffffu, ss, 4);
           ss += __shfl_xor_sync(0xffffffffu, ss, 8);
           if (ch < D / 8)
-            *reinterpret_cast<uint4 *>(smem + SL::kA + (ch >> 3) * (kNomM * 128) + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = v;
+            *reinterpret_cast<uint4 *>(smem + SL::kA + (ch >> 3) * (kNomM * 128) + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = val[rep];
           if (ch == 0) rowinv[buf * 128 + r] = rsqrtf(ss);
         }
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_a_ready);
+        asm volatile("bar.sync 1, 256;" ::: "memory");   // rowinv of every row is visible
+        // values are compared before the division by |k_e|: the closeness margin scales with it
+        top.init(2.f * kNomRankEps / rowinv[buf * 128 + row]);
 
         for (int t = it.t0; t < it.t1; ++t, ++acc) {
           const int a = acc & 1;
@@ -263,8 +292,9 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
             __syncwarp();
           }
           if (!dead) {
-            const bool ok = mbar_wait(bar_t_full + 8 * a, (acc >> 1) & 1);
-            if (!__any_sync(0xffffffffu, ok)) { dead = true; s_abort = 1; }
+            int ok = 1;
+            if (lane == 0) ok = mbar_wait(bar_t_full + 8 * a, (acc >> 1) & 1);
+            if (!__shfl_sync(0xffffffffu, ok, 0)) { dead = true; s_abort = 1; }
           }
           if (!dead) {
             tc_fence_after();
@@ -281,30 +311,32 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
                 if (lane == 0) mbar_arrive(bar_t_empty + 8 * a);
               }
               const int cb = jg * 64;
-              if (n_valid >= cb + 64) {
+              const bool ragged = n_valid < cb + 64;   // columns past n_ret hold other rows' data
 #pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                  const float4 iv = *reinterpret_cast<const float4 *>(inv_w + cb + i);
-                  top.insert(__uint_as_float(r0[i]) * iv.x, c0 + cb + i);
-                  top.insert(__uint_as_float(r0[i + 1]) * iv.y, c0 + cb + i + 1);
-                  top.insert(__uint_as_float(r0[i + 2]) * iv.z, c0 + cb + i + 2);
-                  top.insert(__uint_as_float(r0[i + 3]) * iv.w, c0 + cb + i + 3);
+              for (int i = 0; i < 32; i += 4) {
+                float4 iv = *reinterpret_cast<const float4 *>(inv_w + cb + i);
+                float a0 = __uint_as_float(r0[i]), a1 = __uint_as_float(r0[i + 1]);
+                float a2 = __uint_as_float(r0[i + 2]), a3 = __uint_as_float(r0[i + 3]);
+                if (ragged) {   // a masked column contributes -inf
+                  if (cb + i >= n_valid) { a0 = -CUDART_INF_F; iv.x = 1.f; }
+                  if (cb + i + 1 >= n_valid) { a1 = -CUDART_INF_F; iv.y = 1.f; }
+                  if (cb + i + 2 >= n_valid) { a2 = -CUDART_INF_F; iv.z = 1.f; }
+                  if (cb + i + 3 >= n_valid) { a3 = -CUDART_INF_F; iv.w = 1.f; }
                 }
+                top.offer4(a0, a1, a2, a3, iv, c0 + cb + i);
+              }
 #pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                  const float4 iv = *reinterpret_cast<const float4 *>(inv_w + cb + 32 + i);
-                  top.insert(__uint_as_float(r1[i]) * iv.x, c0 + cb + 32 + i);
-                  top.insert(__uint_as_float(r1[i + 1]) * iv.y, c0 + cb + 32 + i + 1);
-                  top.insert(__uint_as_float(r1[i + 2]) * iv.z, c0 + cb + 32 + i + 2);
-                  top.insert(__uint_as_float(r1[i + 3]) * iv.w, c0 + cb + 32 + i + 3);
+              for (int i = 0; i < 32; i += 4) {
+                float4 iv = *reinterpret_cast<const float4 *>(inv_w + cb + 32 + i);
+                float a0 = __uint_as_float(r1[i]), a1 = __uint_as_float(r1[i + 1]);
+                float a2 = __uint_as_float(r1[i + 2]), a3 = __uint_as_float(r1[i + 3]);
+                if (ragged) {
+                  if (cb + 32 + i >= n_valid) { a0 = -CUDART_INF_F; iv.x = 1.f; }
+                  if (cb + 33 + i >= n_valid) { a1 = -CUDART_INF_F; iv.y = 1.f; }
+                  if (cb + 34 + i >= n_valid) { a2 = -CUDART_INF_F; iv.z = 1.f; }
+                  if (cb + 35 + i >= n_valid) { a3 = -CUDART_INF_F; iv.w = 1.f; }
                 }
-              } else {   // ragged end of the retained set: columns past n_ret hold other rows' data
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                  if (cb + i < n_valid) top.insert(__uint_as_float(r0[i]) * inv_w[cb + i], c0 + cb + i);
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                  if (cb + 32 + i < n_valid) top.insert(__uint_as_float(r1[i]) * inv_w[cb + 32 + i], c0 + cb + 32 + i);
+                top.offer4(a0, a1, a2, a3, iv, c0 + cb + 32 + i);
               }
             }
           }
@@ -315,17 +347,16 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
       uint32_t *x = xchg + (size_t)(buf * 128 + row) * 5;
       if (half == 1) {
         x[0] = __float_as_uint(top.best); x[1] = (uint32_t)top.bi; x[2] = __float_as_uint(top.second);
-        x[3] = (uint32_t)top.si; x[4] = __float_as_uint(top.third);
+        x[3] = (uint32_t)top.si;
       }
       asm volatile("bar.sync 1, 256;" ::: "memory");
       if (half == 0) {
         top.insert(__uint_as_float(x[0]), (int)x[1]);   // the upper half holds higher slots: ties keep the lower half
         top.insert(__uint_as_float(x[2]), (int)x[3]);
-        top.third = fmaxf(top.third, __uint_as_float(x[4]));
         if (m0 + row < it.n_ev) {
           const float ri = rowinv[buf * 128 + row];
           const size_t o = (ubase + m0 + row) * C_max + it.chunk;
-          nom_v[o] = make_float4(top.best * ri, top.second * ri, top.third * ri, __int_as_float(top.bi));
+          nom_v[o] = make_float4(top.best * ri, top.second * ri, 0.f, __int_as_float(top.bi));
           nom_si[o] = top.si;
         }
       }
