@@ -158,9 +158,9 @@ int keepkv_decode_step_host(const keepkv_params *p, const keepkv_cache *cache, c
  * of KEEPKV_STATIC_SCRATCH_BYTES inside the library image; every GPU that loads the library holds
  * it until the process exits.  The call allocates and frees nothing.
  *  - Arguments as keepkv_decode_attention, without ws / ws_bytes; inputs and outputs stay the caller's.
- *  - Shapes whose decode scratch (4*U + 4*U*S*G*(d+2) bytes rounded up to 256-byte pieces, U = B*H_kv,
- *    S the split factor the library picks for the shape) exceeds the array are refused with
- *    KEEPKV_ERR_WORKSPACE before anything is enqueued; the five benchmark shapes need 0.3-4.3 MB.
+ *  - Shapes whose decode scratch (4 bytes per unit, U = B*H_kv, plus a pool of 1024 partial results of
+ *    (16 + G*d) floats, each rounded up to 256-byte pieces) exceeds the array are refused with
+ *    KEEPKV_ERR_WORKSPACE before anything is enqueued; G = 8, d = 128 leaves room for 900 000 units.
  *  - The first call on each device looks up the array's device address; make that call outside any
  *    stream capture, with the device current that `stream` belongs to.
  *  - All calls on one GPU share the array and find in it whatever the previous call left: the call

@@ -14,18 +14,10 @@ static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 WsLayout ws_layout(const keepkv_params &p) {
   WsLayout L;
   const size_t U = (size_t)p.B * p.H_kv, N = (size_t)p.N_cap, G = (size_t)(p.H_q / p.H_kv);
-  // Enough splits to put at least four waves of CTAs on 148 SMs, never more than the tiles of a unit.
-  size_t tiles = (N + kTile - 1) / kTile;
-  size_t want = (4 * 148 + U - 1) / U;
-  size_t S = want < 1 ? 1 : want;
-  if (S > tiles) S = tiles;
-  if (S > (size_t)kMaxSplits) S = kMaxSplits;
-  L.max_splits = (int)S;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   L.counters = take(U * 4);
-  L.part_ml = take(U * S * G * 2 * 4);
-  L.part_acc = take(U * S * G * (size_t)p.d * 4);
+  L.part_pool = take((size_t)kDecMaxCtas * 2 * (16 + G * (size_t)p.d) * 4);
   L.decode_bytes = off;
   L.counter_bytes = U * 4;
   L.unit_info = take(U * sizeof(UnitInfo));
@@ -48,15 +40,6 @@ WsLayout ws_layout(const keepkv_params &p) {
   L.stats = take(U * sizeof(keepkv_stats));
   L.total = off;
   return L;
-}
-
-int choose_splits(const keepkv_params &p, int max_splits) {
-  // Two resident CTAs per SM: the largest split factor that still fits one wave of 296 CTAs.
-  const int U = p.B * p.H_kv;
-  int S = (2 * 148) / U;
-  if (S < 1) S = 1;
-  if (S > max_splits) S = max_splits;
-  return S;
 }
 
 static int validate(const keepkv_params *p) {

@@ -10,7 +10,7 @@
 namespace keepkv {
 
 constexpr int kTile = 64;          // entries per K/V tile of the decode kernel
-constexpr int kMaxSplits = 64;     // upper bound on split-KV factor
+constexpr int kDecMaxCtas = 512;    // upper bound on the persistent decode grid (sizes the partial pool)
 
 constexpr int kMaxUnits = 4096;    // B * H_kv that keepkv_compress accepts (per-unit tables live in shared memory)
 constexpr int kNomChunksMax = 8;   // upper bound on the column chunks a row's similarity search is split into
@@ -21,8 +21,7 @@ struct UnitInfo { int len, n_ret, n_ev, n_groups, n_keys, ticket, pad0, pad1; };
 // Byte offsets of the arrays kept in the caller's workspace.  U = B*H_kv, N = N_cap.
 struct WsLayout {
   size_t counters;    // i32 [U]            split-KV arrival counters (zero between calls)
-  size_t part_ml;     // f32 [U,S,G,2]      split-KV partial (max, sum)
-  size_t part_acc;    // f32 [U,S,G,d]      split-KV partial numerators
+  size_t part_pool;   // f32 [kDecMaxCtas,2,16+G*d]  partial results of units cut across CTAs (two per CTA)
   size_t unit_info;   // UnitInfo [U]       len, n_ret, n_ev, n_groups of the running compression
   size_t sched;       // i32 [4]            column-chunk count the nomination kernel settled on
   size_t ret_idx;     // i32 [U,N]          source index of each retained slot, ascending
@@ -37,13 +36,11 @@ struct WsLayout {
   size_t total;
   size_t decode_bytes;   // the leading part that keepkv_decode_attention uses (counters and partials)
   size_t counter_bytes;  // size of the counters array
-  int max_splits;
   int nom_chunks;        // C: column chunks reserved per evicted row
   int key_stride;        // Npow2: N rounded up to a power of two
 };
 
 WsLayout ws_layout(const keepkv_params &p);
-int choose_splits(const keepkv_params &p, int max_splits);
 
 struct LaunchCtx {
   cudaStream_t stream;

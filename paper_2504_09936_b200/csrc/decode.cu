@@ -1,98 +1,64 @@
-// keepkv_decode_attention: Electoral-Votes attention (Eq. 6) over the cache, split along the
-// entry axis (split-KV), with the per-entry score estimate of Eq. 8 advanced in the same pass.
+// keepkv_decode_attention: Electoral-Votes attention (Eq. 6) over the cache, with the per-entry
+// score estimate of Eq. 8 advanced in the same pass.
 //
-// One CTA = 4 warps works through a contiguous range of 64-entry tiles of one (sequence, kv-head)
-// unit.  K/V tiles arrive by TMA (128-byte swizzled boxes) into a 3-stage shared-memory ring,
-// votes and lscore of the tile by bulk copies on the same mbarrier.  Each warp owns 16 entries
-// of a tile: the G query heads of the unit are the rows of an m16n8k16 bf16 MMA (rows >= G are
-// zero), so K is read once for all heads; logits come out in fp32, the vote weight enters as
-// + ln p_i before the online softmax (p_i e^{l_i} = e^{l_i + ln p_i}), and the probabilities go
-// back into the tensor core split into a bf16 head (A rows 0-7) and a bf16 remainder (A rows
-// 8-15) so that P.V keeps fp32-level accuracy in one MMA.
-#include <cuda.h>
-
+// Work is the list of all 64-entry tiles of all (sequence, kv-head) units, in unit order.  A
+// persistent grid (two CTAs per SM) cuts the list into equal contiguous ranges, so ragged batches
+// and any number of units load every SM alike; a unit whose tiles fall into several ranges is
+// finished by the last of those CTAs to arrive (one ticket per unit), in a fixed order, so results
+// are bit-reproducible.
+//
+// One CTA = 4 consumer warps + 1 producer warp.  The producer walks the range and, per tile, issues
+// TMA loads of the K and V tiles (128-byte swizzled boxes), bulk copies of the tile's votes and
+// lscore, and a small descriptor, into a ring of shared-memory stages guarded by full/empty
+// mbarriers.  Each consumer warp owns 16 entries of a tile: the G query heads of the unit are the
+// rows of an m16n8k16 bf16 MMA (rows >= G are zero), so K is read once for all heads; logits come
+// out in fp32; the vote weight enters as + log2 p_i before the online softmax
+// (p_i e^{l_i} = 2^{l_i log2 e + log2 p_i}), and the probabilities go back into the tensor core
+// split into a bf16 head (A rows 0-7) and a bf16 remainder (A rows 8-15), so that P.V keeps
+// fp32-level accuracy in one MMA.  The Eq. 8 update is done by 16 lanes, one entry each, from the
+// logits the warp exchanges through shared memory.
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace keepkv {
 
-constexpr int kDecWarps = 4;
-constexpr int kStages = 3;
-constexpr int kSpinLimit = 1 << 20;
+constexpr int kDecConsumers = 4;                        // warps that do the arithmetic
+constexpr int kDecThreads = 32 * (kDecConsumers + 1);   // + one producer warp
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
 
-// ---------------------------------------------------------------- PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait: gives up after kSpinLimit polls (each poll itself blocks for a short hardware interval).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (int it = 0; it < kSpinLimit; ++it)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, int x, int y, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-      "l"(map), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
-__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
-}
-__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-               : "r"(addr));
-}
-__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-               : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                         uint32_t b1) {
-  asm volatile(
-      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
+// Descriptor the producer leaves with every tile.
+struct TileDesc {
+  int u;          // unit
+  int tile;       // tile index inside the unit
+  int len;        // valid entries of the unit
+  int flags;      // bit 0: first tile of this CTA's segment of the unit, bit 1: last tile of the segment
+  int c_first;    // first CTA that holds a segment of the unit
+  int nparts;     // CTAs that hold a segment of the unit
+  int u_next;     // unit of the next tile of this CTA's range when this tile ends its unit, else -1
+  int pad1;
+};
 
-// Split s of a unit covers tiles [t0, t1).
-__device__ __forceinline__ void split_tiles(int len, int S, int s, int &t0, int &t1) {
-  const int tiles = (len + kTile - 1) / kTile;
-  const int per = (tiles + S - 1) / S;
-  t0 = min(tiles, s * per);
-  t1 = min(tiles, t0 + per);
-}
-
-// Shared-memory layout of one stage: K tile, V tile (each D/64 swizzled sub-tiles of 64 rows x 128 B),
-// then the tile's votes and lscore.
 template <int D>
-struct StageLayout {
+struct DecSmem {
   static constexpr int kSub = D / 64;
   static constexpr int kSubBytes = kTile * 128;
   static constexpr int kK = 0;
   static constexpr int kV = kSub * kSubBytes;
   static constexpr int kVotes = 2 * kSub * kSubBytes;
   static constexpr int kLscore = kVotes + kTile * 4;
-  static constexpr int kBytes = kLscore + kTile * 4;                 // what one stage receives
-  static constexpr int kStride = (kBytes + 1023) / 1024 * 1024;      // sub-tiles need 1024-byte alignment
+  static constexpr int kTxBytes = kLscore + kTile * 4;                 // what the async copies deliver
+  static constexpr int kDesc = kTxBytes;
+  static constexpr int kStride = (kDesc + 32 + 1023) / 1024 * 1024;    // sub-tiles need 1024-byte alignment
+  static constexpr int kStages = D == 128 ? 3 : 6;
+  // Per consumer warp one region that serves two purposes at different times: while the warp works on
+  // a tile, the logits it exchanges (f32 [8 heads][32 entries]) and the log2 votes (f32 [32]); while a
+  // segment is combined, the warp's numerators (f32 [4 heads][D]).  A warp writes its numerators only
+  // after its own tile work, and the others read them only between the barriers of the combine.
+  static constexpr int kWarpRegion = (4 * D * 4 > 8 * 32 * 4 + 32 * 4) ? 4 * D * 4 : 8 * 32 * 4 + 32 * 4;
+  static constexpr int kComb = kStages * kStride;
+  static constexpr int kML = kComb + kDecConsumers * kWarpRegion;      // f32 [4 warps][8][2]
+  static constexpr int kBytes = kML + kDecConsumers * 8 * 2 * 4;
 };
 
 // Byte offset of 16-byte chunk `chunk` (0..D/8-1) of tile row `row` inside a swizzled K or V tile.
@@ -100,334 +66,514 @@ __device__ __forceinline__ uint32_t swz(int row, int chunk) {
   return (uint32_t)((chunk >> 3) * (kTile * 128) + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
 
-// Merge the S partial results of a unit: o = sum_s e^{m_s - M} acc_s / sum_s e^{m_s - M} l_s.
-template <int D, int G>
-__device__ void combine_splits(const keepkv_params &p, int u, int S, const float *part_ml, const float *part_acc,
-                               __nv_bfloat16 *out, float *lse) {
-  const int b = u / p.H_kv, h = u % p.H_kv;
-  for (int idx = threadIdx.x; idx < G * D; idx += blockDim.x) {
-    const int g = idx / D, j = idx % D;
-    float M = -CUDART_INF_F;
-    for (int s = 0; s < S; ++s) M = fmaxf(M, part_ml[(((size_t)u * S + s) * G + g) * 2]);
-    float Lsum = 0.f, acc = 0.f;
-    if (M > -CUDART_INF_F) {
-      for (int s = 0; s < S; ++s) {
-        const size_t o = ((size_t)u * S + s) * G + g;
-        const float w = __expf(part_ml[o * 2] - M);
-        Lsum += w * part_ml[o * 2 + 1];
-        acc += w * part_acc[o * D + j];
-      }
-    }
-    const size_t qo = ((size_t)b * p.H_q + h * G + g);
-    out[qo * D + j] = __float2bfloat16_rn(Lsum > 0.f ? acc / Lsum : 0.f);
-    if (lse && j == 0) lse[qo] = Lsum > 0.f ? M + logf(Lsum) : -CUDART_INF_F;
-  }
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float lg2f(float x) {
+  float y;
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
 }
 
+// One partial result of a unit: running maxima (base-2 exponents), sums and numerators of its G heads.
 template <int D, int G>
-__global__ void __launch_bounds__(kDecWarps * 32, 2)
+struct PartRec {
+  float m[8], l[8];
+  float acc[G * D];
+};
+
+template <int D, int G>
+__global__ void __launch_bounds__(kDecThreads, 2)
 decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, keepkv_params p,
               keepkv_cache c, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *__restrict__ out,
-              float *__restrict__ lse, int update_scores, int *counters, float *part_ml, float *part_acc,
-              int32_t *status_dev) {
-  using SL = StageLayout<D>;
+              float *__restrict__ lse, int update_scores, int *counters, PartRec<D, G> *pool, int32_t *status_dev) {
+  using SL = DecSmem<D>;
+  constexpr int S = SL::kStages;
   constexpr int KS = D / 16;   // k-steps of the QK^T product
   constexpr int NT = D / 8;    // 8-channel n-tiles of the PV product
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t full_bar[kStages];
-  __shared__ int s_abort, s_last;
+  __shared__ __align__(8) uint64_t full_bar[S], empty_bar[S];
+  __shared__ int s_scan[8];
+  __shared__ int s_start[4];   // b, h, tile of the first tile of this CTA's range
+  __shared__ volatile int s_abort;
+  __shared__ int s_last;
 
   // dynamic shared memory is only guaranteed 16-byte aligned: round up to the swizzle atom
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t smem_base = smem_u32(smem);
-
-  const int u = blockIdx.y, s = blockIdx.x, S = gridDim.x;
-  const int b = u / p.H_kv, h = u % p.H_kv;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int g = lane >> 2, qd = lane & 3;   // MMA row (query head) and position inside the quad
-  const int len = max(0, min(c.seq_len[b], p.N_cap));
-  int t0, t1;
-  split_tiles(len, S, s, t0, t1);
-  const int ntiles = t1 - t0;
-  const size_t ubase = (size_t)u * p.N_cap;
+  const int cta = blockIdx.x, grid = gridDim.x;
+  const int U = p.B * p.H_kv;
 
   if (tid == 0) {
-    for (int i = 0; i < kStages; ++i) mbar_init(smem_u32(&full_bar[i]), 1);
+    for (int i = 0; i < S; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), kDecConsumers); }
     s_abort = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    s_start[0] = p.B;
+    mbar_fence_init();
+    fence_proxy_async_smem();
+    prefetch_tensormap(&mapK);
+    prefetch_tensormap(&mapV);
+  }
+
+  // ---- the tile list: every thread sums a block of consecutive sequences, a block scan gives the offsets
+  auto tiles_of = [&](int b) { return (max(0, min(c.seq_len[b], p.N_cap)) + kTile - 1) / kTile; };
+  const int per = (p.B + kDecThreads - 1) / kDecThreads;
+  const int b_lo = min(p.B, tid * per), b_hi = min(p.B, b_lo + per);
+  int mine = 0;
+  for (int b = b_lo; b < b_hi; ++b) mine += tiles_of(b);
+  int incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) s_scan[warp] = incl;
+  __syncthreads();
+  int before = incl - mine, total_b = 0;
+  for (int w = 0; w < kDecConsumers + 1; ++w) {
+    if (w < warp) before += s_scan[w];
+    total_b += s_scan[w];
+  }
+  const long long T = (long long)total_b * p.H_kv;
+  const int chunk = (int)((T + grid - 1) / grid);
+  const long long g0 = min(T, (long long)cta * chunk), g1 = min(T, g0 + chunk);
+  const int ntiles = (int)(g1 - g0);
+  if (ntiles > 0 && (long long)before * p.H_kv <= g0 && g0 < (long long)(before + mine) * p.H_kv) {
+    long long at = (long long)before * p.H_kv;
+    for (int b = b_lo; b < b_hi; ++b) {
+      const int tb = tiles_of(b);
+      const long long span = (long long)tb * p.H_kv;
+      if (g0 < at + span) {
+        const int r = (int)(g0 - at);
+        s_start[0] = b; s_start[1] = r / tb; s_start[2] = r % tb;
+        break;
+      }
+      at += span;
+    }
   }
   __syncthreads();
 
-  auto issue = [&](int stage, int tile) {
-    const uint32_t bar = smem_u32(&full_bar[stage]);
-    const uint32_t dst = smem_base + stage * SL::kStride;
-    const int row = (int)(ubase) + tile * kTile;
-    mbar_expect_tx(bar, SL::kBytes);
+  if (warp == kDecConsumers) {
+    // ------------------------------------------------------------ producer
+    if (lane == 0 && ntiles > 0) {
+      int b = s_start[0], h = s_start[1], tile = s_start[2];
+      int len = max(0, min(c.seq_len[b], p.N_cap));
+      int tb = (len + kTile - 1) / kTile;
+      long long cur = g0;
+      for (int it = 0; it < ntiles; ++it, ++cur) {
+        const int stage = it % S;
+        if (!mbar_wait(smem_u32(&empty_bar[stage]), ((it / S) & 1) ^ 1)) { s_abort = 1; break; }
+        const int u = b * p.H_kv + h;
+        const long long us = cur - tile, ue = us + tb;
+        TileDesc d;
+        d.u = u; d.tile = tile; d.len = len;
+        d.flags = ((it == 0 || tile == 0) ? 1 : 0) | ((it == ntiles - 1 || tile == tb - 1) ? 2 : 0);
+        d.c_first = (int)(us / chunk);
+        d.nparts = (int)((ue - 1) / chunk) - d.c_first + 1;
+        d.u_next = -1;
+        d.pad1 = 0;
+        const size_t ubase = (size_t)u * p.N_cap;
+        const int row = (int)ubase + tile * kTile;
+        const int this_tile = tile;
+        // next tile of the list (units without entries have no tiles)
+        if (++tile == tb && it + 1 < ntiles) {
+          tile = 0;
+          if (++h == p.H_kv) {
+            h = 0;
+            do {
+              ++b;
+              len = max(0, min(c.seq_len[b], p.N_cap));
+              tb = (len + kTile - 1) / kTile;
+            } while (tb == 0);
+          }
+          d.u_next = b * p.H_kv + h;
+        }
+        uint8_t *st = smem + stage * SL::kStride;
+        *reinterpret_cast<TileDesc *>(st + SL::kDesc) = d;
+        const uint32_t bar = smem_u32(&full_bar[stage]);
+        const uint32_t dst = smem_base + stage * SL::kStride;
+        mbar_expect_tx(bar, SL::kTxBytes);
 #pragma unroll
-    for (int sub = 0; sub < SL::kSub; ++sub) {
-      tma_load_2d(dst + SL::kK + sub * SL::kSubBytes, &mapK, sub * 64, row, bar);
-      tma_load_2d(dst + SL::kV + sub * SL::kSubBytes, &mapV, sub * 64, row, bar);
+        for (int sub = 0; sub < SL::kSub; ++sub) {
+          tma_load_2d(dst + SL::kK + sub * SL::kSubBytes, &mapK, sub * 64, row, bar);
+          tma_load_2d(dst + SL::kV + sub * SL::kSubBytes, &mapV, sub * 64, row, bar);
+        }
+        bulk_load_1d(dst + SL::kVotes, c.votes + ubase + (size_t)this_tile * kTile, kTile * 4, bar);
+        bulk_load_1d(dst + SL::kLscore, c.lscore + ubase + (size_t)this_tile * kTile, kTile * 4, bar);
+      }
     }
-    bulk_load_1d(dst + SL::kVotes, c.votes + ubase + (size_t)tile * kTile, kTile * 4, bar);
-    bulk_load_1d(dst + SL::kLscore, c.lscore + ubase + (size_t)tile * kTile, kTile * 4, bar);
-  };
-  if (tid == 0) {
-    for (int i = 0; i < kStages && i < ntiles; ++i) issue(i, t0 + i);
-  }
+  } else {
+    // ------------------------------------------------------------ consumers
+    const int g = lane >> 2, qd = lane & 3;   // MMA row (query head) and position inside the quad
+    const int pair = warp >> 1;               // the two warp pairs take alternate tiles
+    const int r0 = (warp & 1) * 32;           // this warp's 32 rows inside a tile
+    const int ctid = tid;                     // 0..127
+    constexpr int WR = SL::kWarpRegion / 4;   // floats per warp region
+    float *comb = reinterpret_cast<float *>(smem + SL::kComb);
+    float *cml = reinterpret_cast<float *>(smem + SL::kML);
+    float *sc_w = comb + warp * WR;
+    float *lp_w = sc_w + 8 * 32;
 
-  // Q fragments (A operand of QK^T): row g = query head, rows >= G and rows 8-15 are zero.
-  uint32_t qa[KS][2];
-  {
-    const __nv_bfloat16 *qrow = q + ((size_t)b * p.H_q + h * G + (g < G ? g : 0)) * D;
+    // sequences without entries: output 0, lse = -inf
+    for (int u = cta; u < U; u += grid) {
+      const int b = u / p.H_kv, h = u % p.H_kv;
+      if (c.seq_len[b] <= 0) {
+        for (int idx = ctid; idx < G * D; idx += 32 * kDecConsumers)
+          out[((size_t)b * p.H_q + h * G) * D + idx] = __float2bfloat16_rn(0.f);
+        if (lse && ctid < G) lse[(size_t)b * p.H_q + h * G + ctid] = -CUDART_INF_F;
+      }
+    }
+
+    const float ln_alpha = p.ema_alpha > 0.f ? __logf(p.ema_alpha) : -CUDART_INF_F;
+    const float ln_1ma = log1pf(-p.ema_alpha);
+    const float ln_G = __logf((float)G);
+
+    // Q fragments (A operand of QK^T): row g = query head, rows >= G and rows 8-15 are zero.  They are
+    // fetched ahead of the segment that uses them: before the first tile arrives, and while the
+    // previous segment is being combined.
+    uint32_t qa[KS][2];
+    auto load_q = [&](int u) {
+      const int b = u / p.H_kv, h = u % p.H_kv;
+      const __nv_bfloat16 *qrow = q + ((size_t)b * p.H_q + h * G + (g < G ? g : 0)) * D;
 #pragma unroll
-    for (int ks = 0; ks < KS; ++ks) {
-      qa[ks][0] = g < G ? *reinterpret_cast<const uint32_t *>(qrow + ks * 16 + qd * 2) : 0u;
-      qa[ks][1] = g < G ? *reinterpret_cast<const uint32_t *>(qrow + ks * 16 + 8 + qd * 2) : 0u;
-    }
-  }
-  const float ln_alpha = p.ema_alpha > 0.f ? __logf(p.ema_alpha) : -CUDART_INF_F;
-  const float ln_1ma = log1pf(-p.ema_alpha);
-  const float ln_G = __logf((float)G);
-  float *lscore_g = c.lscore + ubase;
-
-  float o[NT][4];
+      for (int ks = 0; ks < KS; ++ks) {
+        qa[ks][0] = g < G ? *reinterpret_cast<const uint32_t *>(qrow + ks * 16 + qd * 2) : 0u;
+        qa[ks][1] = g < G ? *reinterpret_cast<const uint32_t *>(qrow + ks * 16 + 8 + qd * 2) : 0u;
+      }
+    };
+    if (ntiles > 0) load_q(s_start[0] * p.H_kv + s_start[1]);
+    float o[NT][4];
 #pragma unroll
-  for (int nt = 0; nt < NT; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
-  float m_run = -CUDART_INF_F, l_run = 0.f;   // running max and (per-thread partial) sum of head g
+    for (int nt = 0; nt < NT; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
+    float m_run = -CUDART_INF_F, l_run = 0.f;   // running max (base-2 exponent) and per-thread partial sum of head g
 
-  const int r0 = warp * 16;                   // this warp's rows inside a tile
-  for (int it = 0; it < ntiles; ++it) {
-    const int stage = it % kStages;
-    const uint32_t parity = (it / kStages) & 1;
-    if (!mbar_wait(smem_u32(&full_bar[stage]), parity)) {
-      s_abort = 1;
-      atomicOr(status_dev, KEEPKV_DEV_TIMEOUT);
-    }
-    const uint32_t st = smem_base + stage * SL::kStride;
-    const uint8_t *stp = smem + stage * SL::kStride;
-    const int i_base = (t0 + it) * kTile + r0;    // first entry of this warp's slice
-    const int n_valid = len - i_base;              // entries of the slice that exist (may be <= 0 or >= 16)
+    for (int it = 0; it < ntiles; ++it) {
+      const int stage = it % S;
+      {
+        // A tile that never arrives stops all four warps at this same iteration (none can be past it,
+        // none is held at a combine barrier that needs this warp), so leaving the loop here is safe.
+        int ok = 0;
+        if (lane == 0) ok = !s_abort && mbar_wait(smem_u32(&full_bar[stage]), (it / S) & 1);
+        if (!__shfl_sync(0xffffffffu, ok, 0)) { s_abort = 1; break; }
+      }
+      const uint32_t st = smem_base + stage * SL::kStride;
+      const uint8_t *stp = smem + stage * SL::kStride;
+      const TileDesc d = *reinterpret_cast<const TileDesc *>(stp + SL::kDesc);
+      const int b = d.u / p.H_kv, h = d.u % p.H_kv;
 
-    if (n_valid < 16) {
-      // ragged tail: rows past the sequence hold unspecified bits; zero their V so that 0 * garbage
-      // cannot turn into NaN inside the tensor core
-      for (int idx = lane; idx < 16 * (D / 8); idx += 32) {
-        const int r = idx / (D / 8), ch = idx % (D / 8);
-        if (r >= n_valid) *reinterpret_cast<uint4 *>(smem + stage * SL::kStride + SL::kV + swz(r0 + r, ch)) = make_uint4(0, 0, 0, 0);
+      const int i_base = d.tile * kTile + r0;     // first entry of this warp's slice
+      const int n_valid = d.len - i_base;         // entries of the slice that exist (may be <= 0 or >= 32)
+      const bool mine = (it & 1) == pair;
+      if (mine && n_valid > 0) {
+        const bool ragged = n_valid < 32;
+        if (ragged) {
+          // rows past the sequence hold unspecified bits; zero their V so that 0 * garbage cannot turn
+          // into NaN inside the tensor core
+          for (int idx = lane; idx < 32 * (D / 8); idx += 32) {
+            const int r = idx / (D / 8), ch = idx % (D / 8);
+            if (r >= n_valid)
+              *reinterpret_cast<uint4 *>(smem + stage * SL::kStride + SL::kV + swz(r0 + r, ch)) = make_uint4(0, 0, 0, 0);
+          }
+          __syncwarp();
+        }
+
+        // ---- logits: S[head][entry] for the 32 entries, four independent n-tiles of 8
+        float sc[4][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f;
+#pragma unroll
+        for (int kk = 0; kk < KS / 2; ++kk) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int row = r0 + j * 8 + (lane & 7);
+            uint32_t b0, b1, b2, b3;
+            ldsm_x4(st + SL::kK + swz(row, kk * 4 + (lane >> 3)), b0, b1, b2, b3);
+            mma_bf16(sc[j], qa[2 * kk][0], 0u, qa[2 * kk][1], 0u, b0, b1);
+            mma_bf16(sc[j], qa[2 * kk + 1][0], 0u, qa[2 * kk + 1][1], 0u, b2, b3);
+          }
+        }
+        // this thread holds head g, entries e(j,t) = 8 j + 2 qd + t of the slice, in natural-log units
+        float x[4][2];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          x[j][0] = sc[j][0] * p.sm_scale;
+          x[j][1] = sc[j][1] * p.sm_scale;
+          if (g < G) *reinterpret_cast<float2 *>(sc_w + g * 32 + j * 8 + qd * 2) = make_float2(x[j][0], x[j][1]);
+        }
+        __syncwarp();
+
+        // ---- one lane per entry: log2 of the vote; Eq. 8 with the kv head's score = mean over its G heads of e^{l}
+        {
+          const int e = lane;
+          const float pv = reinterpret_cast<const float *>(stp + SL::kVotes)[r0 + e];
+          if (update_scores) {
+            float mx = sc_w[e];
+#pragma unroll
+            for (int gg = 1; gg < G; ++gg) mx = fmaxf(mx, sc_w[gg * 32 + e]);
+            float sigma = mx;
+            if (G > 1) {
+              float se = 0.f;
+#pragma unroll
+              for (int gg = 0; gg < G; ++gg) se += ex2f((sc_w[gg * 32 + e] - mx) * kLog2e);
+              sigma = mx + lg2f(se) * kLn2 - ln_G;
+            }
+            const float old = reinterpret_cast<const float *>(stp + SL::kLscore)[r0 + e];
+            float r = sigma;
+            if (old > -CUDART_INF_F && p.ema_alpha > 0.f) {
+              const float a = ln_alpha + old, bb = ln_1ma + sigma;
+              const float hi = fmaxf(a, bb), lo = fminf(a, bb);
+              r = hi + lg2f(1.f + ex2f((lo - hi) * kLog2e)) * kLn2;
+            }
+            if (e < n_valid) c.lscore[(size_t)d.u * p.N_cap + i_base + e] = r;
+          }
+          lp_w[e] = e < n_valid ? lg2f(pv) : -CUDART_INF_F;
+        }
+        __syncwarp();
+
+        // ---- Eq. 6: weights p_i e^{l_i} = 2^{x log2e + log2 p} through an online softmax
+        float mloc = -CUDART_INF_F;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float2 lp = *reinterpret_cast<const float2 *>(lp_w + j * 8 + qd * 2);
+          x[j][0] = fmaf(x[j][0], kLog2e, lp.x);   // -inf for entries past the sequence
+          x[j][1] = fmaf(x[j][1], kLog2e, lp.y);
+          if (ragged) {   // garbage logits of missing entries may be NaN or +inf
+            if (j * 8 + qd * 2 >= n_valid) x[j][0] = -CUDART_INF_F;
+            if (j * 8 + qd * 2 + 1 >= n_valid) x[j][1] = -CUDART_INF_F;
+          }
+          mloc = fmaxf(mloc, fmaxf(x[j][0], x[j][1]));
+        }
+        mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, 1));
+        mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, 2));
+        const float m_new = fmaxf(m_run, mloc);
+        const bool grow = m_new > m_run;
+        if (__any_sync(0xffffffffu, grow)) {
+          const float scale = grow ? ex2f(m_run - m_new) : 1.f;   // m_run = -inf gives 0; o and l are 0 then anyway
+          l_run *= scale;
+#pragma unroll
+          for (int nt = 0; nt < NT; ++nt) {
+            o[nt][0] *= scale; o[nt][1] *= scale; o[nt][2] *= scale; o[nt][3] *= scale;
+          }
+          m_run = m_new;
+        }
+        // A fragments of P for the two 16-entry k-steps: a0/a2 = bf16 head (rows 0-7), a1/a3 = bf16
+        // remainder (rows 8-15)
+        uint32_t pa[2][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float p0 = m_run > -CUDART_INF_F ? ex2f(x[j][0] - m_run) : 0.f;
+          const float p1 = m_run > -CUDART_INF_F ? ex2f(x[j][1] - m_run) : 0.f;
+          l_run += p0 + p1;
+          const uint32_t hi2 = pack_bf16(p0, p1);
+          pa[j >> 1][2 * (j & 1)] = hi2;
+          pa[j >> 1][2 * (j & 1) + 1] = pack_bf16(p0 - bf16_lo(hi2), p1 - bf16_hi(hi2));
+        }
+        // ---- O += P V   (rows 0-7 collect the head part, rows 8-15 the remainder part)
+#pragma unroll
+        for (int ks = 0; ks < 2; ++ks) {
+          const int vrow = r0 + ks * 16 + (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+          for (int np = 0; np < NT / 2; ++np) {
+            uint32_t b0, b1, b2, b3;
+            ldsm_x4_t(st + SL::kV + swz(vrow, np * 2 + (lane >> 4)), b0, b1, b2, b3);
+            mma_bf16(o[2 * np], pa[ks][0], pa[ks][1], pa[ks][2], pa[ks][3], b0, b1);
+            mma_bf16(o[2 * np + 1], pa[ks][0], pa[ks][1], pa[ks][2], pa[ks][3], b2, b3);
+          }
+        }
+        if (ragged) fence_proxy_async_smem();   // the zeroed V rows precede the next TMA write
       }
       __syncwarp();
-    }
+      if (lane == 0) mbar_arrive(smem_u32(&empty_bar[stage]));   // this warp is done with the stage
 
-    // ---- logits: S[head][entry] for the 16 entries, two n-tiles of 8
-    float sc[2][4];
+      if (d.flags & 2) {
+        // ---- end of this CTA's segment of the unit: combine the four warps
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+        if (g < G && qd == 0) { cml[(warp * 8 + g) * 2] = m_run; cml[(warp * 8 + g) * 2 + 1] = l_run; }
+        const bool whole = d.nparts == 1;
+        PartRec<D, G> *rec = pool + (size_t)cta * 2 + (d.c_first == cta ? 1 : 0);
+        float osum[NT][2];
 #pragma unroll
-    for (int j = 0; j < 2; ++j) sc[j][0] = sc[j][1] = sc[j][2] = sc[j][3] = 0.f;
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      const int row = r0 + j * 8 + (lane & 7);
-#pragma unroll
-      for (int kk = 0; kk < KS / 2; ++kk) {
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4(st + SL::kK + swz(row, kk * 4 + (lane >> 3)), b0, b1, b2, b3);
-        mma_bf16(sc[j], qa[2 * kk][0], 0u, qa[2 * kk][1], 0u, b0, b1);
-        mma_bf16(sc[j], qa[2 * kk + 1][0], 0u, qa[2 * kk + 1][1], 0u, b2, b3);
-      }
-    }
-    // this thread holds head g, entries e(j,t) = i_base + 8 j + 2 qd + t
-    float x[2][2];
-#pragma unroll
-    for (int j = 0; j < 2; ++j)
-#pragma unroll
-      for (int t = 0; t < 2; ++t) x[j][t] = sc[j][t] * p.sm_scale;
-
-    // ---- Eq. 8: score of the kv head = mean over its G heads of e^{l}; kept as a logarithm
-    if (update_scores) {
-      const float *ls_s = reinterpret_cast<const float *>(stp + SL::kLscore) + r0;
-#pragma unroll
-      for (int j = 0; j < 2; ++j) {
-        float sig[2];
-#pragma unroll
-        for (int t = 0; t < 2; ++t) {
-          const float v = g < G ? x[j][t] : -CUDART_INF_F;
-          float mx = v;
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-          float se = __expf(v - mx);
-          se += __shfl_xor_sync(0xffffffffu, se, 4);
-          se += __shfl_xor_sync(0xffffffffu, se, 8);
-          se += __shfl_xor_sync(0xffffffffu, se, 16);
-          sig[t] = mx + __logf(se) - ln_G;
+        for (int nt = 0; nt < NT; ++nt) {
+          osum[nt][0] = o[nt][0] + o[nt][2]; osum[nt][1] = o[nt][1] + o[nt][3];
+          o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
         }
-        if (g == 0) {
-          const int e = j * 8 + qd * 2;
-          float r[2];
+        if (d.u_next >= 0) load_q(d.u_next);   // in flight while this segment is combined
+        m_run = -CUDART_INF_F;
+        l_run = 0.f;
+        constexpr int ROUNDS = (G + 3) / 4, RG = G < 4 ? G : 4;
 #pragma unroll
-          for (int t = 0; t < 2; ++t) {
-            const float old = ls_s[e + t];
-            r[t] = sig[t];
-            if (old > -CUDART_INF_F && p.ema_alpha > 0.f) {
-              const float a = ln_alpha + old, bb = ln_1ma + sig[t];
-              const float mm = fmaxf(a, bb);
-              r[t] = mm + __logf(__expf(a - mm) + __expf(bb - mm));
+        for (int rd = 0; rd < ROUNDS; ++rd) {
+          if (g < G && (g >> 2) == rd) {
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+              *reinterpret_cast<float2 *>(&comb[(size_t)warp * WR + (g & 3) * D + nt * 8 + qd * 2]) =
+                  make_float2(osum[nt][0], osum[nt][1]);
+          }
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          for (int idx = ctid; idx < RG * D; idx += 32 * kDecConsumers) {
+            const int gl = idx / D, j = idx % D, gg = rd * 4 + gl;
+            float M = cml[gg * 2];
+#pragma unroll
+            for (int w = 1; w < kDecConsumers; ++w) M = fmaxf(M, cml[(w * 8 + gg) * 2]);
+            float Ls = 0.f, a = 0.f;
+            if (M > -CUDART_INF_F) {
+#pragma unroll
+              for (int w = 0; w < kDecConsumers; ++w) {
+                const float f = ex2f(cml[(w * 8 + gg) * 2] - M);
+                Ls += f * cml[(w * 8 + gg) * 2 + 1];
+                a += f * comb[(size_t)w * WR + gl * D + j];
+              }
+            }
+            if (whole) {
+              const size_t qo = (size_t)b * p.H_q + h * G + gg;
+              out[qo * D + j] = __float2bfloat16_rn(Ls > 0.f ? a / Ls : 0.f);
+              if (lse && j == 0) lse[qo] = Ls > 0.f ? (M + lg2f(Ls)) * kLn2 : -CUDART_INF_F;
+            } else {
+              rec->acc[gg * D + j] = a;
+              if (j == 0) { rec->m[gg] = M; rec->l[gg] = Ls; }
             }
           }
-          if (e + 1 < n_valid)
-            *reinterpret_cast<float2 *>(lscore_g + i_base + e) = make_float2(r[0], r[1]);
-          else if (e < n_valid)
-            lscore_g[i_base + e] = r[0];
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
+        if (!whole) {
+          // ---- the last CTA of the unit to arrive merges the partials, in CTA order
+          __threadfence();
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          if (ctid == 0) {
+            const int ticket = atomicAdd(&counters[d.u], 1);
+            s_last = (ticket == d.nparts - 1);
+            if (s_last) counters[d.u] = 0;   // ready for the next call
+          }
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          if (s_last) {
+            __threadfence();
+            // comb[part][head] = (m_k, scale factor 2^{m_k - M}); cml[head] = M
+            constexpr int kMaxParts = kDecConsumers * WR / (2 * G);
+            const int np_ = d.nparts;
+            auto part = [&](int k) { return pool + (size_t)(d.c_first + k) * 2 + (k == 0 ? 1 : 0); };
+            constexpr int NI = (G * D + 32 * kDecConsumers - 1) / (32 * kDecConsumers);   // outputs per thread
+            constexpr int KF = NI <= 4 ? 8 : 4;   // parts the register path holds
+            if (np_ <= KF) {
+              // few parts (the usual case): everything in registers, one round trip to L2
+              float pm[KF][NI], pl[KF][NI], pa_[KF][NI];
+#pragma unroll
+              for (int k = 0; k < KF; ++k) {
+                const PartRec<D, G> *r = part(k < np_ ? k : 0);
+#pragma unroll
+                for (int i = 0; i < NI; ++i) {
+                  const int idx = min(ctid + i * 32 * kDecConsumers, G * D - 1);
+                  pm[k][i] = k < np_ ? __ldcg(&r->m[idx / D]) : -CUDART_INF_F;
+                  pl[k][i] = __ldcg(&r->l[idx / D]);
+                  pa_[k][i] = __ldcg(&r->acc[idx]);
+                }
+              }
+#pragma unroll
+              for (int i = 0; i < NI; ++i) {
+                const int idx = ctid + i * 32 * kDecConsumers;
+                float M = pm[0][i];
+#pragma unroll
+                for (int k = 1; k < KF; ++k) M = fmaxf(M, pm[k][i]);
+                float Ls = 0.f, a = 0.f;
+#pragma unroll
+                for (int k = 0; k < KF; ++k) {
+                  const float f = pm[k][i] > -CUDART_INF_F ? ex2f(pm[k][i] - M) : 0.f;
+                  Ls = fmaf(f, pl[k][i], Ls);
+                  a = fmaf(f, pa_[k][i], a);
+                }
+                if (idx < G * D) {
+                  const int gg = idx / D, j = idx % D;
+                  const size_t qo = (size_t)b * p.H_q + h * G + gg;
+                  out[qo * D + j] = __float2bfloat16_rn(Ls > 0.f ? a / Ls : 0.f);
+                  if (lse && j == 0) lse[qo] = Ls > 0.f ? (M + lg2f(Ls)) * kLn2 : -CUDART_INF_F;
+                }
+              }
+            } else if (np_ <= kMaxParts) {
+              for (int idx = ctid; idx < np_ * G; idx += 32 * kDecConsumers)
+                comb[idx * 2] = __ldcg(&part(idx / G)->m[idx % G]);
+              asm volatile("bar.sync 1, 128;" ::: "memory");
+              for (int idx = ctid; idx < np_ * G; idx += 32 * kDecConsumers) {
+                const int gg = idx % G;
+                float M = -CUDART_INF_F;
+                for (int k = 0; k < np_; ++k) M = fmaxf(M, comb[(k * G + gg) * 2]);
+                comb[idx * 2 + 1] = M > -CUDART_INF_F ? ex2f(comb[idx * 2] - M) : 0.f;
+                if (idx < G) cml[gg] = M;
+              }
+              asm volatile("bar.sync 1, 128;" ::: "memory");
+              // every thread owns NI outputs; the parts are the outer loop so that all loads of a part
+              // are in flight together
+              float Ls[NI], a[NI];
+#pragma unroll
+              for (int i = 0; i < NI; ++i) Ls[i] = a[i] = 0.f;
+#pragma unroll 2
+              for (int k = 0; k < np_; ++k) {
+                const PartRec<D, G> *r = part(k);
+#pragma unroll
+                for (int i = 0; i < NI; ++i) {
+                  const int idx = ctid + i * 32 * kDecConsumers;
+                  if (idx < G * D) {
+                    const int gg = idx / D;
+                    const float f = comb[(k * G + gg) * 2 + 1];
+                    Ls[i] = fmaf(f, __ldcg(&r->l[gg]), Ls[i]);
+                    a[i] = fmaf(f, __ldcg(&r->acc[idx]), a[i]);
+                  }
+                }
+              }
+#pragma unroll
+              for (int i = 0; i < NI; ++i) {
+                const int idx = ctid + i * 32 * kDecConsumers;
+                if (idx < G * D) {
+                  const int gg = idx / D, j = idx % D;
+                  const size_t qo = (size_t)b * p.H_q + h * G + gg;
+                  out[qo * D + j] = __float2bfloat16_rn(Ls[i] > 0.f ? a[i] / Ls[i] : 0.f);
+                  if (lse && j == 0) lse[qo] = Ls[i] > 0.f ? (cml[gg] + lg2f(Ls[i])) * kLn2 : -CUDART_INF_F;
+                }
+              }
+            } else {
+              for (int idx = ctid; idx < G * D; idx += 32 * kDecConsumers) {
+                const int gg = idx / D, j = idx % D;
+                float M = -CUDART_INF_F;
+                for (int k = 0; k < np_; ++k) M = fmaxf(M, __ldcg(&part(k)->m[gg]));
+                float Ls = 0.f, a = 0.f;
+                if (M > -CUDART_INF_F) {
+                  for (int k = 0; k < np_; ++k) {
+                    const float f = ex2f(__ldcg(&part(k)->m[gg]) - M);
+                    Ls = fmaf(f, __ldcg(&part(k)->l[gg]), Ls);
+                    a = fmaf(f, __ldcg(&part(k)->acc[gg * D + j]), a);
+                  }
+                }
+                const size_t qo = (size_t)b * p.H_q + h * G + gg;
+                out[qo * D + j] = __float2bfloat16_rn(Ls > 0.f ? a / Ls : 0.f);
+                if (lse && j == 0) lse[qo] = Ls > 0.f ? (M + lg2f(Ls)) * kLn2 : -CUDART_INF_F;
+              }
+            }
+          }
+          asm volatile("bar.sync 1, 128;" ::: "memory");   // s_last is reused by the next segment
         }
       }
     }
-
-    // ---- Eq. 6: weights p_i e^{l_i} through an online softmax over x + ln p
-    const float *vt_s = reinterpret_cast<const float *>(stp + SL::kVotes) + r0;
-    float mloc = -CUDART_INF_F;
-#pragma unroll
-    for (int j = 0; j < 2; ++j)
-#pragma unroll
-      for (int t = 0; t < 2; ++t) {
-        const int e = j * 8 + qd * 2 + t;
-        x[j][t] = e < n_valid ? x[j][t] + __logf(vt_s[e]) : -CUDART_INF_F;
-        mloc = fmaxf(mloc, x[j][t]);
-      }
-    mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, 1));
-    mloc = fmaxf(mloc, __shfl_xor_sync(0xffffffffu, mloc, 2));
-    const float m_new = fmaxf(m_run, mloc);
-    const bool grow = m_new > m_run;
-    if (__any_sync(0xffffffffu, grow)) {
-      const float scale = grow ? __expf(m_run - m_new) : 1.f;   // m_run = -inf gives 0, o and l are 0 then anyway
-      l_run *= scale;
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        o[nt][0] *= scale; o[nt][1] *= scale; o[nt][2] *= scale; o[nt][3] *= scale;
-      }
-      m_run = m_new;
-    }
-    uint32_t pa[4];   // A fragment of P: a0/a2 = bf16 head (rows 0-7), a1/a3 = bf16 remainder (rows 8-15)
-#pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      float pr[2], hi[2];
-#pragma unroll
-      for (int t = 0; t < 2; ++t) {
-        pr[t] = m_run > -CUDART_INF_F ? __expf(x[j][t] - m_run) : 0.f;
-        l_run += pr[t];
-        hi[t] = __bfloat162float(__float2bfloat16_rn(pr[t]));
-      }
-      pa[2 * j] = pack_bf16(hi[0], hi[1]);
-      pa[2 * j + 1] = pack_bf16(pr[0] - hi[0], pr[1] - hi[1]);
-    }
-    // ---- O += P V   (rows 0-7 collect the head part, rows 8-15 the remainder part)
-    {
-      const int vrow = r0 + (lane & 7) + ((lane >> 3) & 1) * 8;
-#pragma unroll
-      for (int np = 0; np < NT / 2; ++np) {
-        uint32_t b0, b1, b2, b3;
-        ldsm_x4_t(st + SL::kV + swz(vrow, np * 2 + (lane >> 4)), b0, b1, b2, b3);
-        mma_bf16(o[2 * np], pa[0], pa[1], pa[2], pa[3], b0, b1);
-        mma_bf16(o[2 * np + 1], pa[0], pa[1], pa[2], pa[3], b2, b3);
-      }
-    }
-    __syncthreads();   // every warp is done with this stage
-    if (s_abort) break;
-    if (tid == 0 && it + kStages < ntiles) {
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      issue(stage, t0 + it + kStages);
-    }
   }
+
+  __syncthreads();
   if (s_abort) {
     // give copies still in flight a bounded chance to land before the CTA's shared memory goes away
-    __syncthreads();
-    if (tid == 0)
-      for (int i = 0; i < kStages; ++i) { mbar_wait(smem_u32(&full_bar[i]), 0); mbar_wait(smem_u32(&full_bar[i]), 1); }
-    __syncthreads();
-  }
-
-  // ---- combine the four warps of this CTA (stage memory is free now)
-  l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-  l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-  float *cm = reinterpret_cast<float *>(smem);            // [warps][8]
-  float *cl = cm + kDecWarps * 8;                          // [warps][8]
-  float *co = cl + kDecWarps * 8;                          // [warps][G][D]
-  if (g < G) {
-    if (qd == 0) { cm[warp * 8 + g] = m_run; cl[warp * 8 + g] = l_run; }
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) {
-      const float2 v = make_float2(o[nt][0] + o[nt][2], o[nt][1] + o[nt][3]);
-      *reinterpret_cast<float2 *>(&co[((size_t)warp * G + g) * D + nt * 8 + qd * 2]) = v;
+    if (tid == 0) {
+      atomicOr(status_dev, KEEPKV_DEV_TIMEOUT);
+      for (int i = 0; i < S; ++i) { mbar_wait(smem_u32(&full_bar[i]), 0); mbar_wait(smem_u32(&full_bar[i]), 1); }
     }
-  }
-  __syncthreads();
-  for (int idx = tid; idx < G * D; idx += blockDim.x) {
-    const int gg = idx / D, j = idx % D;
-    float M = cm[gg];
-#pragma unroll
-    for (int w = 1; w < kDecWarps; ++w) M = fmaxf(M, cm[w * 8 + gg]);
-    float Ls = 0.f, a = 0.f;
-    if (M > -CUDART_INF_F) {
-#pragma unroll
-      for (int w = 0; w < kDecWarps; ++w) {
-        const float f = __expf(cm[w * 8 + gg] - M);
-        Ls += f * cl[w * 8 + gg];
-        a += f * co[((size_t)w * G + gg) * D + j];
-      }
-    }
-    const size_t oo = ((size_t)u * S + s) * G + gg;
-    part_acc[oo * D + j] = a;
-    if (j == 0) { part_ml[oo * 2] = M; part_ml[oo * 2 + 1] = Ls; }
-  }
-  // ---- the last CTA of the unit to arrive merges the partials
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    const int ticket = atomicAdd(&counters[u], 1);
-    s_last = (ticket == S - 1);
-    if (s_last) counters[u] = 0;   // ready for the next call
-  }
-  __syncthreads();
-  if (s_last) {
-    __threadfence();
-    combine_splits<D, G>(p, u, S, part_ml, part_acc, out, lse);
+    __syncthreads();
   }
 }
 
 // ---------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  if (!fn) {
-    void *ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
-}
-
-// Tensor map over a [rows, D] bf16 matrix with boxes of 64 rows x 64 channels, 128-byte swizzle;
-// rows past the end read as zero.
-static bool make_map(CUtensorMap *map, void *base, uint64_t rows, int D) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)D * 2};
-  cuuint32_t box[2] = {64, (cuuint32_t)kTile};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 template <int D, int G>
 static void launch_t(const keepkv_params &p, const keepkv_cache &c, const void *q, void *out, float *lse,
                      int update_scores, char *ws, const WsLayout &L, int32_t *status_dev, LaunchCtx &ctx) {
-  using SL = StageLayout<D>;
-  constexpr size_t smem_bytes = (size_t)kStages * SL::kStride + 1024;
+  using SL = DecSmem<D>;
+  constexpr size_t smem_bytes = (size_t)SL::kBytes + 1024;
+  static_assert(sizeof(PartRec<D, G>) == (16 + G * D) * 4, "partial record layout");
   static bool attr_done_dev[64] = {};
   int dev = 0;
   cudaGetDevice(&dev);
@@ -437,16 +583,19 @@ static void launch_t(const keepkv_params &p, const keepkv_cache &c, const void *
   }
   CUtensorMap mapK, mapV;
   const uint64_t rows = (uint64_t)p.B * p.H_kv * p.N_cap;
-  if (!make_map(&mapK, c.K, rows, D) || !make_map(&mapV, c.V, rows, D)) {
+  if (!make_bf16_rows_map(&mapK, c.K, rows, D, kTile) || !make_bf16_rows_map(&mapV, c.V, rows, D, kTile)) {
     if (ctx.err == cudaSuccess) ctx.err = cudaErrorInvalidValue;
     return;
   }
-  const int S = choose_splits(p, L.max_splits);
-  dim3 grid(S, p.B * p.H_kv);
-  decode_kernel<D, G><<<grid, kDecWarps * 32, smem_bytes, ctx.stream>>>(
+  // two CTAs per SM, never more than tiles could exist or than the partial pool holds
+  const long long max_tiles = (long long)p.B * p.H_kv * (p.N_cap / kTile);
+  long long grid = 2LL * sm_count();
+  if (grid > kDecMaxCtas) grid = kDecMaxCtas;
+  if (grid > max_tiles) grid = max_tiles;
+  decode_kernel<D, G><<<(unsigned)grid, kDecThreads, smem_bytes, ctx.stream>>>(
       mapK, mapV, p, c, reinterpret_cast<const __nv_bfloat16 *>(q), reinterpret_cast<__nv_bfloat16 *>(out), lse,
-      update_scores, reinterpret_cast<int *>(ws + L.counters), reinterpret_cast<float *>(ws + L.part_ml),
-      reinterpret_cast<float *>(ws + L.part_acc), status_dev);
+      update_scores, reinterpret_cast<int *>(ws + L.counters), reinterpret_cast<PartRec<D, G> *>(ws + L.part_pool),
+      status_dev);
   KEEPKV_CHECK_LAUNCH(ctx);
 }
 

@@ -19,7 +19,7 @@ from paper_2504_09936_b200 import binding as kb
 def test_static_scratch_refuses_shapes_beyond_its_size():
     """A shape whose split-KV partials do not fit the built-in array is refused on the host, before
     any CUDA call, with KEEPKV_ERR_WORKSPACE."""
-    p = kb.make_params(B=512, H_q=256, H_kv=32, d=128, N_cap=4096)      # 16384 units x 8 heads x 130 floats > 8 MiB
+    p = kb.make_params(B=65536, H_q=128, H_kv=16, d=128, N_cap=64)     # 2^20 unit counters + the partial pool > 8 MiB
     dummy = C.c_void_p(256)
     cache = kb.keepkv_cache(256, 256, 256, 256, 256)
     rc = kb.lib().keepkv_decode_attention_static(C.byref(p), C.byref(cache), dummy, dummy, None, 0, dummy, None)
