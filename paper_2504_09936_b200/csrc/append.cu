@@ -8,6 +8,8 @@ namespace keepkv {
 __global__ void __launch_bounds__(128) append_kernel(keepkv_params p, keepkv_cache c, const uint4 *__restrict__ k_new,
                                                      const uint4 *__restrict__ v_new, int32_t *status_dev) {
   const int b = blockIdx.x;
+  pdl_wait();
+  pdl_trigger();
   const int pos = c.seq_len[b];
   if (pos >= p.N_cap) {
     if (threadIdx.x == 0) atomicOr(status_dev, KEEPKV_DEV_APPEND_FULL);
@@ -33,8 +35,8 @@ __global__ void __launch_bounds__(128) append_kernel(keepkv_params p, keepkv_cac
 
 void launch_append(const keepkv_params &p, const keepkv_cache &c, const void *k_new, const void *v_new,
                    int32_t *status_dev, LaunchCtx &ctx) {
-  append_kernel<<<p.B, 128, 0, ctx.stream>>>(p, c, reinterpret_cast<const uint4 *>(k_new),
-                                             reinterpret_cast<const uint4 *>(v_new), status_dev);
+  launch_pdl(append_kernel, dim3(p.B), dim3(128), 0, ctx.stream, p, c, reinterpret_cast<const uint4 *>(k_new),
+             reinterpret_cast<const uint4 *>(v_new), status_dev);
   KEEPKV_CHECK_LAUNCH(ctx);
 }
 

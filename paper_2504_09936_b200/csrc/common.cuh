@@ -5,6 +5,8 @@
 #include <math_constants.h>
 #include <stdint.h>
 
+#include <utility>
+
 #include "keepkv.h"
 
 namespace keepkv {
@@ -65,6 +67,29 @@ void launch_nominate(const keepkv_params &p, const keepkv_cache &src, const keep
                      const UnitInfo *unit_info, const float *inv_norm, int32_t *sched, float4 *nom_v, int32_t *nom_si,
                      int nom_chunks, int32_t *status_dev, LaunchCtx &ctx);
 int sm_count();
+
+// Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor in
+// the stream is still draining, and runs its preamble (barrier set-up, tensor-map prefetch, tensor
+// memory allocation) there.  Every kernel of this library calls pdl_wait() before it touches global
+// memory, which blocks until the predecessor has completed and its writes are visible, so stream
+// order is preserved; pdl_trigger() lets the successor start its own preamble early.
+template <typename... KArgs, typename... Args>
+inline void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                       Args &&...args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 #define KEEPKV_CHECK_LAUNCH(ctx)                        \
   do {                                                  \

@@ -73,6 +73,8 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
   __shared__ uint32_t s_prefix;
   __shared__ int s_kr;
   const int u = blockIdx.x, b = u / p.H_kv, h = u % p.H_kv, tid = threadIdx.x;
+  pdl_wait();
+  pdl_trigger();
   const int len = max(0, min(src.seq_len[b], p.N_cap));
   int budget = budget_dev ? budget_dev[b] : budget_scalar;
   budget = max(0, min(budget, p.N_cap));
@@ -196,6 +198,8 @@ __global__ void __launch_bounds__(256)
 compact_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_t *__restrict__ ret_idx,
                const UnitInfo *__restrict__ unit_info, float *__restrict__ inv_norm) {
   constexpr int CH = D / 8;       // 16-byte chunks per row
+  pdl_wait();
+  pdl_trigger();
   const int u = blockIdx.y, n_ret = unit_info[u].n_ret;
   const int s0 = blockIdx.x * 64;
   if (s0 >= n_ret) return;
@@ -273,6 +277,8 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
       q_b[kResolveThreads];
   __shared__ int res_slot[kResolveThreads], res_merge[kResolveThreads];
   const int u = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  pdl_wait();
+  pdl_trigger();
   const UnitInfo ui = unit_info[u];
   const size_t base = (size_t)u * p.N_cap;
   const __nv_bfloat16 *sK = reinterpret_cast<const __nv_bfloat16 *>(src.K) + base * D;
@@ -417,6 +423,8 @@ merge_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_t 
              keepkv_stats *stats) {
   constexpr int EPL = D / 32;
   const int u = blockIdx.y, lane = threadIdx.x & 31;
+  pdl_wait();
+  pdl_trigger();
   const UnitInfo ui = unit_info[u];
   const size_t base = (size_t)u * p.N_cap;
   const uint32_t *gk = grp_key + (size_t)u * key_stride;
@@ -521,21 +529,22 @@ static void launch_compress_t(const keepkv_params &p, const keepkv_cache &src, c
     cudaFuncSetAttribute(resolve_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
     attr_done = true;
   }
-  select_kernel<<<U, 1024, sel_smem, ctx.stream>>>(p, src, dst.seq_len, budget_dev, budget_scalar, n_recent_dev,
-                                                   ret_idx, target, ev_idx, ui, stats);
+  launch_pdl(select_kernel, dim3(U), dim3(1024), sel_smem, ctx.stream, p, src, dst.seq_len, budget_dev, budget_scalar,
+             n_recent_dev, ret_idx, target, ev_idx, ui, stats);
   KEEPKV_CHECK_LAUNCH(ctx);
   if (ret_bound <= 0) return;   // nothing is kept: every entry is dropped, which select has recorded
-  compact_kernel<D><<<dim3((ret_bound + 63) / 64, U), 256, 0, ctx.stream>>>(p, src, dst, ret_idx, ui, inv_norm);
+  launch_pdl(compact_kernel<D>, dim3((ret_bound + 63) / 64, U), dim3(256), 0, ctx.stream, p, src, dst, ret_idx, ui,
+             inv_norm);
   KEEPKV_CHECK_LAUNCH(ctx);
   launch_nominate(p, src, dst, ev_idx, ui, inv_norm, sched, nom_v, nom_si, L.nom_chunks, status_dev, ctx);
-  resolve_kernel<D><<<dim3(L.nom_chunks, U), kResolveThreads, (size_t)smem_keys * 4, ctx.stream>>>(
+  launch_pdl(resolve_kernel<D>, dim3(L.nom_chunks, U), dim3(kResolveThreads), (size_t)smem_keys * 4, ctx.stream,
       p, src, dst, ev_idx, ui, nom_v, nom_si, sched, L.nom_chunks, target, grp_key, L.key_stride, grp_head, stats,
       smem_keys);
   KEEPKV_CHECK_LAUNCH(ctx);
   int gx = 4096 / U;
   gx = gx < 1 ? 1 : (gx > 32 ? 32 : gx);
-  merge_kernel<D><<<dim3(gx, U), 256, 0, ctx.stream>>>(p, src, dst, ret_idx, ev_idx, target, ui, grp_key,
-                                                        L.key_stride, grp_head, stats);
+  launch_pdl(merge_kernel<D>, dim3(gx, U), dim3(256), 0, ctx.stream, p, src, dst, ret_idx, ev_idx, target, ui, grp_key,
+             L.key_stride, grp_head, stats);
   KEEPKV_CHECK_LAUNCH(ctx);
 }
 

@@ -7,23 +7,24 @@
 // finished by the last of those CTAs to arrive (one ticket per unit), in a fixed order, so results
 // are bit-reproducible.
 //
-// One CTA = 4 consumer warps + 1 producer warp.  The producer walks the range and, per tile, issues
-// TMA loads of the K and V tiles (128-byte swizzled boxes), bulk copies of the tile's votes and
-// lscore, and a small descriptor, into a ring of shared-memory stages guarded by full/empty
-// mbarriers.  Each consumer warp owns 16 entries of a tile: the G query heads of the unit are the
+// One CTA = 4 warps.  Thread 0 also walks the range as producer: per tile it issues TMA loads of the
+// K and V tiles (128-byte swizzled boxes), bulk copies of the tile's votes and lscore, and a small
+// descriptor, into a ring of shared-memory stages guarded by full/empty mbarriers, two tiles ahead
+// of the arithmetic.  The two warp pairs take alternate tiles; a warp owns 32 entries of its tile:
+// the G query heads of the unit are the
 // rows of an m16n8k16 bf16 MMA (rows >= G are zero), so K is read once for all heads; logits come
 // out in fp32; the vote weight enters as + log2 p_i before the online softmax
 // (p_i e^{l_i} = 2^{l_i log2 e + log2 p_i}), and the probabilities go back into the tensor core
 // split into a bf16 head (A rows 0-7) and a bf16 remainder (A rows 8-15), so that P.V keeps
-// fp32-level accuracy in one MMA.  The Eq. 8 update is done by 16 lanes, one entry each, from the
-// logits the warp exchanges through shared memory.
+// fp32-level accuracy in one MMA.  The Eq. 8 update is done one entry per lane, from the logits the
+// warp exchanges through shared memory.
 #include "common.cuh"
 #include "ptx.cuh"
 
 namespace keepkv {
 
-constexpr int kDecConsumers = 4;                        // warps that do the arithmetic
-constexpr int kDecThreads = 32 * (kDecConsumers + 1);   // + one producer warp
+constexpr int kDecConsumers = 4;                  // warps per CTA
+constexpr int kDecThreads = 32 * kDecConsumers;   // 128 threads leave each of them up to 255 registers at two CTAs per SM
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -116,6 +117,8 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     prefetch_tensormap(&mapK);
     prefetch_tensormap(&mapV);
   }
+  pdl_wait();      // everything above ran while the previous kernel of the stream was finishing
+  pdl_trigger();
 
   // ---- the tile list: every thread sums a block of consecutive sequences, a block scan gives the offsets
   auto tiles_of = [&](int b) { return (max(0, min(c.seq_len[b], p.N_cap)) + kTile - 1) / kTile; };
@@ -132,7 +135,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   if (lane == 31) s_scan[warp] = incl;
   __syncthreads();
   int before = incl - mine, total_b = 0;
-  for (int w = 0; w < kDecConsumers + 1; ++w) {
+  for (int w = 0; w < kDecConsumers; ++w) {
     if (w < warp) before += s_scan[w];
     total_b += s_scan[w];
   }
@@ -155,57 +158,64 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   }
   __syncthreads();
 
-  if (warp == kDecConsumers) {
-    // ------------------------------------------------------------ producer
-    if (lane == 0 && ntiles > 0) {
-      int b = s_start[0], h = s_start[1], tile = s_start[2];
-      int len = max(0, min(c.seq_len[b], p.N_cap));
-      int tb = (len + kTile - 1) / kTile;
-      long long cur = g0;
-      for (int it = 0; it < ntiles; ++it, ++cur) {
-        const int stage = it % S;
-        if (!mbar_wait(smem_u32(&empty_bar[stage]), ((it / S) & 1) ^ 1)) { s_abort = 1; break; }
-        const int u = b * p.H_kv + h;
-        const long long us = cur - tile, ue = us + tb;
-        TileDesc d;
-        d.u = u; d.tile = tile; d.len = len;
-        d.flags = ((it == 0 || tile == 0) ? 1 : 0) | ((it == ntiles - 1 || tile == tb - 1) ? 2 : 0);
-        d.c_first = (int)(us / chunk);
-        d.nparts = (int)((ue - 1) / chunk) - d.c_first + 1;
-        d.u_next = -1;
-        d.pad1 = 0;
-        const size_t ubase = (size_t)u * p.N_cap;
-        const int row = (int)ubase + tile * kTile;
-        const int this_tile = tile;
-        // next tile of the list (units without entries have no tiles)
-        if (++tile == tb && it + 1 < ntiles) {
-          tile = 0;
-          if (++h == p.H_kv) {
-            h = 0;
-            do {
-              ++b;
-              len = max(0, min(c.seq_len[b], p.N_cap));
-              tb = (len + kTile - 1) / kTile;
-            } while (tb == 0);
-          }
-          d.u_next = b * p.H_kv + h;
-        }
-        uint8_t *st = smem + stage * SL::kStride;
-        *reinterpret_cast<TileDesc *>(st + SL::kDesc) = d;
-        const uint32_t bar = smem_u32(&full_bar[stage]);
-        const uint32_t dst = smem_base + stage * SL::kStride;
-        mbar_expect_tx(bar, SL::kTxBytes);
-#pragma unroll
-        for (int sub = 0; sub < SL::kSub; ++sub) {
-          tma_load_2d(dst + SL::kK + sub * SL::kSubBytes, &mapK, sub * 64, row, bar);
-          tma_load_2d(dst + SL::kV + sub * SL::kSubBytes, &mapV, sub * 64, row, bar);
-        }
-        bulk_load_1d(dst + SL::kVotes, c.votes + ubase + (size_t)this_tile * kTile, kTile * 4, bar);
-        bulk_load_1d(dst + SL::kLscore, c.lscore + ubase + (size_t)this_tile * kTile, kTile * 4, bar);
+  // ------------------------------------------------------------ producer state (thread 0)
+  int pb = 0, ph = 0, ptile = 0, plen = 0, ptb = 1, pit = 0;
+  if (tid == 0 && ntiles > 0) {
+    pb = s_start[0]; ph = s_start[1]; ptile = s_start[2];
+    plen = max(0, min(c.seq_len[pb], p.N_cap));
+    ptb = (plen + kTile - 1) / kTile;
+  }
+  // Issues the copies of tile `pit` of the range (thread 0 only); false if the stage never came free.
+  auto issue_tile = [&]() -> bool {
+    const int it = pit, stage = it % S;
+    if (!mbar_wait(smem_u32(&empty_bar[stage]), ((it / S) & 1) ^ 1)) return false;
+    const long long cur = g0 + it;
+    const int u = pb * p.H_kv + ph;
+    const long long us = cur - ptile, ue = us + ptb;
+    TileDesc d;
+    d.u = u; d.tile = ptile; d.len = plen;
+    d.flags = ((it == 0 || ptile == 0) ? 1 : 0) | ((it == ntiles - 1 || ptile == ptb - 1) ? 2 : 0);
+    d.c_first = (int)(us / chunk);
+    d.nparts = (int)((ue - 1) / chunk) - d.c_first + 1;
+    d.u_next = -1;
+    d.pad1 = 0;
+    const size_t ubase = (size_t)u * p.N_cap;
+    const int row = (int)ubase + ptile * kTile;
+    const int this_tile = ptile;
+    // next tile of the list (units without entries have no tiles)
+    if (++ptile == ptb && it + 1 < ntiles) {
+      ptile = 0;
+      if (++ph == p.H_kv) {
+        ph = 0;
+        do {
+          ++pb;
+          plen = max(0, min(c.seq_len[pb], p.N_cap));
+          ptb = (plen + kTile - 1) / kTile;
+        } while (ptb == 0);
       }
+      d.u_next = pb * p.H_kv + ph;
     }
-  } else {
-    // ------------------------------------------------------------ consumers
+    uint8_t *st = smem + stage * SL::kStride;
+    *reinterpret_cast<TileDesc *>(st + SL::kDesc) = d;
+    const uint32_t bar = smem_u32(&full_bar[stage]);
+    const uint32_t dst = smem_base + stage * SL::kStride;
+    mbar_expect_tx(bar, SL::kTxBytes);
+#pragma unroll
+    for (int sub = 0; sub < SL::kSub; ++sub) {
+      tma_load_2d(dst + SL::kK + sub * SL::kSubBytes, &mapK, sub * 64, row, bar);
+      tma_load_2d(dst + SL::kV + sub * SL::kSubBytes, &mapV, sub * 64, row, bar);
+    }
+    bulk_load_1d(dst + SL::kVotes, c.votes + ubase + (size_t)this_tile * kTile, kTile * 4, bar);
+    bulk_load_1d(dst + SL::kLscore, c.lscore + ubase + (size_t)this_tile * kTile, kTile * 4, bar);
+    ++pit;
+    return true;
+  };
+  if (tid == 0)
+    while (pit < ntiles && pit < S - 1)
+      if (!issue_tile()) { s_abort = 1; break; }
+
+  {
+    // ------------------------------------------------------------ the arithmetic
     const int g = lane >> 2, qd = lane & 3;   // MMA row (query head) and position inside the quad
     const int pair = warp >> 1;               // the two warp pairs take alternate tiles
     const int r0 = (warp & 1) * 32;           // this warp's 32 rows inside a tile
@@ -251,6 +261,10 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
 
     for (int it = 0; it < ntiles; ++it) {
       const int stage = it % S;
+      // keep the ring S-1 tiles ahead: the stage of tile it-1 is free once all four warps have left it
+      if (tid == 0 && pit < ntiles && pit <= it + S - 1 && !s_abort)
+        if (!issue_tile()) s_abort = 1;
+      __syncwarp();
       {
         // A tile that never arrives stops all four warps at this same iteration (none can be past it,
         // none is held at a combine barrier that needs this warp), so leaving the loop here is safe.
@@ -592,7 +606,7 @@ static void launch_t(const keepkv_params &p, const keepkv_cache &c, const void *
   long long grid = 2LL * sm_count();
   if (grid > kDecMaxCtas) grid = kDecMaxCtas;
   if (grid > max_tiles) grid = max_tiles;
-  decode_kernel<D, G><<<(unsigned)grid, kDecThreads, smem_bytes, ctx.stream>>>(
+  launch_pdl(decode_kernel<D, G>, dim3((unsigned)grid), dim3(kDecThreads), smem_bytes, ctx.stream,
       mapK, mapV, p, c, reinterpret_cast<const __nv_bfloat16 *>(q), reinterpret_cast<__nv_bfloat16 *>(out), lse,
       update_scores, reinterpret_cast<int *>(ws + L.counters), reinterpret_cast<PartRec<D, G> *>(ws + L.part_pool),
       status_dev);

@@ -141,6 +141,8 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
     tmem_alloc(smem_u32(&s_tmem), 512);
     tmem_relinquish();
   }
+  pdl_wait();      // barrier set-up and tensor-memory allocation overlap the previous kernel's tail
+  pdl_trigger();
   if (warp == 2) {   // exclusive prefix of 128-row tiles over the units
     int run = 0;
     for (int u0 = 0; u0 < U; u0 += 32) {
@@ -399,7 +401,7 @@ static void launch_nominate_t(const keepkv_params &p, const keepkv_cache &src, c
     if (ctx.err == cudaSuccess) ctx.err = cudaErrorInvalidValue;
     return;
   }
-  nominate_kernel<D><<<sm_count(), kNomThreads, smem_bytes, ctx.stream>>>(
+  launch_pdl(nominate_kernel<D>, dim3(sm_count()), dim3(kNomThreads), smem_bytes, ctx.stream,
       mapB, p, reinterpret_cast<const __nv_bfloat16 *>(src.K), ev_idx, unit_info, inv_norm, sched, nom_v, nom_si,
       nom_chunks, status_dev);
   KEEPKV_CHECK_LAUNCH(ctx);
