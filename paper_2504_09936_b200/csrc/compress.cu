@@ -12,9 +12,14 @@
 namespace keepkv {
 
 // ------------------------------------------------------------------ block scan of 0/1 flags
-// Exclusive prefix count of `flag` over the block in thread order; total returned through `total`.
+// Exclusive prefix count of `flag` over the first nw warps of the block in thread order (the other
+// warps have left the kernel); total returned through `total`.
+__device__ __forceinline__ int block_excl_count(bool flag, int *warp_tot, int &total, int nw);
 __device__ __forceinline__ int block_excl_count(bool flag, int *warp_tot, int &total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  return block_excl_count(flag, warp_tot, total, (int)(blockDim.x >> 5));
+}
+__device__ __forceinline__ int block_excl_count(bool flag, int *warp_tot, int &total, int nw) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const unsigned bal = __ballot_sync(0xffffffffu, flag);
   const int in_warp = __popc(bal & ((1u << lane) - 1u));
   __syncthreads();  // warp_tot may still be read from the previous call
@@ -31,8 +36,8 @@ __device__ __forceinline__ int block_excl_count(bool flag, int *warp_tot, int &t
 }
 
 // Exclusive prefix sum of small non-negative ints over the block (thread order).
-__device__ __forceinline__ int block_excl_sum(int v, int *warp_tot, int &total) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = blockDim.x >> 5;
+__device__ __forceinline__ int block_excl_sum(int v, int *warp_tot, int &total, int nw) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int x = v;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -51,6 +56,8 @@ __device__ __forceinline__ int block_excl_sum(int v, int *warp_tot, int &total) 
   total = tot;
   return off + x - v;
 }
+
+constexpr int kWarpSelectMax = 2048;   // candidate sets up to this size are searched by one warp, without block barriers
 
 // Order-preserving map of an fp32 value to u32 (-0 folded onto +0 so equal floats give equal keys).
 __device__ __forceinline__ uint32_t ordered_key(float x) {
@@ -71,7 +78,7 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
   __shared__ int hist[256];
   __shared__ int warp_tot[32];
   __shared__ uint32_t s_prefix;
-  __shared__ int s_kr;
+  __shared__ int s_kr, s_cnt;
   const int u = blockIdx.x, b = u / p.H_kv, h = u % p.H_kv, tid = threadIdx.x;
   pdl_wait();
   pdl_trigger();
@@ -91,7 +98,10 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
     n_heavy = budget - n_sink - n_recent;
   }
   const size_t base = (size_t)u * p.N_cap;
-  for (int i = tid; i < len; i += blockDim.x) {
+  // Short units need few threads, and every barrier below costs by the warp: the surplus warps leave.
+  const int nthr = min((int)blockDim.x, max(128, ((len + 3) / 4 + 31) & ~31)), nw = nthr >> 5;
+  if (tid >= nthr) return;
+  for (int i = tid; i < len; i += nthr) {
     const float pv = src.votes[base + i], ls = src.lscore[base + i];
     // kappa = ln p + lscore in fp64, rounded once to fp32 (p = 1 needs no logarithm)
     const float kappa = (pv == 1.0f) ? ls : (float)(log((double)pv) + (double)ls);
@@ -100,15 +110,65 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
   __syncthreads();
 
   uint32_t kth = 0;
-  int n_tie = 0;
-  if (n_heavy > 0) {
+  int n_tie = 0, tot_ties = 0;
+  const int m_cand = hi - lo;
+  if (n_heavy > 0 && m_cand <= kWarpSelectMax) {
+    // few candidates (every steady-state compression): warp 0 alone finds the threshold, so the four
+    // digit passes cost no block barrier
+    if (tid < 32) {
+      const int lane = tid;
+      uint32_t prefix = 0, mask = 0;
+      int kr = n_heavy, cnt_last = 0;
+      for (int pass = 3; pass >= 0; --pass) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) hist[8 * lane + j] = 0;
+        __syncwarp();
+        for (int i = lo + lane; i < hi; i += 32) {
+          const uint32_t k = keys[i];
+          if ((k & mask) == prefix) atomicAdd(&hist[(k >> (8 * pass)) & 255u], 1);
+        }
+        __syncwarp();
+        int c[8], sum = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { c[j] = hist[8 * lane + j]; sum += c[j]; }
+        int x = sum;   // becomes the count in bins of lanes >= lane
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int y = __shfl_down_sync(0xffffffffu, x, o);
+          if (lane + o < 32) x += y;
+        }
+        const int above = x - sum;
+        const bool here = above < kr && x >= kr;
+        int cum = above, bin = 0, cnt = 0;
+        bool found = false;
+#pragma unroll
+        for (int j = 7; j >= 0; --j) {
+          if (!found) {
+            if (cum + c[j] >= kr) { bin = j; cnt = c[j]; found = true; }
+            else cum += c[j];
+          }
+        }
+        const int src_lane = __ffs(__ballot_sync(0xffffffffu, here)) - 1;
+        prefix |= (uint32_t)__shfl_sync(0xffffffffu, 8 * lane + bin, src_lane) << (8 * pass);
+        kr = __shfl_sync(0xffffffffu, kr - cum, src_lane);
+        cnt_last = __shfl_sync(0xffffffffu, cnt, src_lane);
+        mask |= 0xFFu << (8 * pass);
+        __syncwarp();
+      }
+      if (lane == 0) { s_prefix = prefix; s_kr = kr; s_cnt = cnt_last; }
+    }
+    __syncthreads();
+    kth = s_prefix;
+    n_tie = s_kr;
+    tot_ties = s_cnt;
+  } else if (n_heavy > 0) {
     uint32_t prefix = 0, mask = 0;
     int kr = n_heavy;
     const int lane = tid & 31;
     for (int pass = 3; pass >= 0; --pass) {
-      if (tid < 256) hist[tid] = 0;
+      for (int i = tid; i < 256; i += nthr) hist[i] = 0;
       __syncthreads();
-      for (int start = lo; start < hi; start += blockDim.x) {
+      for (int start = lo; start < hi; start += nthr) {
         const int i = start + tid;
         const uint32_t k = i < hi ? keys[i] : 0u;
         const bool in = i < hi && (k & mask) == prefix;
@@ -120,61 +180,92 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
       __syncthreads();
       if (tid < 32) {
         // bins are scanned from the top: lane l owns bins 8l..8l+7
-        int c[8], s = 0;
+        int c[8], sum = 0;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) { c[j] = hist[8 * lane + j]; s += c[j]; }
-        int x = s;   // becomes the count in bins of lanes >= lane
+        for (int j = 0; j < 8; ++j) { c[j] = hist[8 * lane + j]; sum += c[j]; }
+        int x = sum;   // becomes the count in bins of lanes >= lane
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
           const int y = __shfl_down_sync(0xffffffffu, x, o);
           if (lane + o < 32) x += y;
         }
-        const int above = x - s;
+        const int above = x - sum;
         if (above < kr && x >= kr) {
-          int cum = above, bin = 0;
+          int cum = above, bin = 0, cnt = 0;
           bool found = false;
 #pragma unroll
           for (int j = 7; j >= 0; --j) {
             if (!found) {
-              if (cum + c[j] >= kr) { bin = j; found = true; }
+              if (cum + c[j] >= kr) { bin = j; cnt = c[j]; found = true; }
               else cum += c[j];
             }
           }
           s_prefix = prefix | ((uint32_t)(8 * lane + bin) << (8 * pass));
           s_kr = kr - cum;
+          s_cnt = cnt;
         }
       }
-      __syncthreads();
+      __syncthreads();   // s_prefix is not written again before the second barrier of the next pass
       prefix = s_prefix;
       kr = s_kr;
       mask |= 0xFFu << (8 * pass);
-      __syncthreads();
     }
-    kth = prefix;   // the n_heavy-th largest key
-    n_tie = kr;     // how many entries equal to it are taken, lowest index first
+    kth = prefix;        // the n_heavy-th largest key
+    n_tie = kr;          // how many entries equal to it are taken, lowest index first
+    tot_ties = s_cnt;    // how many entries equal to it exist (the last pass counted full keys)
   }
 
+  // One ordered pass writes both lists: every thread owns a run of consecutive entries, so one block
+  // scan per sweep gives the slots.  The rank among keys equal to the threshold is needed only if
+  // some of them lose.
+  const bool rank_ties = n_heavy > 0 && n_tie < tot_ties;
+  constexpr int RUN = 4;
   int base_tie = 0, base_keep = 0;
-  for (int start = 0; start < len; start += blockDim.x) {
-    const int i = start + tid;
-    const bool valid = i < len;
-    const uint32_t k = valid ? keys[i] : 0u;
-    const bool in_mid = valid && i >= lo && i < hi;
-    const bool is_tie = in_mid && n_heavy > 0 && k == kth;
-    int tot_tie, tot_keep;
-    const int tie_rank = base_tie + block_excl_count(is_tie, warp_tot, tot_tie);
-    const bool keep = valid && (!in_mid || (n_heavy > 0 && (k > kth || (is_tie && tie_rank < n_tie))));
-    const int slot = base_keep + block_excl_count(keep, warp_tot, tot_keep);
-    if (valid) {
-      if (keep) {
-        ret_idx[base + slot] = i;
-        target[base + i] = -2;
+  for (int start = 0; start < len; start += nthr * RUN) {
+    const int i0 = start + tid * RUN;
+    bool keepf[RUN], tief[RUN];
+    int n_t = 0;
+#pragma unroll
+    for (int r = 0; r < RUN; ++r) {
+      const int i = i0 + r;
+      const bool valid = i < len, in_mid = valid && i >= lo && i < hi;
+      const uint32_t k = valid ? keys[i] : 0u;
+      tief[r] = false;
+      if (!in_mid) {
+        keepf[r] = valid;
       } else {
-        ev_idx[base + (i - slot)] = i;
-        target[base + i] = -1;
+        tief[r] = n_heavy > 0 && k == kth;
+        keepf[r] = n_heavy > 0 && k > kth;   // ties are added below
+        n_t += tief[r] ? 1 : 0;
       }
     }
-    base_tie += tot_tie;
+    if (n_heavy > 0) {
+      int tie_rank = base_tie, tot_tie = 0;
+      if (rank_ties) tie_rank += block_excl_sum(n_t, warp_tot, tot_tie, nw);
+#pragma unroll
+      for (int r = 0; r < RUN; ++r)
+        if (tief[r]) { keepf[r] = !rank_ties || tie_rank < n_tie; ++tie_rank; }
+      base_tie += tot_tie;
+    }
+    int n_k = 0;
+#pragma unroll
+    for (int r = 0; r < RUN; ++r) n_k += keepf[r] ? 1 : 0;
+    int tot_keep;
+    int slot = base_keep + block_excl_sum(n_k, warp_tot, tot_keep, nw);
+#pragma unroll
+    for (int r = 0; r < RUN; ++r) {
+      const int i = i0 + r;
+      if (i < len) {
+        if (keepf[r]) {
+          ret_idx[base + slot] = i;
+          target[base + i] = -2;
+          ++slot;
+        } else {
+          ev_idx[base + (i - slot)] = i;
+          target[base + i] = -1;
+        }
+      }
+    }
     base_keep += tot_keep;
   }
   if (tid == 0) {
@@ -258,7 +349,13 @@ compact_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
 // Rows that need the exact chain are queued and shared out over the warps of the CTA (coalesced row
 // loads into shared memory, the sequential chains on three lanes).  The last CTA of a unit to finish
 // sorts the entries to merge by (slot, position), which makes every group contiguous and ascending.
+template <int D>
+__device__ __forceinline__ void merge_group(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
+                                            const int32_t *__restrict__ ret_idx, const int32_t *__restrict__ ev_idx,
+                                            int32_t *target, const uint32_t *gk, int beg, int n, size_t base, int u,
+                                            keepkv_stats *stats);
 constexpr float kRankEps = 1e-4f;
+constexpr int kMergeInline = 32;   // units with at most this many groups are merged by resolve_kernel itself
 constexpr int kResolveThreads = 512;
 constexpr int kResolveWarps = kResolveThreads / 32;
 
@@ -266,8 +363,8 @@ template <int D>
 __global__ void __launch_bounds__(kResolveThreads)
 resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_t *__restrict__ ev_idx,
                UnitInfo *unit_info, const float4 *__restrict__ nom_v, const int32_t *__restrict__ nom_si,
-               const int32_t *__restrict__ sched, int C_max, int32_t *__restrict__ target, uint32_t *grp_key,
-               int key_stride, int32_t *__restrict__ grp_head, keepkv_stats *stats, int smem_keys) {
+               const int32_t *__restrict__ sched, int C_max, const int32_t *__restrict__ ret_idx, int32_t *target,
+               uint32_t *grp_key, int key_stride, int32_t *grp_head, keepkv_stats *stats, int smem_keys) {
   extern __shared__ uint32_t key_smem[];
   __shared__ float ke_s[kResolveWarps][D];
   __shared__ float kc_s[kResolveWarps][2][D];
@@ -379,17 +476,30 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
     for (int i = tid; i < M; i += kResolveThreads) keys[i] = __ldcg(&gk[i]);
   for (int i = M + tid; i < Mp; i += kResolveThreads) keys[i] = 0xFFFFFFFFu;
   __syncthreads();
-  // bitonic sort, ascending
-  for (int k = 2; k <= Mp; k <<= 1) {
-    for (int jj = k >> 1; jj > 0; jj >>= 1) {
-      for (int i = tid; i < Mp; i += kResolveThreads) {
-        const int ixj = i ^ jj;
-        if (ixj > i) {
-          const uint32_t a = keys[i], b = keys[ixj];
-          if ((a > b) == ((i & k) == 0)) { keys[i] = b; keys[ixj] = a; }
+  if (Mp <= kResolveThreads && keys == key_smem) {
+    // few keys (all distinct): every thread finds the rank of its key by counting, one barrier
+    uint32_t mine = 0xFFFFFFFFu;
+    int rank = 0;
+    if (tid < M) {
+      mine = keys[tid];
+      for (int j = 0; j < M; ++j) rank += keys[j] < mine ? 1 : 0;
+    }
+    __syncthreads();
+    if (tid < M) keys[rank] = mine;
+    __syncthreads();
+  } else {
+    // bitonic sort, ascending
+    for (int k = 2; k <= Mp; k <<= 1) {
+      for (int jj = k >> 1; jj > 0; jj >>= 1) {
+        for (int i = tid; i < Mp; i += kResolveThreads) {
+          const int ixj = i ^ jj;
+          if (ixj > i) {
+            const uint32_t a = keys[i], b = keys[ixj];
+            if ((a > b) == ((i & k) == 0)) { keys[i] = b; keys[ixj] = a; }
+          }
         }
+        __syncthreads();
       }
-      __syncthreads();
     }
   }
   // publish the sorted members and the start of every group
@@ -405,8 +515,16 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
   }
   if (tid == 0) {
     grp_head[base + n_groups] = M;
-    unit_info[u].n_groups = n_groups;
+    unit_info[u].n_groups = n_groups <= kMergeInline ? 0 : n_groups;
     stats[u].n_below_T = ui.n_ev - M;
+  }
+  if (n_groups <= kMergeInline) {
+    // few groups (every steady-state compression): merge them here, one warp per group
+    __syncthreads();   // the keys and group starts written above are visible to the whole CTA
+    for (int g = warp; g < n_groups; g += kResolveWarps) {
+      const int beg = grp_head[base + g], n = grp_head[base + g + 1] - beg;
+      merge_group<D>(p, src, dst, ret_idx, ev_idx, target, gk, beg, n, base, u, stats);
+    }
   }
 }
 
@@ -414,90 +532,120 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
 // One warp per group.  With a_i = ln p_i + lscore_i over the group K'_e (target first, then members
 // ascending):  omega = softmax(a),  v_r = sum omega_i v_i,  k_r = gamma * sum omega_i k_i,
 // gamma = L / lambda_bar,  L = LSE(a) - ln(sum p),  lambda_bar = sum omega_i lscore_i,  p_r = sum p,
-// lscore_r = L   (Eq. A.3 in logarithms).
+// lscore_r = L   (Eq. A.3 in logarithms).  `gk` holds the unit's sorted (slot << 16 | position) keys.
+template <int D>
+__device__ __forceinline__ void merge_group(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
+                                            const int32_t *__restrict__ ret_idx, const int32_t *__restrict__ ev_idx,
+                                            int32_t *target, const uint32_t *gk, int beg, int n, size_t base, int u,
+                                            keepkv_stats *stats) {
+  constexpr int EPL = D / 32;
+  const int lane = threadIdx.x & 31;
+  const float *votes = src.votes + base, *ls = src.lscore + base;
+  const __nv_bfloat16 *sK = reinterpret_cast<const __nv_bfloat16 *>(src.K) + base * D;
+  const __nv_bfloat16 *sV = reinterpret_cast<const __nv_bfloat16 *>(src.V) + base * D;
+  const int c = (int)(gk[beg] >> 16);
+  const int ci = ret_idx[base + c];
+  auto member = [&](int t) { return ev_idx[base + (gk[beg + t] & 0xFFFFu)]; };
+
+  float ka[EPL], va[EPL], lbar = 0.f, L, Ps;
+#pragma unroll
+  for (int e = 0; e < EPL; ++e) { ka[e] = 0.f; va[e] = 0.f; }
+  auto accumulate = [&](int i, float om, float lsi) {
+    lbar = fmaf(om, lsi, lbar);
+    if constexpr (EPL == 4) {
+      const uint2 kk = *reinterpret_cast<const uint2 *>(sK + (size_t)i * D + lane * 4);
+      const uint2 vv = *reinterpret_cast<const uint2 *>(sV + (size_t)i * D + lane * 4);
+      ka[0] = fmaf(om, bf16_lo(kk.x), ka[0]); ka[1] = fmaf(om, bf16_hi(kk.x), ka[1]);
+      ka[2] = fmaf(om, bf16_lo(kk.y), ka[2]); ka[3] = fmaf(om, bf16_hi(kk.y), ka[3]);
+      va[0] = fmaf(om, bf16_lo(vv.x), va[0]); va[1] = fmaf(om, bf16_hi(vv.x), va[1]);
+      va[2] = fmaf(om, bf16_lo(vv.y), va[2]); va[3] = fmaf(om, bf16_hi(vv.y), va[3]);
+    } else {
+      const uint32_t kk = *reinterpret_cast<const uint32_t *>(sK + (size_t)i * D + lane * 2);
+      const uint32_t vv = *reinterpret_cast<const uint32_t *>(sV + (size_t)i * D + lane * 2);
+      ka[0] = fmaf(om, bf16_lo(kk), ka[0]); ka[1] = fmaf(om, bf16_hi(kk), ka[1]);
+      va[0] = fmaf(om, bf16_lo(vv), va[0]); va[1] = fmaf(om, bf16_hi(vv), va[1]);
+    }
+  };
+  if (n < 32) {
+    // the usual case: lane 0 holds the target, lane t the t-th member, so that their votes and scores are
+    // fetched together and the row loads of the accumulation do not wait on one another
+    const int idx = lane == 0 ? ci : (lane <= n ? member(lane - 1) : -1);
+    const float pv = idx >= 0 ? votes[idx] : 0.f, lsv = idx >= 0 ? ls[idx] : 0.f;
+    const float a = idx >= 0 ? logf(pv) + lsv : -CUDART_INF_F;
+    const float M = warp_max(a);
+    const float Z = warp_sum(idx >= 0 ? expf(a - M) : 0.f);
+    Ps = warp_sum(pv);
+    const float Lam = M + logf(Z);
+    L = Lam - logf(Ps);
+    const float om = idx >= 0 ? expf(a - Lam) : 0.f;
+#pragma unroll 4
+    for (int t = 0; t <= n; ++t)
+      accumulate(__shfl_sync(0xffffffffu, idx, t), __shfl_sync(0xffffffffu, om, t), __shfl_sync(0xffffffffu, lsv, t));
+  } else {
+    const float a_c = logf(votes[ci]) + ls[ci];
+    float M = a_c;
+    for (int t = lane; t < n; t += 32) { const int e = member(t); M = fmaxf(M, logf(votes[e]) + ls[e]); }
+    M = warp_max(M);
+    float Z = 0.f;
+    Ps = 0.f;
+    if (lane == 0) { Z = expf(a_c - M); Ps = votes[ci]; }
+    for (int t = lane; t < n; t += 32) { const int e = member(t); Z += expf(logf(votes[e]) + ls[e] - M); Ps += votes[e]; }
+    Z = warp_sum(Z);
+    Ps = warp_sum(Ps);
+    const float Lam = M + logf(Z);
+    L = Lam - logf(Ps);
+    for (int t = -1; t < n; ++t) {
+      const int i = t < 0 ? ci : member(t);
+      const float lsi = ls[i];
+      accumulate(i, expf(logf(votes[i]) + lsi - Lam), lsi);
+    }
+  }
+  const float gamma = L / lbar;
+  const bool ok = gamma > p.gamma_min && gamma <= p.gamma_max && fabsf(lbar) >= 1e-6f;
+  if (!ok) {
+    // guard: the members are dropped after all and the target keeps the row copied by compaction
+    for (int t = lane; t < n; t += 32) target[base + member(t)] = -1;
+    if (lane == 0) { atomicAdd(&stats[u].n_guard_groups, 1); atomicAdd(&stats[u].n_groups, 1); }
+    return;
+  }
+  __nv_bfloat16 *dK = reinterpret_cast<__nv_bfloat16 *>(dst.K) + (base + c) * D;
+  __nv_bfloat16 *dV = reinterpret_cast<__nv_bfloat16 *>(dst.V) + (base + c) * D;
+  if constexpr (EPL == 4) {
+    uint2 ko, vo;
+    ko.x = pack_bf16(gamma * ka[0], gamma * ka[1]); ko.y = pack_bf16(gamma * ka[2], gamma * ka[3]);
+    vo.x = pack_bf16(va[0], va[1]); vo.y = pack_bf16(va[2], va[3]);
+    *reinterpret_cast<uint2 *>(dK + lane * 4) = ko;
+    *reinterpret_cast<uint2 *>(dV + lane * 4) = vo;
+  } else {
+    *reinterpret_cast<uint32_t *>(dK + lane * 2) = pack_bf16(gamma * ka[0], gamma * ka[1]);
+    *reinterpret_cast<uint32_t *>(dV + lane * 2) = pack_bf16(va[0], va[1]);
+  }
+  if (lane == 0) {
+    dst.votes[base + c] = Ps;
+    dst.lscore[base + c] = L;
+    atomicAdd(&stats[u].n_merged, n);
+    atomicAdd(&stats[u].n_groups, 1);
+    atomicMax(&stats[u].max_group, n);
+  }
+}
+
+// Units with many groups (the first compression of a long prompt): warps of several CTAs share them.
+// Units with few groups were already merged by resolve_kernel, which left n_groups = 0 here.
 template <int D>
 __global__ void __launch_bounds__(256)
 merge_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_t *__restrict__ ret_idx,
              const int32_t *__restrict__ ev_idx, int32_t *target, const UnitInfo *__restrict__ unit_info,
              const uint32_t *__restrict__ grp_key, int key_stride, const int32_t *__restrict__ grp_head,
              keepkv_stats *stats) {
-  constexpr int EPL = D / 32;
-  const int u = blockIdx.y, lane = threadIdx.x & 31;
+  const int u = blockIdx.y;
   pdl_wait();
   pdl_trigger();
   const UnitInfo ui = unit_info[u];
   const size_t base = (size_t)u * p.N_cap;
   const uint32_t *gk = grp_key + (size_t)u * key_stride;
-  const float *votes = src.votes + base, *ls = src.lscore + base;
-  const __nv_bfloat16 *sK = reinterpret_cast<const __nv_bfloat16 *>(src.K) + base * D;
-  const __nv_bfloat16 *sV = reinterpret_cast<const __nv_bfloat16 *>(src.V) + base * D;
   for (int g = blockIdx.x * 8 + (threadIdx.x >> 5); g < ui.n_groups; g += gridDim.x * 8) {
     const int beg = grp_head[base + g], n = grp_head[base + g + 1] - beg;
-    const int c = (int)(gk[beg] >> 16);
-    const int ci = ret_idx[base + c];
-    auto member = [&](int t) { return ev_idx[base + (gk[beg + t] & 0xFFFFu)]; };
-
-    const float a_c = logf(votes[ci]) + ls[ci];
-    float M = a_c;
-    for (int t = lane; t < n; t += 32) { const int e = member(t); M = fmaxf(M, logf(votes[e]) + ls[e]); }
-    M = warp_max(M);
-    float Z = 0.f, Ps = 0.f;
-    if (lane == 0) { Z = expf(a_c - M); Ps = votes[ci]; }
-    for (int t = lane; t < n; t += 32) { const int e = member(t); Z += expf(logf(votes[e]) + ls[e] - M); Ps += votes[e]; }
-    Z = warp_sum(Z);
-    Ps = warp_sum(Ps);
-    const float Lam = M + logf(Z);
-    const float L = Lam - logf(Ps);
-
-    float ka[EPL], va[EPL], lbar = 0.f;
-#pragma unroll
-    for (int e = 0; e < EPL; ++e) { ka[e] = 0.f; va[e] = 0.f; }
-    for (int t = -1; t < n; ++t) {
-      const int i = t < 0 ? ci : member(t);
-      const float lsi = ls[i];
-      const float om = expf(logf(votes[i]) + lsi - Lam);
-      lbar = fmaf(om, lsi, lbar);
-      if constexpr (EPL == 4) {
-        const uint2 kk = *reinterpret_cast<const uint2 *>(sK + (size_t)i * D + lane * 4);
-        const uint2 vv = *reinterpret_cast<const uint2 *>(sV + (size_t)i * D + lane * 4);
-        ka[0] = fmaf(om, bf16_lo(kk.x), ka[0]); ka[1] = fmaf(om, bf16_hi(kk.x), ka[1]);
-        ka[2] = fmaf(om, bf16_lo(kk.y), ka[2]); ka[3] = fmaf(om, bf16_hi(kk.y), ka[3]);
-        va[0] = fmaf(om, bf16_lo(vv.x), va[0]); va[1] = fmaf(om, bf16_hi(vv.x), va[1]);
-        va[2] = fmaf(om, bf16_lo(vv.y), va[2]); va[3] = fmaf(om, bf16_hi(vv.y), va[3]);
-      } else {
-        const uint32_t kk = *reinterpret_cast<const uint32_t *>(sK + (size_t)i * D + lane * 2);
-        const uint32_t vv = *reinterpret_cast<const uint32_t *>(sV + (size_t)i * D + lane * 2);
-        ka[0] = fmaf(om, bf16_lo(kk), ka[0]); ka[1] = fmaf(om, bf16_hi(kk), ka[1]);
-        va[0] = fmaf(om, bf16_lo(vv), va[0]); va[1] = fmaf(om, bf16_hi(vv), va[1]);
-      }
-    }
-    const float gamma = L / lbar;
-    const bool ok = gamma > p.gamma_min && gamma <= p.gamma_max && fabsf(lbar) >= 1e-6f;
-    if (!ok) {
-      // guard: the members are dropped after all and the target keeps the row copied by compaction
-      for (int t = lane; t < n; t += 32) target[base + member(t)] = -1;
-      if (lane == 0) { atomicAdd(&stats[u].n_guard_groups, 1); atomicAdd(&stats[u].n_groups, 1); }
-      continue;
-    }
-    __nv_bfloat16 *dK = reinterpret_cast<__nv_bfloat16 *>(dst.K) + (base + c) * D;
-    __nv_bfloat16 *dV = reinterpret_cast<__nv_bfloat16 *>(dst.V) + (base + c) * D;
-    if constexpr (EPL == 4) {
-      uint2 ko, vo;
-      ko.x = pack_bf16(gamma * ka[0], gamma * ka[1]); ko.y = pack_bf16(gamma * ka[2], gamma * ka[3]);
-      vo.x = pack_bf16(va[0], va[1]); vo.y = pack_bf16(va[2], va[3]);
-      *reinterpret_cast<uint2 *>(dK + lane * 4) = ko;
-      *reinterpret_cast<uint2 *>(dV + lane * 4) = vo;
-    } else {
-      *reinterpret_cast<uint32_t *>(dK + lane * 2) = pack_bf16(gamma * ka[0], gamma * ka[1]);
-      *reinterpret_cast<uint32_t *>(dV + lane * 2) = pack_bf16(va[0], va[1]);
-    }
-    if (lane == 0) {
-      dst.votes[base + c] = Ps;
-      dst.lscore[base + c] = L;
-      atomicAdd(&stats[u].n_merged, n);
-      atomicAdd(&stats[u].n_groups, 1);
-      atomicMax(&stats[u].max_group, n);
-    }
+    merge_group<D>(p, src, dst, ret_idx, ev_idx, target, gk, beg, n, base, u, stats);
   }
 }
 
@@ -538,8 +686,8 @@ static void launch_compress_t(const keepkv_params &p, const keepkv_cache &src, c
   KEEPKV_CHECK_LAUNCH(ctx);
   launch_nominate(p, src, dst, ev_idx, ui, inv_norm, sched, nom_v, nom_si, L.nom_chunks, status_dev, ctx);
   launch_pdl(resolve_kernel<D>, dim3(L.nom_chunks, U), dim3(kResolveThreads), (size_t)smem_keys * 4, ctx.stream,
-      p, src, dst, ev_idx, ui, nom_v, nom_si, sched, L.nom_chunks, target, grp_key, L.key_stride, grp_head, stats,
-      smem_keys);
+      p, src, dst, ev_idx, ui, nom_v, nom_si, sched, L.nom_chunks, ret_idx, target, grp_key, L.key_stride, grp_head,
+      stats, smem_keys);
   KEEPKV_CHECK_LAUNCH(ctx);
   int gx = 4096 / U;
   gx = gx < 1 ? 1 : (gx > 32 ? 32 : gx);

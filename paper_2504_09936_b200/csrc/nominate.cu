@@ -165,7 +165,9 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
 
   const uint32_t tmem = s_tmem;
   const int total_m = prefix[U];
-  int C = total_m > 0 ? (2 * (int)gridDim.x + total_m - 1) / total_m : 1;
+  // few row tiles: split every row's columns into chunks so that all SMs get one item (a second wave
+  // of items would cost more in fixed latency than the shorter items save)
+  int C = total_m > 0 ? (int)gridDim.x / total_m : 1;
   C = max(1, min(C, C_max));
   const int n_items = total_m * C;
   if (blockIdx.x == 0 && tid == 0) sched[0] = C;
