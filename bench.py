@@ -191,6 +191,12 @@ def run_ours(args, w, rank, world):
 
     # inputs: one seeded prompt cache (per rank its own seed offset), replicated into L distinct buffers
     Kb, Vb, lens = W.make_cache(w, layer=rank, n_cap=n_cap)
+    # budgets follow each sequence's own prompt length (they differ only for the ragged workload)
+    bud = np.array([w.budget(int(n)) for n in lens], dtype=np.int32)
+    nrec = np.array([w.n_recent(int(x)) for x in bud], dtype=np.int32)
+    ragged = bool(np.any(bud != bud[0]))
+    budget_arg = torch.from_numpy(bud).cuda() if ragged else b
+    nrec_arg = torch.from_numpy(nrec).cuda() if ragged else None
     K0, V0 = dev(Kb).view(w.B, w.H_kv, n_cap, w.d), dev(Vb).view(w.B, w.H_kv, n_cap, w.d)
     del Kb, Vb
     A = [kb.Cache(K0.clone(), V0.clone(), torch.ones(w.B, w.H_kv, n_cap, device="cuda"),
@@ -235,7 +241,7 @@ def run_ours(args, w, rank, world):
         stats = torch.zeros(L, w.U, 8, dtype=torch.int32, device="cuda")
         e0.record()
         for l in range(L):
-            kb.keepkv_compress(p, A[l], Bc[l], b, ws, st, stats=stats[l])
+            kb.keepkv_compress(p, A[l], Bc[l], budget_arg, ws, st, n_recent_dev=nrec_arg, stats=stats[l])
         e1.record(); stream.synchronize()
         t_full_compress = e0.elapsed_time(e1) * 1e-3 / L
         m_full = float(stats[:, :, 2].sum().item()) / (L * w.U)
@@ -250,7 +256,8 @@ def run_ours(args, w, rank, world):
                     kb.keepkv_decode_attention(p, cur[l], q_all[t + 1], out, None, True, ws, st)
                     n += 2
             for l in range(L):
-                kb.keepkv_compress(p, cur[l], oth[l], b, ws, st, stats=None if stats_t is None else stats_t[l])
+                kb.keepkv_compress(p, cur[l], oth[l], budget_arg, ws, st, n_recent_dev=nrec_arg,
+                                   stats=None if stats_t is None else stats_t[l])
                 n += compress_launches
             return n
 
@@ -310,7 +317,7 @@ def run_ours(args, w, rank, world):
         stream.synchronize()
         with torch.cuda.graph(gc, stream=stream):
             for l in range(L):
-                kb.keepkv_compress(p, cur[l], oth[l], b, ws, st, stats=stats[l])
+                kb.keepkv_compress(p, cur[l], oth[l], budget_arg, ws, st, n_recent_dev=nrec_arg, stats=stats[l])
         gc.replay(); stream.synchronize()
         e0.record(); gc.replay(); gc.replay(); e1.record(); stream.synchronize()
         t_inc_compress = e0.elapsed_time(e1) * 1e-3 / (2 * L)
@@ -332,7 +339,7 @@ def run_ours(args, w, rank, world):
                     kb.keepkv_decode_step_host(p, cur[l], qh[i], knh[i], vnh[i], oh, qd, kd, vd, out, True, ws, st)
                 stream.synchronize()          # the next token's queries depend on this step's output
             for l in range(L):
-                kb.keepkv_compress(p, cur[l], oth[l], b, ws, st)
+                kb.keepkv_compress(p, cur[l], oth[l], budget_arg, ws, st, n_recent_dev=nrec_arg)
 
         pair = [(cur, oth), (oth, cur)]
         period_e2e(*pair[0]); period_e2e(*pair[1])
@@ -355,11 +362,19 @@ def run_ours(args, w, rank, world):
     value = tokens_per_step * args.steps / t_steps
     e2e_val = tokens_per_step / t_e2e
     hbm, src = peaks()
-    entries = w.U * (b + P // 2)
+    bud64 = bud.astype(np.int64)
+    entries = int((bud64 + P // 2).sum()) * w.H_kv
     ach = decode_bytes(w, entries) / t_decode / 1e9
     full_dec_gbs = decode_bytes(w, int(lens.astype(np.int64).sum()) * w.H_kv) / t_full_decode / 1e9
-    inc_gbs = compress_bytes(w, b + P, b, m_inc) / t_inc_compress / 1e9
-    full_gbs = compress_bytes(w, w.N, b, m_full) / t_full_compress / 1e9
+
+    def cbytes(len_b, m_per_unit):   # algorithmic bytes of one compression, summed over the units
+        per_seq = len_b * 2 * w.d + (bud64 + m_per_unit) * 2 * w.d + len_b * 8 + bud64 * (4 * w.d + 8)
+        return float(per_seq.sum()) * w.H_kv
+
+    inc_bytes, full_bytes = cbytes(bud64 + P, m_inc), cbytes(lens.astype(np.int64), m_full)
+    inc_gbs = inc_bytes / t_inc_compress / 1e9
+    full_gbs = full_bytes / t_full_compress / 1e9
+    gemm_flops = float((2.0 * (lens.astype(np.int64) - bud64) * bud64 * w.d).sum()) * w.H_kv
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": t_steps / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -382,7 +397,7 @@ def run_ours(args, w, rank, world):
             "compress_incremental_frac_hbm": inc_gbs / hbm, "merged_per_unit_incremental": m_inc,
             "compress_full_us": t_full_compress * 1e6, "compress_full_gbs": full_gbs,
             "compress_full_frac_hbm": full_gbs / hbm, "merged_per_unit_full": m_full,
-            "compress_full_gemm_tflops": 2.0 * (w.N - b) * b * w.d * w.U / t_full_compress / 1e12,
+            "compress_full_gemm_tflops": gemm_flops / t_full_compress / 1e12,
         },
     }
     if rank == 0:

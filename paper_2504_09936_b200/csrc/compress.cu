@@ -677,7 +677,7 @@ static void launch_compress_t(const keepkv_params &p, const keepkv_cache &src, c
     cudaFuncSetAttribute(resolve_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
     attr_done = true;
   }
-  launch_pdl(select_kernel, dim3(U), dim3(1024), sel_smem, ctx.stream, p, src, dst.seq_len, budget_dev, budget_scalar,
+  launch_pdl(select_kernel, dim3(U), dim3(512), sel_smem, ctx.stream, p, src, dst.seq_len, budget_dev, budget_scalar,
              n_recent_dev, ret_idx, target, ev_idx, ui, stats);
   KEEPKV_CHECK_LAUNCH(ctx);
   if (ret_bound <= 0) return;   // nothing is kept: every entry is dropped, which select has recorded

@@ -33,7 +33,7 @@ struct NomSmem {
   static constexpr int kABytes = kSub * kNomM * 128;
   static constexpr int kBBytes = kSub * kNomN * 128;
   static constexpr int kA = 0;
-  static constexpr int kB = kABytes;
+  static constexpr int kB = 2 * kABytes;                  // two A tiles: the next item is gathered while this one is drained
   static constexpr int kInv = kB + kNomStages * kBBytes;  // f32 [8 warps][128]   inverse norms of the warp's columns
   static constexpr int kRowInv = kInv + 8 * 128 * 4;      // f32 [2][128]         inverse norms of the staged rows
   static constexpr int kXchg = kRowInv + 2 * 128 * 4;     // u32 [2][128][5]      column-half exchange
@@ -108,24 +108,24 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
   constexpr int KSTEPS = D / 16;
   constexpr uint32_t IDESC = umma_idesc_bf16(kNomM, kNomN);
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[10];   // a_ready, b_full[2], b_empty[2], t_full[2], t_empty[2], drain
+  __shared__ __align__(8) uint64_t bars[11];   // a_ready[2], b_full[2], b_empty[2], t_full[2], t_empty[2], drain
   __shared__ uint32_t s_tmem;
   __shared__ volatile int s_abort;
 
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sbase = smem_u32(smem);
   const uint32_t bar_a_ready = smem_u32(&bars[0]);
-  const uint32_t bar_b_full = smem_u32(&bars[1]), bar_b_empty = smem_u32(&bars[3]);
-  const uint32_t bar_t_full = smem_u32(&bars[5]), bar_t_empty = smem_u32(&bars[7]);
-  const uint32_t bar_drain = smem_u32(&bars[9]);
+  const uint32_t bar_b_full = smem_u32(&bars[2]), bar_b_empty = smem_u32(&bars[4]);
+  const uint32_t bar_t_full = smem_u32(&bars[6]), bar_t_empty = smem_u32(&bars[8]);
+  const uint32_t bar_drain = smem_u32(&bars[10]);
   int *prefix = reinterpret_cast<int *>(smem + SL::kPrefix);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int U = p.B * p.H_kv;
 
   if (tid == 0) {
-    mbar_init(bar_a_ready, 8);
     for (int i = 0; i < 2; ++i) {
+      mbar_init(bar_a_ready + 8 * i, 8);
       mbar_init(bar_b_full + 8 * i, 1);
       mbar_init(bar_b_empty + 8 * i, 1);
       mbar_init(bar_t_full + 8 * i, 1);
@@ -197,7 +197,8 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
       for (int item = blockIdx.x; item < n_items && !s_abort; item += gridDim.x) {
         const NomItem it = nom_item(item, C, prefix, U, unit_info);
         if (it.t0 == it.t1) continue;
-        if (!mbar_wait(bar_a_ready, n_done & 1)) { s_abort = 1; break; }
+        const int abuf = n_done & 1;
+        if (!mbar_wait(bar_a_ready + 8 * abuf, (n_done >> 1) & 1)) { s_abort = 1; break; }
         ++n_done;
         tc_fence_after();
         for (int t = it.t0; t < it.t1; ++t, ++ring, ++acc) {
@@ -205,7 +206,7 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
           if (!mbar_wait(bar_b_full + 8 * s, (ring >> 1) & 1) ||
               !mbar_wait(bar_t_empty + 8 * a, ((acc >> 1) & 1) ^ 1)) { s_abort = 1; break; }
           tc_fence_after();
-          const uint32_t a_base = sbase + SL::kA, b_base = sbase + SL::kB + s * SL::kBBytes;
+          const uint32_t a_base = sbase + SL::kA + abuf * SL::kABytes, b_base = sbase + SL::kB + s * SL::kBBytes;
 #pragma unroll
           for (int k = 0; k < KSTEPS; ++k) {
             const uint64_t ad = umma_desc_sw128(a_base + (k >> 2) * (kNomM * 128) + (k & 3) * 32);
@@ -228,7 +229,46 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
     uint32_t *xchg = reinterpret_cast<uint32_t *>(smem + SL::kXchg);
     const size_t n_total = (size_t)U * p.N_cap;
     int acc = 0, n_done = 0;
-    bool dead = false;
+    bool dead = false, staged = false;
+    // Gathers the 128 evicted rows of an item into swizzled A tile `abuf`, sixteen lanes per row, and
+    // leaves the rows' inverse norms in rowinv[abuf].
+    auto stage_rows = [&](const NomItem &si, int abuf) {
+      constexpr int REPS = kNomM / 16;
+      const size_t sbase_u = (size_t)si.u * p.N_cap;
+      const int sm0 = si.m_tile * kNomM;
+      const int ch = lane & 15, rsub = ew * 2 + (lane >> 4);
+      int esrc[REPS];
+      uint4 val[REPS];
+#pragma unroll
+      for (int rep = 0; rep < REPS; ++rep) {
+        const int r = rep * 16 + rsub;
+        esrc[rep] = (ch < D / 8 && sm0 + r < si.n_ev) ? ev_idx[sbase_u + sm0 + r] : -1;
+      }
+#pragma unroll
+      for (int rep = 0; rep < REPS; ++rep) {
+        val[rep] = make_uint4(0, 0, 0, 0);
+        if (esrc[rep] >= 0) val[rep] = *reinterpret_cast<const uint4 *>(srcK + (sbase_u + esrc[rep]) * D + ch * 8);
+      }
+#pragma unroll
+      for (int rep = 0; rep < REPS; ++rep) {
+        const int r = rep * 16 + rsub;
+        float ss = 0.f;
+        const uint32_t w[4] = {val[rep].x, val[rep].y, val[rep].z, val[rep].w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { const float a = bf16_lo(w[q]), b = bf16_hi(w[q]); ss = fmaf(a, a, ss); ss = fmaf(b, b, ss); }
+        ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+        ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+        ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+        ss += __shfl_xor_sync(0xffffffffu, ss, 8);
+        if (ch < D / 8)
+          *reinterpret_cast<uint4 *>(smem + SL::kA + abuf * SL::kABytes + (ch >> 3) * (kNomM * 128) + r * 128 +
+                                     (((ch & 7) ^ (r & 7)) << 4)) = val[rep];
+        if (ch == 0) rowinv[abuf * 128 + r] = rsqrtf(ss);
+      }
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_a_ready + 8 * abuf);
+    };
     for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
       const NomItem it = nom_item(item, C, prefix, U, unit_info);
       const size_t ubase = (size_t)it.u * p.N_cap;
@@ -246,41 +286,24 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
       }
       dead = __any_sync(0xffffffffu, dead || s_abort != 0);
       {
-        // ---- gather the evicted rows into the swizzled A tile (the previous item's MMAs have retired:
-        //      this warp has seen the barrier of that item's last accumulator).  Sixteen lanes per row.
-        constexpr int REPS = kNomM / 16;
-        const int ch = lane & 15, rsub = ew * 2 + (lane >> 4);
-        int esrc[REPS];
-        uint4 val[REPS];
-#pragma unroll
-        for (int rep = 0; rep < REPS; ++rep) {
-          const int r = rep * 16 + rsub;
-          esrc[rep] = (ch < D / 8 && m0 + r < it.n_ev) ? ev_idx[ubase + m0 + r] : -1;
+        if (!staged) {   // the first item of this CTA; every later one was gathered while its predecessor was drained
+          stage_rows(it, buf);
+          staged = true;
         }
-#pragma unroll
-        for (int rep = 0; rep < REPS; ++rep) {
-          val[rep] = make_uint4(0, 0, 0, 0);
-          if (esrc[rep] >= 0) val[rep] = *reinterpret_cast<const uint4 *>(srcK + (ubase + esrc[rep]) * D + ch * 8);
+        // rowinv of this item is visible to every warp, and nobody still reads the other buffer's
+        // rowinv (the previous item's results have been published)
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        // gather the next item's rows into the other A tile now, so that its MMAs can start while this
+        // item is drained (the MMAs that last read that tile belong to the item before this one: retired)
+        {
+          int nx = item + gridDim.x;
+          NomItem nit;
+          for (; nx < n_items; nx += gridDim.x) {
+            nit = nom_item(nx, C, prefix, U, unit_info);
+            if (nit.t0 < nit.t1) break;
+          }
+          if (nx < n_items) stage_rows(nit, buf ^ 1);
         }
-#pragma unroll
-        for (int rep = 0; rep < REPS; ++rep) {
-          const int r = rep * 16 + rsub;
-          float ss = 0.f;
-          const uint32_t w[4] = {val[rep].x, val[rep].y, val[rep].z, val[rep].w};
-#pragma unroll
-          for (int q = 0; q < 4; ++q) { const float a = bf16_lo(w[q]), b = bf16_hi(w[q]); ss = fmaf(a, a, ss); ss = fmaf(b, b, ss); }
-          ss += __shfl_xor_sync(0xffffffffu, ss, 1);
-          ss += __shfl_xor_sync(0xffffffffu, ss, 2);
-          ss += __shfl_xor_sync(0xffffffffu, ss, 4);
-          ss += __shfl_xor_sync(0xffffffffu, ss, 8);
-          if (ch < D / 8)
-            *reinterpret_cast<uint4 *>(smem + SL::kA + (ch >> 3) * (kNomM * 128) + r * 128 + (((ch & 7) ^ (r & 7)) << 4)) = val[rep];
-          if (ch == 0) rowinv[buf * 128 + r] = rsqrtf(ss);
-        }
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar_a_ready);
-        asm volatile("bar.sync 1, 256;" ::: "memory");   // rowinv of every row is visible
         // values are compared before the division by |k_e|: the closeness margin scales with it
         top.init(2.f * kNomRankEps / rowinv[buf * 128 + row]);
 
