@@ -323,7 +323,14 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
             if (lane == 0) ok = mbar_wait(bar_t_full + 8 * a, (acc >> 1) & 1);
             if (!__shfl_sync(0xffffffffu, ok, 0)) { dead = true; s_abort = 1; }
           }
-          if (!dead) {
+          // nothing to track if this warp's 32 rows lie past the evicted entries or its columns past the
+          // retained ones: release the accumulator without reading it
+          const bool live = m0 + quarter * 32 < it.n_ev && c0 < it.n_ret;
+          if (!dead && !live) {
+            tc_fence_before();
+            if (lane == 0) mbar_arrive(bar_t_empty + 8 * a);
+          }
+          if (!dead && live) {
             tc_fence_after();
             const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + a * kNomN + half * 128;
             const int n_valid = it.n_ret - c0;   // columns of this half that exist
