@@ -398,7 +398,7 @@ def run_ours(args, w, rank, world):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": t_steps / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 storage, fp32 accumulate", "data": "synthetic",
+        "dtype": "bf16", "data": "synthetic",
         "config": config_dict(w, args, f"each call works on one of {L} distinct layer caches visited round-robin "
                                        f"({L} x {decode_bytes(w, entries) / 1e6:.0f} MB > 126 MB L2)"),
         "clocks": clocks, "gpu_launches": launches,

@@ -16,6 +16,8 @@
 //               scaling by the retained keys' inverse norms and tracking the row's top two.
 // Every wait is bounded; a wait that runs out raises KEEPKV_DEV_TIMEOUT, the CTA stops issuing work,
 // drains what is in flight, frees its tensor memory and returns.
+#include <type_traits>
+
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -64,17 +66,35 @@ struct Top2 {
     bi = p1 ? idx : bi;
     best = fmaxf(best, v);
   }
-  // a_i: accumulators, w_i: inverse norms of the four columns idx..idx+3
-  __device__ __forceinline__ void offer4(float a0, float a1, float a2, float a3, const float4 w, int idx) {
-    const float ncut = -cut;
-    const uint32_t s = __float_as_uint(fmaf(a0, w.x, ncut)) & __float_as_uint(fmaf(a1, w.y, ncut)) &
-                       __float_as_uint(fmaf(a2, w.z, ncut)) & __float_as_uint(fmaf(a3, w.w, ncut));
-    if (__any_sync(0xffffffffu, (int)s >= 0)) {   // some lane has a value that is not below its cut
-      insert(a0 * w.x, idx); insert(a1 * w.y, idx + 1); insert(a2 * w.z, idx + 2); insert(a3 * w.w, idx + 3);
-      cut = best - thr;
-    }
+  // Insert for candidates that arrive out of slot order (the other tracker of the thread): equal values
+  // go to the lower slot, as if the columns had been scanned in order.
+  __device__ __forceinline__ void insert_any(float v, int idx) {
+    const bool p1 = v > best || (v == best && idx < bi), p2 = v > second || (v == second && idx < si);
+    second = p1 ? best : (p2 ? v : second);
+    si = p1 ? bi : (p2 ? idx : si);
+    bi = p1 ? idx : bi;
+    best = p1 ? v : best;
   }
 };
+
+// Two trackers per thread, one for the even and one for the odd columns, so that the select chains of
+// neighbouring columns do not wait on each other; both share the lower of their cuts (kept in ta.cut).
+// a_i: accumulators, w_i: inverse norms of the four columns idx..idx+3.
+// TEST = false (the first tile of an item, where nearly every group holds a new candidate for some row):
+// all four columns are inserted without the skip test, so nothing but the select chains is on the
+// critical path.
+template <bool TEST>
+__device__ __forceinline__ void offer4(Top2 &ta, Top2 &tb, float a0, float a1, float a2, float a3, const float4 w,
+                                       int idx) {
+  if (TEST) {
+    const float ncut = -ta.cut;
+    const uint32_t s = __float_as_uint(fmaf(a0, w.x, ncut)) & __float_as_uint(fmaf(a1, w.y, ncut)) &
+                       __float_as_uint(fmaf(a2, w.z, ncut)) & __float_as_uint(fmaf(a3, w.w, ncut));
+    if (!__any_sync(0xffffffffu, (int)s >= 0)) return;   // no lane has a value that is not below its cut
+  }
+  ta.insert(a0 * w.x, idx); tb.insert(a1 * w.y, idx + 1); ta.insert(a2 * w.z, idx + 2); tb.insert(a3 * w.w, idx + 3);
+  if (TEST) ta.cut = fminf(ta.best, tb.best) - ta.thr;
+}
 
 struct NomItem { int u, m_tile, chunk, t0, t1, n_ev, n_ret; };
 
@@ -110,6 +130,7 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t bars[11];   // a_ready[2], b_full[2], b_empty[2], t_full[2], t_empty[2], drain
   __shared__ uint32_t s_tmem;
+  __shared__ int s_wtot[kNomThreads / 32];
   __shared__ volatile int s_abort;
 
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -143,10 +164,10 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
   }
   pdl_wait();      // barrier set-up and tensor-memory allocation overlap the previous kernel's tail
   pdl_trigger();
-  if (warp == 2) {   // exclusive prefix of 128-row tiles over the units
+  {   // exclusive prefix of 128-row tiles over the units: one unit per thread and pass
     int run = 0;
-    for (int u0 = 0; u0 < U; u0 += 32) {
-      const int u = u0 + lane;
+    for (int u0 = 0; u0 < U; u0 += kNomThreads) {
+      const int u = u0 + tid;
       const int t = u < U ? (unit_info[u].n_ev + kNomM - 1) / kNomM : 0;
       int x = t;
 #pragma unroll
@@ -154,10 +175,20 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
         const int y = __shfl_up_sync(0xffffffffu, x, o);
         if (lane >= o) x += y;
       }
-      if (u < U) prefix[u] = run + x - t;
-      run += __shfl_sync(0xffffffffu, x, 31);
+      if (lane == 31) s_wtot[warp] = x;
+      __syncthreads();
+      int off = 0, tot = 0;
+#pragma unroll
+      for (int w = 0; w < kNomThreads / 32; ++w) {
+        const int v = s_wtot[w];
+        off += w < warp ? v : 0;
+        tot += v;
+      }
+      if (u < U) prefix[u] = run + off + x - t;
+      run += tot;
+      __syncthreads();
     }
-    if (lane == 0) prefix[U] = run;
+    if (tid == 0) prefix[U] = run;
   }
   tc_fence_before();
   __syncthreads();
@@ -274,7 +305,7 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
       const size_t ubase = (size_t)it.u * p.N_cap;
       const int m0 = it.m_tile * kNomM;
       const int buf = n_done & 1;
-      Top2 top;
+      Top2 top, topb;   // two trackers over alternate groups of four columns: two independent dependency chains
       top.init(0.f);
       if (it.t0 == it.t1) {   // a chunk without tiles (fewer tiles than chunks): publish an empty result
         if (half == 0 && m0 + row < it.n_ev) {
@@ -306,6 +337,7 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
         }
         // values are compared before the division by |k_e|: the closeness margin scales with it
         top.init(2.f * kNomRankEps / rowinv[buf * 128 + row]);
+        topb.init(top.thr);
 
         for (int t = it.t0; t < it.t1; ++t, ++acc) {
           const int a = acc & 1;
@@ -346,37 +378,36 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
               }
               const int cb = jg * 64;
               const bool ragged = n_valid < cb + 64;   // columns past n_ret hold other rows' data
+              auto drain32 = [&](auto test, const uint32_t (&r)[32], int off) {
 #pragma unroll
-              for (int i = 0; i < 32; i += 4) {
-                float4 iv = *reinterpret_cast<const float4 *>(inv_w + cb + i);
-                float a0 = __uint_as_float(r0[i]), a1 = __uint_as_float(r0[i + 1]);
-                float a2 = __uint_as_float(r0[i + 2]), a3 = __uint_as_float(r0[i + 3]);
-                if (ragged) {   // a masked column contributes -inf
-                  if (cb + i >= n_valid) { a0 = -CUDART_INF_F; iv.x = 1.f; }
-                  if (cb + i + 1 >= n_valid) { a1 = -CUDART_INF_F; iv.y = 1.f; }
-                  if (cb + i + 2 >= n_valid) { a2 = -CUDART_INF_F; iv.z = 1.f; }
-                  if (cb + i + 3 >= n_valid) { a3 = -CUDART_INF_F; iv.w = 1.f; }
+                for (int i = 0; i < 32; i += 4) {
+                  float4 iv = *reinterpret_cast<const float4 *>(inv_w + off + i);
+                  float a0 = __uint_as_float(r[i]), a1 = __uint_as_float(r[i + 1]);
+                  float a2 = __uint_as_float(r[i + 2]), a3 = __uint_as_float(r[i + 3]);
+                  if (ragged) {   // a masked column contributes -inf
+                    if (off + i >= n_valid) { a0 = -CUDART_INF_F; iv.x = 1.f; }
+                    if (off + i + 1 >= n_valid) { a1 = -CUDART_INF_F; iv.y = 1.f; }
+                    if (off + i + 2 >= n_valid) { a2 = -CUDART_INF_F; iv.z = 1.f; }
+                    if (off + i + 3 >= n_valid) { a3 = -CUDART_INF_F; iv.w = 1.f; }
+                  }
+                  offer4<decltype(test)::value>(top, topb, a0, a1, a2, a3, iv, c0 + off + i);
                 }
-                top.offer4(a0, a1, a2, a3, iv, c0 + cb + i);
-              }
-#pragma unroll
-              for (int i = 0; i < 32; i += 4) {
-                float4 iv = *reinterpret_cast<const float4 *>(inv_w + cb + 32 + i);
-                float a0 = __uint_as_float(r1[i]), a1 = __uint_as_float(r1[i + 1]);
-                float a2 = __uint_as_float(r1[i + 2]), a3 = __uint_as_float(r1[i + 3]);
-                if (ragged) {
-                  if (cb + 32 + i >= n_valid) { a0 = -CUDART_INF_F; iv.x = 1.f; }
-                  if (cb + 33 + i >= n_valid) { a1 = -CUDART_INF_F; iv.y = 1.f; }
-                  if (cb + 34 + i >= n_valid) { a2 = -CUDART_INF_F; iv.z = 1.f; }
-                  if (cb + 35 + i >= n_valid) { a3 = -CUDART_INF_F; iv.w = 1.f; }
-                }
-                top.offer4(a0, a1, a2, a3, iv, c0 + cb + 32 + i);
+              };
+              if (t == it.t0) {   // cold trackers: insert everything
+                drain32(std::false_type{}, r0, cb);
+                drain32(std::false_type{}, r1, cb + 32);
+                if (jg == 1) top.cut = fminf(top.best, topb.best) - top.thr;
+              } else {
+                drain32(std::true_type{}, r0, cb);
+                drain32(std::true_type{}, r1, cb + 32);
               }
             }
           }
         }
         ++n_done;
       }
+      top.insert_any(topb.best, topb.bi);
+      top.insert_any(topb.second, topb.si);
       // ---- combine the two column halves of each row and publish the chunk's result
       uint32_t *x = xchg + (size_t)(buf * 128 + row) * 5;
       if (half == 1) {
