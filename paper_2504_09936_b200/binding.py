@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkeepkv.so")
 
 EXPORTS = ("keepkv_workspace_bytes", "keepkv_workspace_init", "keepkv_append", "keepkv_decode_attention",
-           "keepkv_compress", "keepkv_decode_step_host", "keepkv_decode_attention_static", "keepkv_status_string", "keepkv_last_cuda_error",
+           "keepkv_compress", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_status_string", "keepkv_last_cuda_error",
            "keepkv_last_launch_count")
 
 
@@ -62,6 +62,7 @@ def lib() -> C.CDLL:
         l.keepkv_decode_attention_static.argtypes = [pp, pc, vp, vp, vp, C.c_int, vp, vp]
         l.keepkv_compress.argtypes = [pp, pc, pc, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         l.keepkv_decode_step_host.argtypes = [pp, pc] + [vp] * 8 + [C.c_int, vp, sz, vp, vp]
+        l.keepkv_decode_step_host_layers.argtypes = [pp, pc, i32] + [vp] * 8 + [C.c_int, vp, sz, vp, vp]
         _lib = l
     return _lib
 
@@ -169,6 +170,17 @@ def keepkv_decode_step_host(p, cache: Cache, q_host, k_new_host, v_new_host, out
                                          k_new_dev.data_ptr(), v_new_dev.data_ptr(), out_dev.data_ptr(),
                                          int(update_scores), ws.data_ptr(), ws.numel(), status.data_ptr(),
                                          _stream(stream)), "keepkv_decode_step_host")
+
+
+def keepkv_decode_step_host_layers(p, caches, q_host, k_new_host, v_new_host, out_host, q_dev, k_new_dev, v_new_dev,
+                                   out_dev, update_scores: bool, ws, status, stream=None):
+    """caches: list of Cache, one per layer; host / staging tensors carry the layers as their first axis."""
+    arr = (keepkv_cache * len(caches))(*[c.c() for c in caches])
+    _check(lib().keepkv_decode_step_host_layers(C.byref(p), arr, len(caches), q_host.data_ptr(), k_new_host.data_ptr(),
+                                                v_new_host.data_ptr(), out_host.data_ptr(), q_dev.data_ptr(),
+                                                k_new_dev.data_ptr(), v_new_dev.data_ptr(), out_dev.data_ptr(),
+                                                int(update_scores), ws.data_ptr(), ws.numel(), status.data_ptr(),
+                                                _stream(stream)), "keepkv_decode_step_host_layers")
 
 
 def last_launch_count() -> int:

@@ -202,6 +202,42 @@ int keepkv_decode_step_host(const keepkv_params *p, const keepkv_cache *cache, c
   return finish(ctx);
 }
 
+int keepkv_decode_step_host_layers(const keepkv_params *p, const keepkv_cache *caches_host, int32_t n_layers,
+                                   const void *q_host, const void *k_new_host, const void *v_new_host, void *out_host,
+                                   void *q_dev, void *k_new_dev, void *v_new_dev, void *out_dev, int update_scores,
+                                   void *ws, size_t ws_bytes, int32_t *status_dev, void *stream) {
+  int rc = validate(p);
+  if (rc) return rc;
+  if (!caches_host || n_layers <= 0) return KEEPKV_ERR_INVALID_ARG;
+  for (int l = 0; l < n_layers; ++l)
+    if ((rc = validate_cache(&caches_host[l]))) return rc;
+  if (!q_host || !k_new_host || !v_new_host || !out_host || !q_dev || !k_new_dev || !v_new_dev || !out_dev || !ws ||
+      !status_dev)
+    return KEEPKV_ERR_INVALID_ARG;
+  if (!aligned(q_dev, 16) || !aligned(k_new_dev, 16) || !aligned(v_new_dev, 16) || !aligned(out_dev, 16) ||
+      !aligned(ws, 256))
+    return KEEPKV_ERR_INVALID_ARG;
+  WsLayout L = ws_layout(*p);
+  if (ws_bytes < L.total) return KEEPKV_ERR_WORKSPACE;
+  LaunchCtx ctx{(cudaStream_t)stream, 0, cudaSuccess};
+  const size_t qb = (size_t)p->B * p->H_q * p->d * 2, kb = (size_t)p->B * p->H_kv * p->d * 2;
+  auto cp = [&](void *dstp, const void *srcp, size_t n, cudaMemcpyKind kind) {
+    cudaError_t e = cudaMemcpyAsync(dstp, srcp, n, kind, ctx.stream);
+    if (e != cudaSuccess && ctx.err == cudaSuccess) ctx.err = e;
+  };
+  cp(q_dev, q_host, qb * n_layers, cudaMemcpyHostToDevice);
+  cp(k_new_dev, k_new_host, kb * n_layers, cudaMemcpyHostToDevice);
+  cp(v_new_dev, v_new_host, kb * n_layers, cudaMemcpyHostToDevice);
+  for (int l = 0; l < n_layers && ctx.err == cudaSuccess; ++l) {
+    launch_append(*p, caches_host[l], (const char *)k_new_dev + kb * l, (const char *)v_new_dev + kb * l, status_dev, ctx);
+    if (ctx.err == cudaSuccess)
+      launch_decode(*p, caches_host[l], (const char *)q_dev + qb * l, (char *)out_dev + qb * l, nullptr, update_scores,
+                    (char *)ws, L, status_dev, ctx);
+  }
+  if (ctx.err == cudaSuccess) cp(out_host, out_dev, qb * n_layers, cudaMemcpyDeviceToHost);
+  return finish(ctx);
+}
+
 const char *keepkv_status_string(int status) {
   switch (status) {
     case KEEPKV_OK: return "KEEPKV_OK";

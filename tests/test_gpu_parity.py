@@ -267,6 +267,30 @@ def test_decode_step_host_matches_separate_calls():
     assert list(c1.seq_len.cpu()) == [101, 201]
 
 
+def test_decode_step_host_layers_matches_per_layer_calls():
+    p = kb.make_params(B=2, H_q=8, H_kv=2, d=128, N_cap=256)
+    Lr = 3
+    base = [random_cache(p, [100 + 7 * l, 200 - 5 * l], seed=40 + l) for l in range(Lr)]
+    clone = lambda c: kb.Cache(c.K.clone(), c.V.clone(), c.votes.clone(), c.lscore.clone(), c.seq_len.clone())
+    a, b = [clone(c) for c in base], [clone(c) for c in base]
+    ws, st = kb.new_workspace(p), kb.new_status()
+    rng = np.random.default_rng(6)
+    mk = lambda *s: torch.from_numpy(W.f32_to_bf16_bits(rng.standard_normal(s).astype(np.float32)).view(np.int16)).view(torch.bfloat16).pin_memory()
+    qh, kh, vh = mk(Lr, 2, 8, 128), mk(Lr, 2, 2, 128), mk(Lr, 2, 2, 128)
+    oh = torch.empty(Lr, 2, 8, 128, dtype=torch.bfloat16).pin_memory()
+    qd, kd, vd, od = (torch.empty_like(t, device="cuda") for t in (qh, kh, vh, oh))
+    kb.keepkv_decode_step_host_layers(p, a, qh, kh, vh, oh, qd, kd, vd, od, True, ws, st)
+    torch.cuda.synchronize()
+    for l in range(Lr):
+        out2 = torch.empty(2, 8, 128, dtype=torch.bfloat16, device="cuda")
+        kb.keepkv_append(p, b[l], kh[l].cuda(), vh[l].cuda(), st)
+        kb.keepkv_decode_attention(p, b[l], qh[l].cuda(), out2, None, True, ws, st)
+        torch.cuda.synchronize()
+        assert torch.equal(oh[l].cuda(), out2) and torch.equal(a[l].lscore, b[l].lscore) and torch.equal(a[l].K, b[l].K)
+        assert torch.equal(a[l].seq_len, b[l].seq_len)
+    assert int(st.item()) == 0
+
+
 def test_decode_is_deterministic():
     p = kb.make_params(B=2, H_q=8, H_kv=2, d=128, N_cap=2048)
     cache = random_cache(p, [2048, 1500], seed=8, vote_max=3)
