@@ -151,6 +151,15 @@ def score_update(P: Params, q, K, lscore):
     return ls
 
 
+def prefill_scores(P: Params, q_window, K):
+    """Eq. 8 first case for one unit: q_window [W, G, d] (oldest first), K [len, d] -> lscore [len]."""
+    q, K = _f64(q_window), _f64(K)
+    ls = np.empty(K.shape[0], dtype=np.float64)
+    cp = P.c()
+    lib().okv_prefill_scores(C.byref(cp), C.c_int32(K.shape[0]), C.c_int32(q.shape[0]), _p(q), _p(K), _p(ls))
+    return ls
+
+
 def kappa(votes, lscore):
     votes, lscore = _f64(votes), _f64(lscore)
     k = np.empty(votes.shape[0], dtype=np.float32)

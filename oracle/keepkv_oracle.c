@@ -154,6 +154,50 @@ void okv_score_update(const okv_params *P, int32_t len, const double *q, const d
   free(ell);
 }
 
+/* ---------------------------------- Eq. 8, first case: windowed initialisation */
+
+/* Score estimate at the end of prefill (t = L in Eq. 8) from the last W = w + 1 prompt queries.
+ * q is [W][G][d], oldest query first; query k sits at prompt position pos_k = len - W + k and, the
+ * prompt being causal, has a score only for entries i <= pos_k (queries with pos_k < 0 do not
+ * exist).  With weights omega_k = alpha^(W-1-k) -- the (1 - alpha) alpha^(t-k) of Eq. 8 up to the
+ * common factor --
+ *   s_hat_i = sum_{k visible} omega_k s_i^k / sum_{k visible} omega_k ,
+ *   s_i^k   = (1/G) sum_g exp(sm_scale * q_{k,g} . k_i)        (group mean as in okv_score_update),
+ * i.e. the bias correction divides by the weight actually accumulated, which for an entry seen by
+ * the whole window is the printed 1 - alpha^(w+1).  alpha = 0 keeps the last query only.
+ * lscore_i = ln s_hat_i overwrites whatever the entry held. */
+void okv_prefill_scores(const okv_params *P, int32_t len, int32_t W, const double *q, const double *K,
+                        double *lscore) {
+  const int G = P->G, d = P->d;
+  for (int i = 0; i < len; ++i) {
+    /* log-sum-exp over the visible (k, g) pairs of  ln omega_k + l_{k,g,i} */
+    double M = -INFINITY, wsum = 0.0;
+    for (int pass = 0; pass < 2; ++pass) {
+      double acc = 0.0;
+      for (int k = 0; k < W; ++k) {
+        const int pos = len - W + k;
+        if (pos < 0 || i > pos) continue;
+        double lw;
+        if (P->ema_alpha == 0.0) {
+          if (k != W - 1) continue;
+          lw = 0.0;
+        } else {
+          lw = (double)(W - 1 - k) * log(P->ema_alpha);
+        }
+        if (pass == 0) wsum += exp(lw);
+        for (int g = 0; g < G; ++g) {
+          double dot = 0.0;
+          for (int j = 0; j < d; ++j) dot += q[((size_t)k * G + g) * d + j] * K[(size_t)i * d + j];
+          const double x = lw + P->sm_scale * dot;
+          if (pass == 0) { if (x > M) M = x; }
+          else acc += exp(x - M);
+        }
+      }
+      if (pass == 1) lscore[i] = store_f32(P, M + log(acc) - log(wsum) - log((double)G));
+    }
+  }
+}
+
 /* ------------------------------------------------------------- selection */
 
 /* Selection key: the entry's whole attention mass p_i * s_hat_i, as a logarithm,

@@ -480,3 +480,60 @@ def test_batch_wrappers_match_per_unit():
         assert m == len(c["ret_idx"])
         assert np.array_equal(r["K"][u, :m], c["K"]) and np.array_equal(r["votes"][u, :m], c["votes"])
         assert np.array_equal(r["ret_idx"][u, :m], c["ret_idx"]) and np.array_equal(r["target"][u, :n], c["target"])
+
+
+# ------------------------------------------------------------------ Eq. 8, first case (windowed initialisation)
+
+def _raw_scores(q_window, K, d):
+    """s_i^k = mean over the group of exp(q.k/sqrt(d)), written out with numpy: [W, len]."""
+    logits = np.einsum("kgd,id->kgi", q_window, K) / np.sqrt(d)
+    return np.exp(logits).mean(axis=1)
+
+
+@pytest.mark.parametrize("alpha,W,G", [(0.9, 8, 1), (0.5, 5, 4), (0.9, 33, 2)])
+def test_windowed_init_equals_bias_corrected_recursion(alpha, W, G):
+    """Eq. 8: running the recursion S <- alpha S + (1 - alpha) s over the window from S = 0 and dividing
+    by 1 - alpha^n (n = steps taken) gives the windowed first case.  Entries older than the window see
+    every query; the recursion is written out here in numpy, independently of the oracle."""
+    rng = np.random.default_rng(int(alpha * 100) + W)
+    d, n = 16, 40 + W
+    K = rng.standard_normal((n, d)) * 0.7
+    qw = rng.standard_normal((W, G, d))
+    P = O.Params(G=G, d=d, ema_alpha=alpha)
+    got = O.prefill_scores(P, qw, K)
+    s = _raw_scores(qw, K, d)
+    old = np.arange(n) <= n - W            # entries every query of the window can see
+    S = np.zeros(n)
+    for k in range(W):
+        S = alpha * S + (1 - alpha) * s[k]
+    want = np.log(S / (1 - alpha ** W))
+    assert np.allclose(got[old], want[old], rtol=1e-12, atol=1e-12)
+
+
+def test_windowed_init_respects_causality_and_constant_scores():
+    """An entry inside the window is scored only by the queries at or after its position, with the weights
+    renormalised (brute force per entry); identical queries give s_hat = s whatever alpha is; W = 1 is
+    the first observation of the decode path."""
+    rng = np.random.default_rng(7)
+    d, n, W, G, alpha = 8, 12, 5, 2, 0.8
+    K = rng.standard_normal((n, d))
+    qw = rng.standard_normal((W, G, d))
+    P = O.Params(G=G, d=d, ema_alpha=alpha)
+    got = O.prefill_scores(P, qw, K)
+    s = _raw_scores(qw, K, d)
+    for i in range(n):
+        ks = [k for k in range(W) if n - W + k >= i]
+        w = np.array([alpha ** (W - 1 - k) for k in ks])
+        want = np.log((w * s[ks, i]).sum() / w.sum())
+        assert abs(got[i] - want) < 1e-12, i
+    # constant query sequence: the estimate is the score itself
+    qc = np.repeat(qw[:1], W, axis=0)
+    assert np.allclose(O.prefill_scores(P, qc, K), np.log(_raw_scores(qc, K, d)[0]), atol=1e-12)
+    # window of one query = first observation in the recursive path; alpha = 0 keeps only the last query
+    one = O.prefill_scores(P, qw[-1:], K)
+    assert np.allclose(one, O.score_update(P, qw[-1], K, np.full(n, -np.inf)), atol=1e-12)
+    P0 = O.Params(G=G, d=d, ema_alpha=0.0)
+    assert np.allclose(O.prefill_scores(P0, qw, K), one, atol=1e-12)
+    # a prompt shorter than the window: the queries before position 0 do not exist
+    short = O.prefill_scores(P, qw, K[:3])
+    assert np.allclose(short, O.prefill_scores(P, qw[-3:], K[:3]), atol=1e-12)
