@@ -119,6 +119,17 @@ int keepkv_decode_attention(const keepkv_params *p, const keepkv_cache *cache, c
                             float *lse_or_null, int update_scores, void *ws, size_t ws_bytes, int32_t *status_dev,
                             void *stream);
 
+/* Eq. 8, first case: the score estimate at the end of prefill, from the last W prompt queries
+ * (W = w + 1 <= 32).  q_window: bf16 [B, H_q, W, d], oldest query first; query k sits at position
+ * seq_len[b] - W + k and, the prompt being causal, scores only the entries at or before it.  For every entry
+ * i < seq_len[b] of every kv head
+ *   lscore_i <- ln( sum_k alpha^(W-1-k) s_i^k / sum_k alpha^(W-1-k) ),   k over the window queries that see i,
+ * with s_i^k the mean over the head's G query heads of exp(sm_scale q_k . k_i); alpha = 0 keeps the last query
+ * only.  The division by the accumulated weight is the bias correction of Eq. 8 (1 - alpha^(w+1) for an entry
+ * older than the window).  Whatever lscore held before is overwritten; K, V, votes are only read. */
+int keepkv_prefill_scores(const keepkv_params *p, const keepkv_cache *cache, const void *q_window, int32_t W,
+                          int32_t *status_dev, void *stream);
+
 /* Algorithm 1, out of place: reads `src` (unchanged), writes `dst` (distinct buffers of the same
  * shape).  Per unit, with len = src.seq_len[b] and budget b_b (budget_dev[b] if given, else
  * budget_scalar; likewise n_recent_dev[b] / p->n_recent):

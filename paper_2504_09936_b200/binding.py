@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkeepkv.so")
 
 EXPORTS = ("keepkv_workspace_bytes", "keepkv_workspace_init", "keepkv_append", "keepkv_decode_attention",
-           "keepkv_compress", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_status_string", "keepkv_last_cuda_error",
+           "keepkv_compress", "keepkv_prefill_scores", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_status_string", "keepkv_last_cuda_error",
            "keepkv_last_launch_count")
 
 
@@ -60,6 +60,7 @@ def lib() -> C.CDLL:
         l.keepkv_append.argtypes = [pp, pc, vp, vp, vp, vp]
         l.keepkv_decode_attention.argtypes = [pp, pc, vp, vp, vp, C.c_int, vp, sz, vp, vp]
         l.keepkv_decode_attention_static.argtypes = [pp, pc, vp, vp, vp, C.c_int, vp, vp]
+        l.keepkv_prefill_scores.argtypes = [pp, pc, vp, i32, vp, vp]
         l.keepkv_compress.argtypes = [pp, pc, pc, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         l.keepkv_decode_step_host.argtypes = [pp, pc] + [vp] * 8 + [C.c_int, vp, sz, vp, vp]
         l.keepkv_decode_step_host_layers.argtypes = [pp, pc, i32] + [vp] * 8 + [C.c_int, vp, sz, vp, vp]
@@ -152,6 +153,13 @@ def keepkv_decode_attention_static(p, cache: Cache, q, out, lse, update_scores: 
     _check(lib().keepkv_decode_attention_static(C.byref(p), C.byref(cache.c()), q.data_ptr(), out.data_ptr(),
                                                 _ptr(lse), int(update_scores), status.data_ptr(), _stream(stream)),
            "keepkv_decode_attention_static")
+
+
+def keepkv_prefill_scores(p, cache: Cache, q_window, status, stream=None):
+    """q_window: bf16 CUDA tensor [B, H_q, W, d], the last W prompt queries, oldest first (Eq. 8, first case)."""
+    assert q_window.is_contiguous() and q_window.dim() == 4
+    _check(lib().keepkv_prefill_scores(C.byref(p), C.byref(cache.c()), q_window.data_ptr(), int(q_window.shape[2]),
+                                       status.data_ptr(), _stream(stream)), "keepkv_prefill_scores")
 
 
 def keepkv_compress(p, src: Cache, dst: Cache, budget, ws, status, n_recent_dev=None, retained_idx=None,

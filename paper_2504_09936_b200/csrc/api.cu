@@ -143,6 +143,19 @@ int keepkv_decode_attention(const keepkv_params *p, const keepkv_cache *cache, c
   return finish(ctx);
 }
 
+int keepkv_prefill_scores(const keepkv_params *p, const keepkv_cache *cache, const void *q_window, int32_t W,
+                          int32_t *status_dev, void *stream) {
+  int rc = validate(p);
+  if (rc) return rc;
+  if ((rc = validate_cache(cache))) return rc;
+  if (!q_window || !status_dev || !aligned(q_window, 16)) return KEEPKV_ERR_INVALID_ARG;
+  if (W < 1) return KEEPKV_ERR_INVALID_ARG;
+  if (W > 32) return KEEPKV_ERR_UNSUPPORTED;
+  LaunchCtx ctx{(cudaStream_t)stream, 0, cudaSuccess};
+  launch_prefill_scores(*p, *cache, q_window, W, status_dev, ctx);
+  return finish(ctx);
+}
+
 int keepkv_compress(const keepkv_params *p, const keepkv_cache *src, const keepkv_cache *dst,
                     const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
                     int32_t *retained_idx_or_null, int32_t *target_or_null, keepkv_stats *stats_or_null, void *ws,

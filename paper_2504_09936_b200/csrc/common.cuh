@@ -66,6 +66,8 @@ void launch_compress(const keepkv_params &p, const keepkv_cache &src, const keep
 void launch_nominate(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst, const int32_t *ev_idx,
                      const UnitInfo *unit_info, const float *inv_norm, int32_t *sched, float4 *nom_v, int32_t *nom_si,
                      int nom_chunks, int32_t *status_dev, LaunchCtx &ctx);
+void launch_prefill_scores(const keepkv_params &p, const keepkv_cache &c, const void *q_window, int W,
+                           int32_t *status_dev, LaunchCtx &ctx);
 int sm_count();
 
 // Launch with programmatic stream serialisation: the kernel may be scheduled while its predecessor in

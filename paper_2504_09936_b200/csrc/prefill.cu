@@ -1,0 +1,358 @@
+// keepkv_prefill_scores: the score estimate every entry starts decoding with (Eq. 8, first case): a
+// bias-corrected exponentially weighted mean of the entry's scores under the last W prompt queries.
+//
+// Per (sequence, kv-head) unit this is a (len x d) . (d x G*W) contraction followed by a weighted
+// log-sum-exp along the G*W query columns, bound by the one pass over the keys.  The keys are the A
+// operand of a tcgen05.mma (128 entries = 128 tensor-memory lanes per tile), the unit's G*W window
+// queries the B operand (head g, query k in column g*32 + k), so every drain thread owns one entry and
+// reduces its columns in registers, without shuffles.  One persistent CTA per SM walks a contiguous
+// range of the global list of 128-entry tiles:
+//   warp 0     TMA producer: the unit's window queries (one box of W rows per head) when the unit
+//              changes, key tiles into a 3-stage ring;
+//   warp 1     one thread issues the MMAs into one of two accumulators and commits to the barriers;
+//   warps 2-9  drain (two warps per 32 entries, alternate heads, combined through shared memory): per
+//              entry a running max / weighted sum of 2^(x - max) over the visible queries
+//              (a prompt is causal: query k, at position len - W + k, scores only entries at or before
+//              it), then lscore = ln(sum / sum of the visible weights / G).
+// Every wait is bounded; one that runs out raises KEEPKV_DEV_TIMEOUT and the CTA winds down.
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace keepkv {
+
+constexpr int kPfM = 128;        // entries per tile
+constexpr int kPfStages = 3;     // key-tile ring
+constexpr int kPfThreads = 320;  // producer, MMA issuer, eight drain warps (two per 32-lane quarter, alternate heads)
+constexpr int kPfWmax = 32;      // window queries per head (columns reserved per head)
+constexpr float kPfLog2e = 1.4426950408889634f;
+constexpr float kPfLn2 = 0.6931471805599453f;
+
+template <int D, int G>
+struct PfSmem {
+  static constexpr int kSub = D / 64;
+  static constexpr int kNB = G * kPfWmax;                   // columns of the accumulator
+  static constexpr int kABytes = kSub * kPfM * 128;
+  static constexpr int kBBytes = kSub * kNB * 128;
+  static constexpr int kA = 0;
+  static constexpr int kB = kPfStages * kABytes;
+  static constexpr int kWt = kB + kBBytes;                  // f32 [32] weights, f32 [33] their suffix sums (as ln)
+  static constexpr int kXchg = kWt + 512;                   // f32 [2 accumulators][128 entries][2]: the odd heads' (max, sum)
+  static constexpr int kBytes = kXchg + 2 * 128 * 2 * 4;
+};
+
+// Position in the global tile list: sequence, kv head, tile of the unit; next() moves to the next tile.
+__device__ __forceinline__ float pf_ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+struct PfWalker {
+  int b, h, tile, len, tb;
+  __device__ __forceinline__ void load(const keepkv_params &p, const int32_t *seq_len) {
+    len = max(0, min(seq_len[b], p.N_cap));
+    tb = (len + kPfM - 1) / kPfM;
+  }
+  __device__ __forceinline__ void next(const keepkv_params &p, const int32_t *seq_len, bool more) {
+    if (++tile == tb && more) {
+      tile = 0;
+      if (++h == p.H_kv) {
+        h = 0;
+        do { ++b; load(p, seq_len); } while (tb == 0);
+      }
+    }
+  }
+};
+
+template <int D, int G>
+__global__ void __launch_bounds__(kPfThreads, 1)
+prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapQ,
+                      keepkv_params p, keepkv_cache c, int W, int32_t *status_dev) {
+  using SL = PfSmem<D, G>;
+  constexpr int KSTEPS = D / 16, NB = SL::kNB;
+  constexpr uint32_t IDESC = umma_idesc_bf16(kPfM, NB);
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * kPfStages + 7];   // a_full[S], a_empty[S], b_full, b_empty, t_full[2], t_empty[2], drain
+  __shared__ uint32_t s_tmem;
+  __shared__ int s_scan[kPfThreads / 32];
+  __shared__ int s_start[4];
+  __shared__ volatile int s_abort;
+
+  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sbase = smem_u32(smem);
+  const uint32_t bar_a_full = smem_u32(&bars[0]), bar_a_empty = smem_u32(&bars[kPfStages]);
+  const uint32_t bar_b_full = smem_u32(&bars[2 * kPfStages]), bar_b_empty = smem_u32(&bars[2 * kPfStages + 1]);
+  const uint32_t bar_t_full = smem_u32(&bars[2 * kPfStages + 2]), bar_t_empty = smem_u32(&bars[2 * kPfStages + 4]);
+  const uint32_t bar_drain = smem_u32(&bars[2 * kPfStages + 6]);
+  float *wt = reinterpret_cast<float *>(smem + SL::kWt);   // wt[k], k < 32
+  float *lnwsuf = wt + 32;                                  // ln sum_{k' >= k} wt[k'], k <= 32
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int cta = blockIdx.x, grid = gridDim.x;
+
+  if (tid == 0) {
+    for (int i = 0; i < kPfStages; ++i) { mbar_init(bar_a_full + 8 * i, 1); mbar_init(bar_a_empty + 8 * i, 1); }
+    mbar_init(bar_b_full, 1);
+    mbar_init(bar_b_empty, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_t_full + 8 * i, 1); mbar_init(bar_t_empty + 8 * i, 8); }
+    mbar_init(bar_drain, 1);
+    s_abort = 0;
+    s_start[0] = p.B;
+    mbar_fence_init();
+    prefetch_tensormap(&mapK);
+    prefetch_tensormap(&mapQ);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&s_tmem), 512);
+    tmem_relinquish();
+  }
+  // rows of the query tile that no copy writes (k >= W) must hold finite numbers: zero the tile once
+  for (int i = tid; i < SL::kBBytes / 16; i += kPfThreads)
+    *reinterpret_cast<uint4 *>(smem + SL::kB + i * 16) = make_uint4(0, 0, 0, 0);
+  if (tid < 32) {
+    // weights alpha^(W-1-k) of the window's queries (alpha = 0: the last query only) and the logarithms of
+    // their suffix sums (the weight an entry first seen by query k has accumulated)
+    const float wk = tid < W ? (p.ema_alpha > 0.f ? expf((float)(W - 1 - tid) * logf(p.ema_alpha)) : (tid == W - 1 ? 1.f : 0.f))
+                             : 0.f;
+    wt[tid] = wk;
+    float suf = wk;   // inclusive suffix sum over lanes
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const float y = __shfl_down_sync(0xffffffffu, suf, o);
+      if (lane + o < 32) suf += y;
+    }
+    lnwsuf[tid] = logf(suf);
+    if (tid == 0) lnwsuf[32] = -CUDART_INF_F;
+  }
+  fence_proxy_async_smem();
+  pdl_wait();
+  pdl_trigger();
+
+  // ---- the tile list: every thread sums a block of consecutive sequences, a block scan gives the offsets
+  auto tiles_of = [&](int b) { return (max(0, min(c.seq_len[b], p.N_cap)) + kPfM - 1) / kPfM; };
+  const int per = (p.B + kPfThreads - 1) / kPfThreads;
+  const int b_lo = min(p.B, tid * per), b_hi = min(p.B, b_lo + per);
+  int mine = 0;
+  for (int b = b_lo; b < b_hi; ++b) mine += tiles_of(b);
+  int incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int y = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += y;
+  }
+  if (lane == 31) s_scan[warp] = incl;
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  int before = incl - mine, total_b = 0;
+  for (int w = 0; w < kPfThreads / 32; ++w) {
+    if (w < warp) before += s_scan[w];
+    total_b += s_scan[w];
+  }
+  const long long T = (long long)total_b * p.H_kv;
+  const int chunk = (int)((T + grid - 1) / grid);
+  const long long g0 = min(T, (long long)cta * chunk), g1 = min(T, g0 + chunk);
+  const int ntiles = (int)(g1 - g0);
+  if (ntiles > 0 && (long long)before * p.H_kv <= g0 && g0 < (long long)(before + mine) * p.H_kv) {
+    long long at = (long long)before * p.H_kv;
+    for (int b = b_lo; b < b_hi; ++b) {
+      const int tb = tiles_of(b);
+      const long long span = (long long)tb * p.H_kv;
+      if (g0 < at + span) {
+        const int r = (int)(g0 - at);
+        s_start[0] = b; s_start[1] = r / tb; s_start[2] = r % tb;
+        break;
+      }
+      at += span;
+    }
+  }
+  __syncthreads();
+  const uint32_t tmem = s_tmem;
+  PfWalker wk;
+  wk.b = s_start[0]; wk.h = s_start[1]; wk.tile = s_start[2]; wk.len = 0; wk.tb = 1;
+  if (ntiles > 0) wk.load(p, c.seq_len);
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int n_units = 0;
+      for (int it = 0; it < ntiles && !s_abort; ++it) {
+        const int u = wk.b * p.H_kv + wk.h;
+        if (it == 0 || wk.tile == 0) {   // the unit's window queries: W rows per head into columns g*32 ..
+          if (n_units > 0 && !mbar_wait(bar_b_empty, (n_units - 1) & 1)) { s_abort = 1; break; }
+          ++n_units;
+          mbar_expect_tx(bar_b_full, (uint32_t)(G * SL::kSub * W * 128));
+#pragma unroll
+          for (int g = 0; g < G; ++g)
+#pragma unroll
+            for (int sub = 0; sub < SL::kSub; ++sub)
+              tma_load_2d(sbase + SL::kB + sub * (NB * 128) + g * kPfWmax * 128, &mapQ, sub * 64,
+                          (wk.b * p.H_q + wk.h * G + g) * W, bar_b_full);
+        }
+        const int s = it % kPfStages;
+        if (!mbar_wait(bar_a_empty + 8 * s, ((it / kPfStages) & 1) ^ 1)) { s_abort = 1; break; }
+        mbar_expect_tx(bar_a_full + 8 * s, SL::kABytes);
+#pragma unroll
+        for (int sub = 0; sub < SL::kSub; ++sub)
+          tma_load_2d(sbase + SL::kA + s * SL::kABytes + sub * (kPfM * 128), &mapK, sub * 64,
+                      u * p.N_cap + wk.tile * kPfM, bar_a_full + 8 * s);
+        wk.next(p, c.seq_len, it + 1 < ntiles);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int n_units = 0;
+      for (int it = 0; it < ntiles && !s_abort; ++it) {
+        if (it == 0 || wk.tile == 0) {
+          if (!mbar_wait(bar_b_full, n_units & 1)) { s_abort = 1; break; }
+          ++n_units;
+        }
+        const int s = it % kPfStages, a = it & 1;
+        if (!mbar_wait(bar_a_full + 8 * s, (it / kPfStages) & 1) ||
+            !mbar_wait(bar_t_empty + 8 * a, ((it >> 1) & 1) ^ 1)) { s_abort = 1; break; }
+        tc_fence_after();
+        const uint32_t a_base = sbase + SL::kA + s * SL::kABytes, b_base = sbase + SL::kB;
+#pragma unroll
+        for (int k = 0; k < KSTEPS; ++k) {
+          const uint64_t ad = umma_desc_sw128(a_base + (k >> 2) * (kPfM * 128) + (k & 3) * 32);
+          const uint64_t bd = umma_desc_sw128(b_base + (k >> 2) * (NB * 128) + (k & 3) * 32);
+          umma_bf16(tmem + a * NB, ad, bd, IDESC, k > 0 ? 1u : 0u);
+        }
+        umma_commit(bar_a_empty + 8 * s);
+        umma_commit(bar_t_full + 8 * a);
+        const bool unit_ends = wk.tile == wk.tb - 1 || it == ntiles - 1;
+        if (unit_ends) umma_commit(bar_b_empty);   // the query tile may be replaced once these MMAs have read it
+        wk.next(p, c.seq_len, it + 1 < ntiles);
+      }
+      umma_commit(bar_drain);
+      mbar_wait(bar_drain, 0);   // every MMA issued above has retired (bounded)
+    }
+  } else {
+    // ------------------------------------------------------------ drain: one entry per thread
+    const int quarter = warp & 3, half = (warp - 2) >> 2;       // half 0 takes the even heads, half 1 the odd ones
+    const float scale2 = p.sm_scale * kPfLog2e;
+    const float ln_G = logf((float)G);
+    float *xchg = reinterpret_cast<float *>(smem + SL::kXchg);
+    float wr[32];   // the window weights stay in registers
+#pragma unroll
+    for (int k = 0; k < 32; ++k) wr[k] = wt[k];
+    for (int it = 0; it < ntiles; ++it) {
+      const int a = it & 1;
+      int ok = 0;
+      if (lane == 0) ok = !s_abort && mbar_wait(bar_t_full + 8 * a, (it >> 1) & 1);
+      if (!__shfl_sync(0xffffffffu, ok, 0)) { s_abort = 1; break; }
+      tc_fence_after();
+      const int row = quarter * 32 + lane;
+      const int i = wk.tile * kPfM + row;                         // this thread's entry
+      const int klo = min(32, max(0, i - wk.len + W));            // first window query that sees it
+      const bool full = W == kPfWmax && wk.tile * kPfM + kPfM - 1 - wk.len + W <= 0;   // whole tile sees every query
+      const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + a * NB;
+      float m = -CUDART_INF_F, S = 0.f;
+      constexpr int LAST = G >= 2 ? G - 2 : 0;   // last head index of half 0 (half 1: LAST + 1)
+#pragma unroll 1
+      for (int g = half; g < G; g += 2) {
+        uint32_t r[32];
+        tmem_ld_32x32(taddr + g * 32, r);
+        tmem_ld_wait();
+        if (g >= LAST) {   // this warp's part of the accumulator is in registers: hand it back
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_t_empty + 8 * a);
+        }
+        float x[32], mc = -CUDART_INF_F;
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+          x[k] = __uint_as_float(r[k]) * scale2;
+          if (!full) x[k] = (k >= klo && k < W) ? x[k] : -CUDART_INF_F;
+          mc = fmaxf(mc, x[k]);
+        }
+        const float m_new = fmaxf(m, mc);
+        if (m_new > -CUDART_INF_F) {
+          S *= pf_ex2(m - m_new);   // m = -inf: S is 0 and stays 0
+          float add0 = 0.f, add1 = 0.f;
+#pragma unroll
+          for (int k = 0; k < 32; k += 2) {
+            add0 = fmaf(wr[k], pf_ex2(x[k] - m_new), add0);
+            add1 = fmaf(wr[k + 1], pf_ex2(x[k + 1] - m_new), add1);
+          }
+          S += add0 + add1;
+          m = m_new;
+        }
+      }
+      if (G == 1) {
+        if (half == 1) {   // a single head: nothing for the second warp of the quarter to read
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar_t_empty + 8 * a);
+        }
+      } else {
+        // the two warps of a quarter meet at a barrier of their own (64 threads)
+        float2 *x2 = reinterpret_cast<float2 *>(xchg) + a * 128 + row;
+        if (half == 1) *x2 = make_float2(m, S);
+        asm volatile("bar.sync %0, 64;" ::"r"(1 + quarter) : "memory");
+        if (half == 0) {
+          const float2 o = *x2;
+          const float mm = fmaxf(m, o.x);
+          if (mm > -CUDART_INF_F) S = S * pf_ex2(m - mm) + o.y * pf_ex2(o.x - mm);
+          m = mm;
+        }
+      }
+      if (half == 0 && i < wk.len)
+        c.lscore[((size_t)(wk.b * p.H_kv + wk.h)) * p.N_cap + i] = (m + log2f(S)) * kPfLn2 - lnwsuf[klo] - ln_G;
+      wk.next(p, c.seq_len, it + 1 < ntiles);
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (s_abort) {
+    if (tid == 0) {
+      atomicOr(status_dev, KEEPKV_DEV_TIMEOUT);
+      for (int i = 0; i < kPfStages; ++i) { mbar_wait(bar_a_full + 8 * i, 0); mbar_wait(bar_a_full + 8 * i, 1); }
+      mbar_wait(bar_b_full, 0); mbar_wait(bar_b_full, 1);
+    }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    tmem_dealloc(tmem, 512);
+  }
+}
+
+template <int D, int G>
+static void launch_prefill_t(const keepkv_params &p, const keepkv_cache &c, const void *q_window, int W,
+                             int32_t *status_dev, LaunchCtx &ctx) {
+  using SL = PfSmem<D, G>;
+  constexpr size_t smem_bytes = (size_t)SL::kBytes + 1024;
+  static bool attr_done_dev[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (!attr_done_dev[dev & 63]) {
+    cudaFuncSetAttribute(prefill_scores_kernel<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+    attr_done_dev[dev & 63] = true;
+  }
+  CUtensorMap mapK, mapQ;
+  if (!make_bf16_rows_map(&mapK, c.K, (uint64_t)p.B * p.H_kv * p.N_cap, D, kPfM) ||
+      !make_bf16_rows_map(&mapQ, const_cast<void *>(q_window), (uint64_t)p.B * p.H_q * W, D, W)) {
+    if (ctx.err == cudaSuccess) ctx.err = cudaErrorInvalidValue;
+    return;
+  }
+  launch_pdl(prefill_scores_kernel<D, G>, dim3(sm_count()), dim3(kPfThreads), smem_bytes, ctx.stream, mapK, mapQ, p, c,
+             W, status_dev);
+  KEEPKV_CHECK_LAUNCH(ctx);
+}
+
+void launch_prefill_scores(const keepkv_params &p, const keepkv_cache &c, const void *q_window, int W,
+                           int32_t *status_dev, LaunchCtx &ctx) {
+  const int G = p.H_q / p.H_kv;
+#define KEEPKV_DISPATCH(DD, GG) \
+  if (p.d == DD && G == GG) return launch_prefill_t<DD, GG>(p, c, q_window, W, status_dev, ctx);
+  KEEPKV_DISPATCH(128, 1) KEEPKV_DISPATCH(128, 2) KEEPKV_DISPATCH(128, 4) KEEPKV_DISPATCH(128, 8)
+  KEEPKV_DISPATCH(64, 1) KEEPKV_DISPATCH(64, 2) KEEPKV_DISPATCH(64, 4) KEEPKV_DISPATCH(64, 8)
+#undef KEEPKV_DISPATCH
+}
+
+}  // namespace keepkv

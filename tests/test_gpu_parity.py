@@ -299,3 +299,34 @@ def test_decode_is_deterministic():
     for _ in range(3):
         b2, lb = _run_decode(p, cache, q, False)
         assert torch.equal(a, b2) and torch.equal(la, lb)
+
+
+@pytest.mark.parametrize("G,d,W,alpha", [(4, 128, 32, 0.9), (1, 64, 32, 0.9), (8, 128, 32, 0.5), (2, 64, 7, 0.9),
+                                         (4, 128, 1, 0.9), (4, 64, 32, 0.0)])
+def test_prefill_scores_windowed_initialisation(G, d, W, alpha):
+    """Eq. 8, first case: ragged prompts (one shorter than the window, one empty, several tiles with a ragged
+    tail), causal window, every unit against the oracle; K, V, votes untouched, entries past seq_len untouched."""
+    H_kv, B = 2, 5
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=704, ema_alpha=alpha)
+    lens = [700, 0, 20, 129, 384]
+    cache = random_cache(p, lens, seed=G + d + W, scored_frac=0.5, scale=0.6)
+    before = HostCache(cache)
+    rng = np.random.default_rng(W)
+    qw = f32_to_dev_bf16(rng.standard_normal((B, p.H_q, W, d)).astype(np.float32))
+    st = kb.new_status()
+    kb.keepkv_prefill_scores(p, cache, qw, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    after = HostCache(cache)
+    assert np.array_equal(after.K, before.K) and np.array_equal(after.V, before.V) and np.array_equal(after.votes, before.votes)
+    P = oracle_params(p)
+    q64 = to_f64(qw)
+    for u in range(B * H_kv):
+        b, h = divmod(u, H_kv)
+        n = lens[b]
+        assert np.array_equal(after.lscore[u, n:], before.lscore[u, n:], equal_nan=True)
+        if n == 0:
+            continue
+        qu = np.ascontiguousarray(q64[b, h * G:(h + 1) * G].transpose(1, 0, 2))      # [W, G, d]
+        ref = O.prefill_scores(P, qu, before.K[u, :n])
+        check_close(after.lscore[u, :n], ref, f"prefill scores u={u}", ulps=None, max_abs=1e-3, mean_rel=1e-4)
