@@ -281,7 +281,7 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
 }
 
 // ------------------------------------------------------------------ compact
-// grid (ceil(bound/64), U), 256 threads.  Sixteen lanes move one retained row (a 16-byte piece of
+// grid (up to 32, U), 256 threads, 64 slots per CTA and sweep.  Sixteen lanes move one retained row (a 16-byte piece of
 // K and of V each); a warp has eight rows in flight.  The same lanes tree-sum the squared key for
 // the inverse norm the similarity search ranks with.
 template <int D>
@@ -292,8 +292,7 @@ compact_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
   pdl_wait();
   pdl_trigger();
   const int u = blockIdx.y, n_ret = unit_info[u].n_ret;
-  const int s0 = blockIdx.x * 64;
-  if (s0 >= n_ret) return;
+  for (int s0 = blockIdx.x * 64; s0 < n_ret; s0 += gridDim.x * 64) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, ch = lane & 15, sub = lane >> 4;
   const size_t base = (size_t)u * p.N_cap;
   const uint4 *sK = reinterpret_cast<const uint4 *>(src.K), *sV = reinterpret_cast<const uint4 *>(src.V);
@@ -333,6 +332,7 @@ compact_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
       dst.votes[base + slot[r]] = src.votes[base + si[r]];
       dst.lscore[base + slot[r]] = src.lscore[base + si[r]];
     }
+  }
   }
 }
 
@@ -383,7 +383,12 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
   uint32_t *gk = grp_key + (size_t)u * key_stride;
   const int C = sched[0];
   const float T = p.merge_threshold;
-  if (tid == 0) s_nq[0] = s_nq[1] = 0;
+  // CTAs of the unit that have rows; the others leave at once.  A unit whose rows fit one pass of one CTA
+  // (every steady-state compression) needs no exchange through global memory.
+  const int n_cta = min((int)gridDim.x, (ui.n_ev + kResolveThreads - 1) / kResolveThreads);
+  if ((int)blockIdx.x >= n_cta) return;
+  const bool single = ui.n_ev <= kResolveThreads;
+  if (tid == 0) { s_nq[0] = s_nq[1] = 0; s_base = 0; }
   __syncthreads();
 
   int pass = 0;
@@ -454,6 +459,15 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
     // ---- record the decision; entries to merge go to the unit's key list (any order: it is sorted below)
     int tot;
     const int off = block_excl_count(merge, warp_tot, tot);
+    if (single) {   // this CTA holds all rows of the unit: its keys never leave shared memory
+      if (valid) {
+        target[base + e] = merge ? slot : -1;
+        if (merge) key_smem[off] = ((uint32_t)slot << 16) | (uint32_t)j;
+      }
+      if (tid == 0) s_base = tot;
+      __syncthreads();
+      continue;
+    }
     if (tid == 0) s_base = tot ? atomicAdd(&unit_info[u].n_keys, tot) : 0;
     __syncthreads();
     if (valid) {
@@ -461,18 +475,23 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
       if (merge) gk[s_base + off] = ((uint32_t)slot << 16) | (uint32_t)j;
     }
   }
-  // ---- the last CTA of the unit to arrive groups the entries
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) s_last = atomicAdd(&unit_info[u].ticket, 1) == (int)gridDim.x - 1;
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  const int M = *reinterpret_cast<volatile int *>(&unit_info[u].n_keys);
+  int M;
+  if (single) {
+    M = s_base;
+  } else {
+    // ---- the last CTA of the unit to arrive groups the entries
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = atomicAdd(&unit_info[u].ticket, 1) == n_cta - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    M = *reinterpret_cast<volatile int *>(&unit_info[u].n_keys);
+  }
   int Mp = 1;
   while (Mp < M) Mp <<= 1;
-  uint32_t *keys = Mp <= smem_keys ? key_smem : gk;
-  if (keys != gk)
+  uint32_t *keys = (single || Mp <= smem_keys) ? key_smem : gk;
+  if (keys != gk && !single)
     for (int i = tid; i < M; i += kResolveThreads) keys[i] = __ldcg(&gk[i]);
   for (int i = M + tid; i < Mp; i += kResolveThreads) keys[i] = 0xFFFFFFFFu;
   __syncthreads();
@@ -681,7 +700,8 @@ static void launch_compress_t(const keepkv_params &p, const keepkv_cache &src, c
              n_recent_dev, ret_idx, target, ev_idx, ui, stats);
   KEEPKV_CHECK_LAUNCH(ctx);
   if (ret_bound <= 0) return;   // nothing is kept: every entry is dropped, which select has recorded
-  launch_pdl(compact_kernel<D>, dim3((ret_bound + 63) / 64, U), dim3(256), 0, ctx.stream, p, src, dst, ret_idx, ui,
+  const int cgx = (ret_bound + 63) / 64 < 32 ? (ret_bound + 63) / 64 : 32;   // the retained count is only known on the device
+  launch_pdl(compact_kernel<D>, dim3(cgx, U), dim3(256), 0, ctx.stream, p, src, dst, ret_idx, ui,
              inv_norm);
   KEEPKV_CHECK_LAUNCH(ctx);
   launch_nominate(p, src, dst, ev_idx, ui, inv_norm, sched, nom_v, nom_si, L.nom_chunks, status_dev, ctx);

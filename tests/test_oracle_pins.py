@@ -277,7 +277,7 @@ def test_single_step_lossless_theorem_2(seed):
     if not lbar_ok:
         pytest.skip("group with lambda_bar ~ 0: the printed formula is singular there")
     assert c["stats"]["n_merged"] == n - budget          # T = -inf: every evicted entry merges
-    assert np.max(np.abs(o1 - o0)) < 1e-9                # north star asks 1e-5
+    assert np.max(np.abs(o1 - o0)) < 1e-9                # far inside the 1e-5 this invariant is specified to
     assert abs(lse1[0] - lse0[0]) < 1e-9                 # the denominator is conserved too
     # Electoral-Votes conservation: p_r = sum of members' votes
     assert c["votes"].sum() == votes.sum()
