@@ -27,13 +27,17 @@ class keepkv_params(C.Structure):
     _fields_ = [("B", C.c_int32), ("H_q", C.c_int32), ("H_kv", C.c_int32), ("d", C.c_int32), ("N_cap", C.c_int32),
                 ("period", C.c_int32), ("n_sink", C.c_int32), ("n_recent", C.c_int32), ("sm_scale", C.c_float),
                 ("ema_alpha", C.c_float), ("merge_threshold", C.c_float), ("gamma_min", C.c_float),
-                ("gamma_max", C.c_float), ("reserved", C.c_int32 * 3)]
+                ("gamma_max", C.c_float), ("flags", C.c_int32), ("reserved", C.c_int32 * 2)]
 
 
 class keepkv_cache(C.Structure):
     _fields_ = [("K", C.c_void_p), ("V", C.c_void_p), ("votes", C.c_void_p), ("lscore", C.c_void_p),
                 ("seq_len", C.c_void_p)]
 
+
+FLAG_COMPRESS_PIPELINE_ONLY = 1   # keepkv_params.flags: every unit takes the multi-kernel pipeline of keepkv_compress
+FLAG_COMPRESS_STEADY_ONLY = 2     # ... the caller promises steady-state units: only the single kernel is launched
+DEV_APPEND_FULL, DEV_TIMEOUT, DEV_NOT_STEADY = 1, 2, 4   # bits of *status_dev
 
 STATS_FIELDS = ("n_retained", "n_evicted", "n_merged", "n_below_T", "n_guard_groups", "n_groups", "max_group",
                 "reserved")
@@ -76,10 +80,10 @@ def _check(rc: int, what: str):
 
 
 def make_params(B, H_q, H_kv, d, N_cap, period=0, n_sink=4, n_recent=0, sm_scale=None, ema_alpha=0.9,
-                merge_threshold=0.8, gamma_min=0.0, gamma_max=4.0) -> keepkv_params:
+                merge_threshold=0.8, gamma_min=0.0, gamma_max=4.0, flags=0) -> keepkv_params:
     return keepkv_params(B, H_q, H_kv, d, N_cap, period, n_sink, n_recent,
                          sm_scale if sm_scale is not None else 1.0 / math.sqrt(d), ema_alpha, merge_threshold,
-                         gamma_min, gamma_max, (C.c_int32 * 3)(0, 0, 0))
+                         gamma_min, gamma_max, flags, (C.c_int32 * 2)(0, 0))
 
 
 @dataclass

@@ -9,7 +9,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libkeepkv.so")
-SOURCES = ["api.cu", "append.cu", "decode.cu", "decode_static.cu", "compress.cu", "nominate.cu", "prefill.cu"]
+SOURCES = ["api.cu", "append.cu", "decode.cu", "decode_static.cu", "compress.cu", "compress_steady.cu", "nominate.cu",
+           "prefill.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17", "-Xcompiler", "-fPIC",
               "--expt-relaxed-constexpr", "-I", os.path.join(_ROOT, "include"), "-I", CSRC]
 

@@ -7,64 +7,11 @@
 //               arithmetic wherever the tensor-core ranking is too close to call; members
 //               of each retained slot sorted into groups                         (many-to-one, App. A.2)
 //   merge    -> Eq. A.3 with the EMA estimate as score                           (lines 7-10)
-#include "common.cuh"
+#include "compress.cuh"
 
 namespace keepkv {
 
-// ------------------------------------------------------------------ block scan of 0/1 flags
-// Exclusive prefix count of `flag` over the first nw warps of the block in thread order (the other
-// warps have left the kernel); total returned through `total`.
-__device__ __forceinline__ int block_excl_count(bool flag, int *warp_tot, int &total, int nw);
-__device__ __forceinline__ int block_excl_count(bool flag, int *warp_tot, int &total) {
-  return block_excl_count(flag, warp_tot, total, (int)(blockDim.x >> 5));
-}
-__device__ __forceinline__ int block_excl_count(bool flag, int *warp_tot, int &total, int nw) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const unsigned bal = __ballot_sync(0xffffffffu, flag);
-  const int in_warp = __popc(bal & ((1u << lane) - 1u));
-  __syncthreads();  // warp_tot may still be read from the previous call
-  if (lane == 0) warp_tot[warp] = __popc(bal);
-  __syncthreads();
-  int off = 0, tot = 0;
-  for (int w = 0; w < nw; ++w) {
-    const int t = warp_tot[w];
-    if (w < warp) off += t;
-    tot += t;
-  }
-  total = tot;
-  return off + in_warp;
-}
-
-// Exclusive prefix sum of small non-negative ints over the block (thread order).
-__device__ __forceinline__ int block_excl_sum(int v, int *warp_tot, int &total, int nw) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  int x = v;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int y = __shfl_up_sync(0xffffffffu, x, o);
-    if (lane >= o) x += y;
-  }
-  __syncthreads();
-  if (lane == 31) warp_tot[warp] = x;
-  __syncthreads();
-  int off = 0, tot = 0;
-  for (int w = 0; w < nw; ++w) {
-    const int t = warp_tot[w];
-    if (w < warp) off += t;
-    tot += t;
-  }
-  total = tot;
-  return off + x - v;
-}
-
 constexpr int kWarpSelectMax = 2048;   // candidate sets up to this size are searched by one warp, without block barriers
-
-// Order-preserving map of an fp32 value to u32 (-0 folded onto +0 so equal floats give equal keys).
-__device__ __forceinline__ uint32_t ordered_key(float x) {
-  x += 0.0f;
-  const uint32_t b = __float_as_uint(x);
-  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-}
 
 // ------------------------------------------------------------------ select
 // One CTA per unit.  The keys of the whole unit live in shared memory; the heavy-hitter threshold
@@ -73,7 +20,7 @@ __device__ __forceinline__ uint32_t ordered_key(float x) {
 __global__ void __launch_bounds__(1024)
 select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int32_t *budget_dev, int budget_scalar,
               const int32_t *n_recent_dev, int32_t *ret_idx, int32_t *target, int32_t *ev_idx, UnitInfo *unit_info,
-              keepkv_stats *stats) {
+              keepkv_stats *stats, int honor_done) {
   extern __shared__ uint32_t keys[];
   __shared__ int hist[256];
   __shared__ int warp_tot[32];
@@ -82,6 +29,7 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
   const int u = blockIdx.x, b = u / p.H_kv, h = u % p.H_kv, tid = threadIdx.x;
   pdl_wait();
   pdl_trigger();
+  if (honor_done && unit_info[u].done) return;   // the single-kernel path has finished this unit
   const int len = max(0, min(src.seq_len[b], p.N_cap));
   int budget = budget_dev ? budget_dev[b] : budget_scalar;
   budget = max(0, min(budget, p.N_cap));
@@ -116,46 +64,10 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
     // few candidates (every steady-state compression): warp 0 alone finds the threshold, so the four
     // digit passes cost no block barrier
     if (tid < 32) {
-      const int lane = tid;
-      uint32_t prefix = 0, mask = 0;
-      int kr = n_heavy, cnt_last = 0;
-      for (int pass = 3; pass >= 0; --pass) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) hist[8 * lane + j] = 0;
-        __syncwarp();
-        for (int i = lo + lane; i < hi; i += 32) {
-          const uint32_t k = keys[i];
-          if ((k & mask) == prefix) atomicAdd(&hist[(k >> (8 * pass)) & 255u], 1);
-        }
-        __syncwarp();
-        int c[8], sum = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) { c[j] = hist[8 * lane + j]; sum += c[j]; }
-        int x = sum;   // becomes the count in bins of lanes >= lane
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const int y = __shfl_down_sync(0xffffffffu, x, o);
-          if (lane + o < 32) x += y;
-        }
-        const int above = x - sum;
-        const bool here = above < kr && x >= kr;
-        int cum = above, bin = 0, cnt = 0;
-        bool found = false;
-#pragma unroll
-        for (int j = 7; j >= 0; --j) {
-          if (!found) {
-            if (cum + c[j] >= kr) { bin = j; cnt = c[j]; found = true; }
-            else cum += c[j];
-          }
-        }
-        const int src_lane = __ffs(__ballot_sync(0xffffffffu, here)) - 1;
-        prefix |= (uint32_t)__shfl_sync(0xffffffffu, 8 * lane + bin, src_lane) << (8 * pass);
-        kr = __shfl_sync(0xffffffffu, kr - cum, src_lane);
-        cnt_last = __shfl_sync(0xffffffffu, cnt, src_lane);
-        mask |= 0xFFu << (8 * pass);
-        __syncwarp();
-      }
-      if (lane == 0) { s_prefix = prefix; s_kr = kr; s_cnt = cnt_last; }
+      uint32_t k_ = 0;
+      int nt_ = 0, tt_ = 0;
+      warp_radix_select(keys, lo, hi, n_heavy, hist, k_, nt_, tt_);
+      if (tid == 0) { s_prefix = k_; s_kr = nt_; s_cnt = tt_; }
     }
     __syncthreads();
     kth = s_prefix;
@@ -269,7 +181,7 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
     base_keep += tot_keep;
   }
   if (tid == 0) {
-    UnitInfo ui{len, base_keep, len - base_keep, 0, 0, 0, 0, 0};
+    UnitInfo ui{len, base_keep, len - base_keep, 0, 0, 0, 0, 0};   // done = 0
     unit_info[u] = ui;
     if (h == 0) dst_seq_len[b] = base_keep;
     keepkv_stats st;
@@ -291,7 +203,7 @@ compact_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
   constexpr int CH = D / 8;       // 16-byte chunks per row
   pdl_wait();
   pdl_trigger();
-  const int u = blockIdx.y, n_ret = unit_info[u].n_ret;
+  const int u = blockIdx.y, n_ret = unit_info[u].done ? 0 : unit_info[u].n_ret;
   for (int s0 = blockIdx.x * 64; s0 < n_ret; s0 += gridDim.x * 64) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, ch = lane & 15, sub = lane >> 4;
   const size_t base = (size_t)u * p.N_cap;
@@ -349,12 +261,6 @@ compact_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
 // Rows that need the exact chain are queued and shared out over the warps of the CTA (coalesced row
 // loads into shared memory, the sequential chains on three lanes).  The last CTA of a unit to finish
 // sorts the entries to merge by (slot, position), which makes every group contiguous and ascending.
-template <int D>
-__device__ __forceinline__ void merge_group(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
-                                            const int32_t *__restrict__ ret_idx, const int32_t *__restrict__ ev_idx,
-                                            int32_t *target, const uint32_t *gk, int beg, int n, size_t base, int u,
-                                            keepkv_stats *stats);
-constexpr float kRankEps = 1e-4f;
 constexpr int kMergeInline = 32;   // units with at most this many groups are merged by resolve_kernel itself
 constexpr int kResolveThreads = 512;
 constexpr int kResolveWarps = kResolveThreads / 32;
@@ -431,27 +337,11 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
     if (tid == 0) s_nq[par ^ 1] = 0;   // the next pass counts in the other word
     for (int q = warp; q < nq; q += kResolveWarps) {
       const int ee = q_e[q], kd = q_kind[q], ca = q_a[q], cb = kd == 1 ? q_b[q] : q_a[q];
-      __syncwarp();
-      for (int c = lane; c < D; c += 32) ke_s[warp][c] = __bfloat162float(sK[(size_t)ee * D + c]);
-      int win = -1;
-      float wu = -CUDART_INF_F;
-      {
-        for (int c = lane; c < D; c += 32) {
-          kc_s[warp][0][c] = __bfloat162float(dK[(size_t)ca * D + c]);
-          kc_s[warp][1][c] = __bfloat162float(dK[(size_t)cb * D + c]);
-        }
-        __syncwarp();
-        // lanes 0 and 1: dot and |k_c|^2 of one candidate each; lane 2: |k_e|^2
-        const float *x = ke_s[warp], *y = lane == 2 ? ke_s[warp] : kc_s[warp][lane & 1];
-        float dot = 0.f, nn = 0.f;
-        if (lane < 3)
-          for (int c = 0; c < D; ++c) { dot = fmaf(x[c], y[c], dot); nn = fmaf(y[c], y[c], nn); }
-        const float ne = __shfl_sync(0xffffffffu, nn, 2);
-        const float uu = dot / (sqrtf(ne) * sqrtf(nn));
-        const float u0 = __shfl_sync(0xffffffffu, uu, 0), u1 = __shfl_sync(0xffffffffu, uu, 1);
-        win = ca; wu = u0;
-        if (kd == 1 && (u1 > u0 || (u1 == u0 && cb < ca))) { win = cb; wu = u1; }
-      }
+      float u0, u1;
+      exact_cosines<D>(sK + (size_t)ee * D, dK + (size_t)ca * D, dK + (size_t)cb * D, ke_s[warp], &kc_s[warp][0][0], u0, u1);
+      int win = ca;
+      float wu = u0;
+      if (kd == 1 && (u1 > u0 || (u1 == u0 && cb < ca))) { win = cb; wu = u1; }
       if (lane == 0) { res_slot[q_tid[q]] = win; res_merge[q_tid[q]] = win >= 0 && wu > T; }
     }
     __syncthreads();
@@ -542,112 +432,14 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
     __syncthreads();   // the keys and group starts written above are visible to the whole CTA
     for (int g = warp; g < n_groups; g += kResolveWarps) {
       const int beg = grp_head[base + g], n = grp_head[base + g + 1] - beg;
-      merge_group<D>(p, src, dst, ret_idx, ev_idx, target, gk, beg, n, base, u, stats);
+      const int c = (int)(gk[beg] >> 16);
+      merge_group<D>(p, src, dst, c, ret_idx[base + c], [&](int t) { return ev_idx[base + (gk[beg + t] & 0xFFFFu)]; }, n,
+                     target + base, base, stats + u);
     }
   }
 }
 
 // ------------------------------------------------------------------ merge
-// One warp per group.  With a_i = ln p_i + lscore_i over the group K'_e (target first, then members
-// ascending):  omega = softmax(a),  v_r = sum omega_i v_i,  k_r = gamma * sum omega_i k_i,
-// gamma = L / lambda_bar,  L = LSE(a) - ln(sum p),  lambda_bar = sum omega_i lscore_i,  p_r = sum p,
-// lscore_r = L   (Eq. A.3 in logarithms).  `gk` holds the unit's sorted (slot << 16 | position) keys.
-template <int D>
-__device__ __forceinline__ void merge_group(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
-                                            const int32_t *__restrict__ ret_idx, const int32_t *__restrict__ ev_idx,
-                                            int32_t *target, const uint32_t *gk, int beg, int n, size_t base, int u,
-                                            keepkv_stats *stats) {
-  constexpr int EPL = D / 32;
-  const int lane = threadIdx.x & 31;
-  const float *votes = src.votes + base, *ls = src.lscore + base;
-  const __nv_bfloat16 *sK = reinterpret_cast<const __nv_bfloat16 *>(src.K) + base * D;
-  const __nv_bfloat16 *sV = reinterpret_cast<const __nv_bfloat16 *>(src.V) + base * D;
-  const int c = (int)(gk[beg] >> 16);
-  const int ci = ret_idx[base + c];
-  auto member = [&](int t) { return ev_idx[base + (gk[beg + t] & 0xFFFFu)]; };
-
-  float ka[EPL], va[EPL], lbar = 0.f, L, Ps;
-#pragma unroll
-  for (int e = 0; e < EPL; ++e) { ka[e] = 0.f; va[e] = 0.f; }
-  auto accumulate = [&](int i, float om, float lsi) {
-    lbar = fmaf(om, lsi, lbar);
-    if constexpr (EPL == 4) {
-      const uint2 kk = *reinterpret_cast<const uint2 *>(sK + (size_t)i * D + lane * 4);
-      const uint2 vv = *reinterpret_cast<const uint2 *>(sV + (size_t)i * D + lane * 4);
-      ka[0] = fmaf(om, bf16_lo(kk.x), ka[0]); ka[1] = fmaf(om, bf16_hi(kk.x), ka[1]);
-      ka[2] = fmaf(om, bf16_lo(kk.y), ka[2]); ka[3] = fmaf(om, bf16_hi(kk.y), ka[3]);
-      va[0] = fmaf(om, bf16_lo(vv.x), va[0]); va[1] = fmaf(om, bf16_hi(vv.x), va[1]);
-      va[2] = fmaf(om, bf16_lo(vv.y), va[2]); va[3] = fmaf(om, bf16_hi(vv.y), va[3]);
-    } else {
-      const uint32_t kk = *reinterpret_cast<const uint32_t *>(sK + (size_t)i * D + lane * 2);
-      const uint32_t vv = *reinterpret_cast<const uint32_t *>(sV + (size_t)i * D + lane * 2);
-      ka[0] = fmaf(om, bf16_lo(kk), ka[0]); ka[1] = fmaf(om, bf16_hi(kk), ka[1]);
-      va[0] = fmaf(om, bf16_lo(vv), va[0]); va[1] = fmaf(om, bf16_hi(vv), va[1]);
-    }
-  };
-  if (n < 32) {
-    // the usual case: lane 0 holds the target, lane t the t-th member, so that their votes and scores are
-    // fetched together and the row loads of the accumulation do not wait on one another
-    const int idx = lane == 0 ? ci : (lane <= n ? member(lane - 1) : -1);
-    const float pv = idx >= 0 ? votes[idx] : 0.f, lsv = idx >= 0 ? ls[idx] : 0.f;
-    const float a = idx >= 0 ? logf(pv) + lsv : -CUDART_INF_F;
-    const float M = warp_max(a);
-    const float Z = warp_sum(idx >= 0 ? expf(a - M) : 0.f);
-    Ps = warp_sum(pv);
-    const float Lam = M + logf(Z);
-    L = Lam - logf(Ps);
-    const float om = idx >= 0 ? expf(a - Lam) : 0.f;
-#pragma unroll 4
-    for (int t = 0; t <= n; ++t)
-      accumulate(__shfl_sync(0xffffffffu, idx, t), __shfl_sync(0xffffffffu, om, t), __shfl_sync(0xffffffffu, lsv, t));
-  } else {
-    const float a_c = logf(votes[ci]) + ls[ci];
-    float M = a_c;
-    for (int t = lane; t < n; t += 32) { const int e = member(t); M = fmaxf(M, logf(votes[e]) + ls[e]); }
-    M = warp_max(M);
-    float Z = 0.f;
-    Ps = 0.f;
-    if (lane == 0) { Z = expf(a_c - M); Ps = votes[ci]; }
-    for (int t = lane; t < n; t += 32) { const int e = member(t); Z += expf(logf(votes[e]) + ls[e] - M); Ps += votes[e]; }
-    Z = warp_sum(Z);
-    Ps = warp_sum(Ps);
-    const float Lam = M + logf(Z);
-    L = Lam - logf(Ps);
-    for (int t = -1; t < n; ++t) {
-      const int i = t < 0 ? ci : member(t);
-      const float lsi = ls[i];
-      accumulate(i, expf(logf(votes[i]) + lsi - Lam), lsi);
-    }
-  }
-  const float gamma = L / lbar;
-  const bool ok = gamma > p.gamma_min && gamma <= p.gamma_max && fabsf(lbar) >= 1e-6f;
-  if (!ok) {
-    // guard: the members are dropped after all and the target keeps the row copied by compaction
-    for (int t = lane; t < n; t += 32) target[base + member(t)] = -1;
-    if (lane == 0) { atomicAdd(&stats[u].n_guard_groups, 1); atomicAdd(&stats[u].n_groups, 1); }
-    return;
-  }
-  __nv_bfloat16 *dK = reinterpret_cast<__nv_bfloat16 *>(dst.K) + (base + c) * D;
-  __nv_bfloat16 *dV = reinterpret_cast<__nv_bfloat16 *>(dst.V) + (base + c) * D;
-  if constexpr (EPL == 4) {
-    uint2 ko, vo;
-    ko.x = pack_bf16(gamma * ka[0], gamma * ka[1]); ko.y = pack_bf16(gamma * ka[2], gamma * ka[3]);
-    vo.x = pack_bf16(va[0], va[1]); vo.y = pack_bf16(va[2], va[3]);
-    *reinterpret_cast<uint2 *>(dK + lane * 4) = ko;
-    *reinterpret_cast<uint2 *>(dV + lane * 4) = vo;
-  } else {
-    *reinterpret_cast<uint32_t *>(dK + lane * 2) = pack_bf16(gamma * ka[0], gamma * ka[1]);
-    *reinterpret_cast<uint32_t *>(dV + lane * 2) = pack_bf16(va[0], va[1]);
-  }
-  if (lane == 0) {
-    dst.votes[base + c] = Ps;
-    dst.lscore[base + c] = L;
-    atomicAdd(&stats[u].n_merged, n);
-    atomicAdd(&stats[u].n_groups, 1);
-    atomicMax(&stats[u].max_group, n);
-  }
-}
-
 // Units with many groups (the first compression of a long prompt): warps of several CTAs share them.
 // Units with few groups were already merged by resolve_kernel, which left n_groups = 0 here.
 template <int D>
@@ -664,7 +456,9 @@ merge_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_t 
   const uint32_t *gk = grp_key + (size_t)u * key_stride;
   for (int g = blockIdx.x * 8 + (threadIdx.x >> 5); g < ui.n_groups; g += gridDim.x * 8) {
     const int beg = grp_head[base + g], n = grp_head[base + g + 1] - beg;
-    merge_group<D>(p, src, dst, ret_idx, ev_idx, target, gk, beg, n, base, u, stats);
+    const int c = (int)(gk[beg] >> 16);
+    merge_group<D>(p, src, dst, c, ret_idx[base + c], [&](int t) { return ev_idx[base + (gk[beg + t] & 0xFFFFu)]; }, n,
+                   target + base, base, stats + u);
   }
 }
 
@@ -696,8 +490,14 @@ static void launch_compress_t(const keepkv_params &p, const keepkv_cache &src, c
     cudaFuncSetAttribute(resolve_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
     attr_done = true;
   }
+  // Units that evict few entries are finished by one kernel, which marks them done; the pipeline below skips those.
+  const int steady = ret_bound > 0 && !(p.flags & KEEPKV_FLAG_COMPRESS_PIPELINE_ONLY);
+  if (steady)
+    launch_compress_steady(p, src, dst, budget_dev, budget_scalar, n_recent_dev, ret_idx, target, stats, ws, L, status_dev,
+                           ctx);
+  if (p.flags & KEEPKV_FLAG_COMPRESS_STEADY_ONLY) return;   // the caller vouches for every unit
   launch_pdl(select_kernel, dim3(U), dim3(512), sel_smem, ctx.stream, p, src, dst.seq_len, budget_dev, budget_scalar,
-             n_recent_dev, ret_idx, target, ev_idx, ui, stats);
+             n_recent_dev, ret_idx, target, ev_idx, ui, stats, steady);
   KEEPKV_CHECK_LAUNCH(ctx);
   if (ret_bound <= 0) return;   // nothing is kept: every entry is dropped, which select has recorded
   const int cgx = (ret_bound + 63) / 64 < 32 ? (ret_bound + 63) / 64 : 32;   // the retained count is only known on the device

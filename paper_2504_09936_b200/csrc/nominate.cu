@@ -18,7 +18,7 @@
 // drains what is in flight, frees its tensor memory and returns.
 #include <type_traits>
 
-#include "common.cuh"
+#include "compress.cuh"
 #include "ptx.cuh"
 
 namespace keepkv {
@@ -27,7 +27,6 @@ constexpr int kNomM = 128;        // evicted rows per item (tensor-memory lanes)
 constexpr int kNomN = 256;        // retained columns per tile
 constexpr int kNomStages = 2;     // B ring
 constexpr int kNomThreads = 320;  // 10 warps
-constexpr float kNomRankEps = 1e-4f;   // closeness (in cosine units) below which the caller re-evaluates exactly
 
 template <int D>
 struct NomSmem {
@@ -42,59 +41,6 @@ struct NomSmem {
   static constexpr int kPrefix = kXchg + 2 * 128 * 5 * 4; // i32 [kMaxUnits + 1]  row-tile prefix over units
   static constexpr int kBytes = kPrefix + (kMaxUnits + 1) * 4;
 };
-
-// Running top two of one row.  Only values within `thr` of the running best are looked at: the
-// final best can only be larger, so every value within thr of the FINAL best has been inserted, and
-// (best, second) are exact among those -- which is all the caller's closeness tests use.
-// A warp holds 32 rows, and the drain is bound by the ALU pipe (compares and selects), so a group of
-// four columns is either skipped by the whole warp -- four fused multiply-adds give v - cut and the
-// sign bits are AND-ed -- or updated by the whole warp with selects only (no divergent branch).
-struct Top2 {
-  float best, second, cut, thr;
-  int bi, si;
-  __device__ __forceinline__ void init(float thr_) {
-    best = second = cut = -CUDART_INF_F;
-    thr = thr_;
-    bi = si = -1;
-  }
-  // Comparisons are strict, so among equal values the one seen first (the lower slot) stays in
-  // front, and a NaN (a zero-norm key) is never taken.
-  __device__ __forceinline__ void insert(float v, int idx) {
-    const bool p1 = v > best, p2 = v > second;
-    second = p1 ? best : fmaxf(second, v);
-    si = p1 ? bi : (p2 ? idx : si);
-    bi = p1 ? idx : bi;
-    best = fmaxf(best, v);
-  }
-  // Insert for candidates that arrive out of slot order (the other tracker of the thread): equal values
-  // go to the lower slot, as if the columns had been scanned in order.
-  __device__ __forceinline__ void insert_any(float v, int idx) {
-    const bool p1 = v > best || (v == best && idx < bi), p2 = v > second || (v == second && idx < si);
-    second = p1 ? best : (p2 ? v : second);
-    si = p1 ? bi : (p2 ? idx : si);
-    bi = p1 ? idx : bi;
-    best = p1 ? v : best;
-  }
-};
-
-// Two trackers per thread, one for the even and one for the odd columns, so that the select chains of
-// neighbouring columns do not wait on each other; both share the lower of their cuts (kept in ta.cut).
-// a_i: accumulators, w_i: inverse norms of the four columns idx..idx+3.
-// TEST = false (the first tile of an item, where nearly every group holds a new candidate for some row):
-// all four columns are inserted without the skip test, so nothing but the select chains is on the
-// critical path.
-template <bool TEST>
-__device__ __forceinline__ void offer4(Top2 &ta, Top2 &tb, float a0, float a1, float a2, float a3, const float4 w,
-                                       int idx) {
-  if (TEST) {
-    const float ncut = -ta.cut;
-    const uint32_t s = __float_as_uint(fmaf(a0, w.x, ncut)) & __float_as_uint(fmaf(a1, w.y, ncut)) &
-                       __float_as_uint(fmaf(a2, w.z, ncut)) & __float_as_uint(fmaf(a3, w.w, ncut));
-    if (!__any_sync(0xffffffffu, (int)s >= 0)) return;   // no lane has a value that is not below its cut
-  }
-  ta.insert(a0 * w.x, idx); tb.insert(a1 * w.y, idx + 1); ta.insert(a2 * w.z, idx + 2); tb.insert(a3 * w.w, idx + 3);
-  if (TEST) ta.cut = fminf(ta.best, tb.best) - ta.thr;
-}
 
 struct NomItem { int u, m_tile, chunk, t0, t1, n_ev, n_ret; };
 
@@ -336,7 +282,7 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
           if (nx < n_items) stage_rows(nit, buf ^ 1);
         }
         // values are compared before the division by |k_e|: the closeness margin scales with it
-        top.init(2.f * kNomRankEps / rowinv[buf * 128 + row]);
+        top.init(2.f * kRankEps / rowinv[buf * 128 + row]);
         topb.init(top.thr);
 
         for (int t = it.t0; t < it.t1; ++t, ++acc) {

@@ -330,3 +330,79 @@ def test_prefill_scores_windowed_initialisation(G, d, W, alpha):
         qu = np.ascontiguousarray(q64[b, h * G:(h + 1) * G].transpose(1, 0, 2))      # [W, G, d]
         ref = O.prefill_scores(P, qu, before.K[u, :n])
         check_close(after.lscore[u, :n], ref, f"prefill scores u={u}", ulps=None, max_abs=1e-3, mean_rel=1e-4)
+
+
+def _copy_params(p, **kw):
+    args = dict(B=p.B, H_q=p.H_q, H_kv=p.H_kv, d=p.d, N_cap=p.N_cap, period=p.period, n_sink=p.n_sink,
+                n_recent=p.n_recent, sm_scale=p.sm_scale, ema_alpha=p.ema_alpha, merge_threshold=p.merge_threshold,
+                gamma_min=p.gamma_min, gamma_max=p.gamma_max, flags=p.flags)
+    args.update(kw)
+    return kb.make_params(**args)
+
+
+@pytest.mark.parametrize("B,H_kv,G,d,lens,budget,n_recent,T", [
+    (2, 2, 4, 128, [1766, 1700], 1638, 1307, 0.8),          # a steady-state period: 128 resp. 62 evicted, four CTAs per unit
+    (2, 2, 4, 128, [1766, 1767], 1638, 1307, -math.inf),    # 129 evicted: that sequence takes the pipeline, the other does not
+    (1, 1, 1, 64, [900], 800, 600, -math.inf),              # one unit, eight CTAs, everything merged
+    (40, 8, 1, 64, [150 + (7 * i) % 50 for i in range(40)], 120, 90, 0.3),   # 320 units: one CTA per unit
+    (3, 2, 2, 128, [2400, 2300, 90], 2290, 100, 0.5),       # 2186 candidates: the first sequence exceeds the key table
+    (2, 1, 8, 128, [500, 300], 400, 0, 0.1),                # no recent window, one sequence within its budget
+])
+def test_compress_single_kernel_path_equals_pipeline(B, H_kv, G, d, lens, budget, n_recent, T):
+    """Units that evict few entries are finished by one kernel; with KEEPKV_FLAG_COMPRESS_PIPELINE_ONLY every
+    unit goes through the general kernels.  Both must leave the same bits everywhere, and agree with the oracle."""
+    n_cap = -(-(max(lens) + 1) // 64) * 64
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=n_cap, period=0, n_sink=4, n_recent=n_recent,
+                       merge_threshold=T)
+    src = random_cache(p, lens, seed=B * 100 + d + G, vote_max=3, scored_frac=0.9)
+    src.lscore[:, :, 20:30] = src.lscore[:, :, 20:21]                    # equal keys at the selection threshold
+    src.K[:, :, 40] = src.K[:, :, 10]                                    # exactly equal cosines: the lower slot wins
+    src.K[:, :, 41] = src.K[:, :, 10]
+    src.lscore[:, :, 40:42] = -30.0                                      # ... for two entries that are evicted
+    dst, ret, tgt, stats = _run_compress(p, src, budget)
+    dst2, ret2, tgt2, stats2 = _run_compress(_copy_params(p, flags=kb.FLAG_COMPRESS_PIPELINE_ONLY), src, budget)
+    U = B * H_kv
+    new_len = dst.seq_len.cpu().numpy()
+    assert np.array_equal(new_len, dst2.seq_len.cpu().numpy())
+    assert np.array_equal(stats, stats2)
+    for u in range(U):
+        b, h = divmod(u, H_kv)
+        n, L = int(new_len[b]), lens[b]
+        assert np.array_equal(ret[u, :n], ret2[u, :n]) and np.array_equal(tgt[u, :L], tgt2[u, :L]), u
+        for a, c in ((dst.K, dst2.K), (dst.V, dst2.V)):
+            assert torch.equal(a[b, h, :n].view(torch.int16), c[b, h, :n].view(torch.int16)), u
+        for a, c in ((dst.votes, dst2.votes), (dst.lscore, dst2.lscore)):
+            assert torch.equal(a[b, h, :n].view(torch.int32), c[b, h, :n].view(torch.int32)), u
+    hs, hd = HostCache(src), HostCache(dst)
+    for u in range(0, U, max(1, U // 8)):
+        check_compress_unit(p, u, budget, n_recent, hs, hd, ret, tgt, stats, what="single kernel")
+
+
+def test_compress_steady_only_flag_matches_and_reports_violations():
+    """KEEPKV_FLAG_COMPRESS_STEADY_ONLY launches the single kernel alone: same bits as the default call when the
+    promise holds; a unit outside the limits is reported through the device status word."""
+    B, H_kv, G, d = 3, 2, 4, 128
+    lens, budget, n_recent = [900, 870, 880], 820, 600
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=1024, period=128, n_sink=4, n_recent=n_recent,
+                       merge_threshold=0.2)
+    src = random_cache(p, lens, seed=77, vote_max=2)
+    dst, ret, tgt, stats = _run_compress(p, src, budget)
+    dst2, ret2, tgt2, stats2 = _run_compress(_copy_params(p, flags=kb.FLAG_COMPRESS_STEADY_ONLY), src, budget)
+    assert np.array_equal(stats, stats2) and np.array_equal(dst.seq_len.cpu().numpy(), dst2.seq_len.cpu().numpy())
+    for u in range(B * H_kv):
+        b, h = divmod(u, H_kv)
+        assert np.array_equal(ret[u, :budget], ret2[u, :budget]) and np.array_equal(tgt[u, :lens[b]], tgt2[u, :lens[b]])
+        for a, c in ((dst.K, dst2.K), (dst.V, dst2.V)):
+            assert torch.equal(a[b, h, :budget].view(torch.int16), c[b, h, :budget].view(torch.int16)), u
+        for a, c in ((dst.votes, dst2.votes), (dst.lscore, dst2.lscore)):
+            assert torch.equal(a[b, h, :budget].view(torch.int32), c[b, h, :budget].view(torch.int32)), u
+    # 200 evicted entries in the second sequence: the promise is broken there
+    src.seq_len[1] = 1020
+    ws, st = kb.new_workspace(p), kb.new_status()
+    kb.keepkv_compress(_copy_params(p, flags=kb.FLAG_COMPRESS_STEADY_ONLY), src, kb.Cache.empty(p), budget, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == kb.DEV_NOT_STEADY
+    with pytest.raises(kb.KeepKVError):
+        kb.keepkv_compress(_copy_params(p, flags=kb.FLAG_COMPRESS_STEADY_ONLY), src, kb.Cache.empty(p), 0, ws, st)
+    with pytest.raises(kb.KeepKVError):
+        kb.keepkv_compress(_copy_params(p, flags=3), src, kb.Cache.empty(p), budget, ws, st)
