@@ -222,7 +222,7 @@ def run_ours(args, w, rank, world):
     budget_arg = torch.from_numpy(bud).cuda() if ragged else b
     p_inc = kb.make_params(B=w.B, H_q=w.H_q, H_kv=w.H_kv, d=w.d, N_cap=n_cap, period=P, n_sink=w.n_sink,
                            n_recent=w.n_recent(), ema_alpha=0.9, merge_threshold=0.8,
-                           flags=kb.FLAG_COMPRESS_STEADY_ONLY if steady else 0)
+                           flags=kb.FLAG_COMPRESS_STEADY if steady else 0)
     nrec_arg = torch.from_numpy(nrec).cuda() if ragged else None
     K0, V0 = dev(Kb).view(w.B, w.H_kv, n_cap, w.d), dev(Vb).view(w.B, w.H_kv, n_cap, w.d)
     del Kb, Vb
@@ -454,7 +454,7 @@ def run_ours(args, w, rank, world):
             "prefill_scores_frac_hbm": pf_gbs / hbm,
             "compress_incremental_us": t_inc_compress * 1e6, "compress_incremental_gbs": inc_gbs,
             "compress_incremental_frac_hbm": inc_gbs / hbm, "merged_per_unit_incremental": m_inc,
-            "compress_incremental_path": "single kernel (KEEPKV_FLAG_COMPRESS_STEADY_ONLY)" if steady else "pipeline",
+            "compress_incremental_path": "single kernel (KEEPKV_FLAG_COMPRESS_STEADY)" if steady else "pipeline",
             "compress_full_us": t_full_compress * 1e6, "compress_full_gbs": full_gbs,
             "compress_full_frac_hbm": full_gbs / hbm, "merged_per_unit_full": m_full,
             "compress_full_gemm_tflops": gemm_flops / t_full_compress / 1e12,

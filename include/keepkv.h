@@ -52,8 +52,8 @@ typedef enum keepkv_status {
 /* bits OR-ed into *status_dev by kernels */
 #define KEEPKV_DEV_APPEND_FULL 1   /* keepkv_append: seq_len == N_cap, the token was dropped    */
 #define KEEPKV_DEV_TIMEOUT 2       /* a bounded wait inside a kernel ran out                    */
-#define KEEPKV_DEV_NOT_STEADY 4    /* keepkv_compress with KEEPKV_FLAG_COMPRESS_STEADY_ONLY met a  */
-                                   /* unit outside the steady-state limits; it was left untouched */
+#define KEEPKV_DEV_NOT_STEADY 4    /* keepkv_compress with KEEPKV_FLAG_COMPRESS_STEADY met a unit  */
+                                   /* outside the steady-state limits; it was left untouched     */
 
 typedef struct keepkv_params {
   int32_t B;                /* sequences                                                       */
@@ -73,16 +73,13 @@ typedef struct keepkv_params {
   int32_t reserved[2];      /* must be zero                                                    */
 } keepkv_params;
 
-/* keepkv_compress normally finishes a unit that evicts few entries (a steady-state compression: at
- * most 128 evicted, at most 2048 entries between the sinks and the recent window) in one kernel and
- * sends the other units through its multi-kernel pipeline; both give the same bits.  With this flag
- * every unit takes the pipeline (diagnostics, and tests that compare the two). */
-#define KEEPKV_FLAG_COMPRESS_PIPELINE_ONLY 1
-/* The caller promises that every unit is within those limits (a serving loop that compresses every P <= 128
- * steps back to a fixed budget knows this): only the single kernel is launched, which saves the launches
- * of the pipeline.  A unit that breaks the promise is left untouched (its dst rows, dst.seq_len and outputs
- * are unspecified) and KEEPKV_DEV_NOT_STEADY is raised in *status_dev.  Needs budget > 0; excludes the flag above. */
-#define KEEPKV_FLAG_COMPRESS_STEADY_ONLY 2
+/* keepkv_compress for a cache in its steady state: the caller promises that every unit evicts at most 128
+ * entries and has at most 2048 entries between the sinks and the recent window (a serving loop that
+ * compresses every P <= 128 steps back to a fixed budget knows this).  One kernel then does the whole
+ * compression instead of the general pipeline's five, with the same bits as result.  A unit that breaks the
+ * promise is left untouched (its dst rows, dst.seq_len and outputs are unspecified) and
+ * KEEPKV_DEV_NOT_STEADY is raised in *status_dev.  Needs budget > 0. */
+#define KEEPKV_FLAG_COMPRESS_STEADY 1
 
 /* One layer's cache.  Rows [seq_len[b], N_cap) of a unit are unspecified. */
 typedef struct keepkv_cache {

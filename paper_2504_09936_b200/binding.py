@@ -35,8 +35,7 @@ class keepkv_cache(C.Structure):
                 ("seq_len", C.c_void_p)]
 
 
-FLAG_COMPRESS_PIPELINE_ONLY = 1   # keepkv_params.flags: every unit takes the multi-kernel pipeline of keepkv_compress
-FLAG_COMPRESS_STEADY_ONLY = 2     # ... the caller promises steady-state units: only the single kernel is launched
+FLAG_COMPRESS_STEADY = 1   # keepkv_params.flags: the caller promises steady-state units, one kernel compresses them
 DEV_APPEND_FULL, DEV_TIMEOUT, DEV_NOT_STEADY = 1, 2, 4   # bits of *status_dev
 
 STATS_FIELDS = ("n_retained", "n_evicted", "n_merged", "n_below_T", "n_guard_groups", "n_groups", "max_group",

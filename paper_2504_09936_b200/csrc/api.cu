@@ -45,10 +45,7 @@ WsLayout ws_layout(const keepkv_params &p) {
 static int validate(const keepkv_params *p) {
   if (!p) return KEEPKV_ERR_INVALID_ARG;
   if (p->B <= 0 || p->H_q <= 0 || p->H_kv <= 0 || p->N_cap <= 0) return KEEPKV_ERR_INVALID_ARG;
-  if ((p->flags & ~(KEEPKV_FLAG_COMPRESS_PIPELINE_ONLY | KEEPKV_FLAG_COMPRESS_STEADY_ONLY)) || p->reserved[0] || p->reserved[1])
-    return KEEPKV_ERR_INVALID_ARG;
-  if ((p->flags & KEEPKV_FLAG_COMPRESS_PIPELINE_ONLY) && (p->flags & KEEPKV_FLAG_COMPRESS_STEADY_ONLY))
-    return KEEPKV_ERR_INVALID_ARG;
+  if ((p->flags & ~KEEPKV_FLAG_COMPRESS_STEADY) || p->reserved[0] || p->reserved[1]) return KEEPKV_ERR_INVALID_ARG;
   if (p->H_q % p->H_kv) return KEEPKV_ERR_UNSUPPORTED;
   const int G = p->H_q / p->H_kv;
   if (!(G == 1 || G == 2 || G == 4 || G == 8)) return KEEPKV_ERR_UNSUPPORTED;
@@ -174,7 +171,7 @@ int keepkv_compress(const keepkv_params *p, const keepkv_cache *src, const keepk
   if ((long long)p->B * p->H_kv > kMaxUnits) return KEEPKV_ERR_UNSUPPORTED;
   if (!budget_dev) {
     if (budget_scalar < 0) return KEEPKV_ERR_INVALID_ARG;
-    if ((p->flags & KEEPKV_FLAG_COMPRESS_STEADY_ONLY) && budget_scalar == 0) return KEEPKV_ERR_INVALID_ARG;
+    if ((p->flags & KEEPKV_FLAG_COMPRESS_STEADY) && budget_scalar == 0) return KEEPKV_ERR_INVALID_ARG;
     if (budget_scalar > p->N_cap || (long long)budget_scalar + p->period > p->N_cap) return KEEPKV_ERR_CAPACITY;
   }
   WsLayout L = ws_layout(*p);

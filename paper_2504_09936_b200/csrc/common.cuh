@@ -17,9 +17,8 @@ constexpr int kDecMaxCtas = 512;    // upper bound on the persistent decode grid
 constexpr int kMaxUnits = 4096;    // B * H_kv that keepkv_compress accepts (per-unit tables live in shared memory)
 constexpr int kNomChunksMax = 8;   // upper bound on the column chunks a row's similarity search is split into
 
-// n_keys / ticket: entries to merge appended so far and resolve CTAs finished (select_kernel zeroes them);
-// done: the single-kernel path of keepkv_compress has finished the unit, the general pipeline skips it
-struct UnitInfo { int len, n_ret, n_ev, n_groups, n_keys, ticket, done, pad1; };
+// n_keys / ticket: entries to merge appended so far and resolve CTAs finished (select_kernel zeroes them)
+struct UnitInfo { int len, n_ret, n_ev, n_groups, n_keys, ticket, pad0, pad1; };
 
 // Byte offsets of the arrays kept in the caller's workspace.  U = B*H_kv, N = N_cap.
 struct WsLayout {

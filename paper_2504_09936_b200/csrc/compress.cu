@@ -20,7 +20,7 @@ constexpr int kWarpSelectMax = 2048;   // candidate sets up to this size are sea
 __global__ void __launch_bounds__(1024)
 select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int32_t *budget_dev, int budget_scalar,
               const int32_t *n_recent_dev, int32_t *ret_idx, int32_t *target, int32_t *ev_idx, UnitInfo *unit_info,
-              keepkv_stats *stats, int honor_done) {
+              keepkv_stats *stats) {
   extern __shared__ uint32_t keys[];
   __shared__ int hist[256];
   __shared__ int warp_tot[32];
@@ -29,7 +29,6 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
   const int u = blockIdx.x, b = u / p.H_kv, h = u % p.H_kv, tid = threadIdx.x;
   pdl_wait();
   pdl_trigger();
-  if (honor_done && unit_info[u].done) return;   // the single-kernel path has finished this unit
   const int len = max(0, min(src.seq_len[b], p.N_cap));
   int budget = budget_dev ? budget_dev[b] : budget_scalar;
   budget = max(0, min(budget, p.N_cap));
@@ -181,7 +180,7 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
     base_keep += tot_keep;
   }
   if (tid == 0) {
-    UnitInfo ui{len, base_keep, len - base_keep, 0, 0, 0, 0, 0};   // done = 0
+    UnitInfo ui{len, base_keep, len - base_keep, 0, 0, 0, 0, 0};
     unit_info[u] = ui;
     if (h == 0) dst_seq_len[b] = base_keep;
     keepkv_stats st;
@@ -203,7 +202,7 @@ compact_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
   constexpr int CH = D / 8;       // 16-byte chunks per row
   pdl_wait();
   pdl_trigger();
-  const int u = blockIdx.y, n_ret = unit_info[u].done ? 0 : unit_info[u].n_ret;
+  const int u = blockIdx.y, n_ret = unit_info[u].n_ret;
   for (int s0 = blockIdx.x * 64; s0 < n_ret; s0 += gridDim.x * 64) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, ch = lane & 15, sub = lane >> 4;
   const size_t base = (size_t)u * p.N_cap;
@@ -490,14 +489,13 @@ static void launch_compress_t(const keepkv_params &p, const keepkv_cache &src, c
     cudaFuncSetAttribute(resolve_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
     attr_done = true;
   }
-  // Units that evict few entries are finished by one kernel, which marks them done; the pipeline below skips those.
-  const int steady = ret_bound > 0 && !(p.flags & KEEPKV_FLAG_COMPRESS_PIPELINE_ONLY);
-  if (steady)
+  if (p.flags & KEEPKV_FLAG_COMPRESS_STEADY) {   // the caller vouches for every unit: one kernel does it all
     launch_compress_steady(p, src, dst, budget_dev, budget_scalar, n_recent_dev, ret_idx, target, stats, ws, L, status_dev,
                            ctx);
-  if (p.flags & KEEPKV_FLAG_COMPRESS_STEADY_ONLY) return;   // the caller vouches for every unit
+    return;
+  }
   launch_pdl(select_kernel, dim3(U), dim3(512), sel_smem, ctx.stream, p, src, dst.seq_len, budget_dev, budget_scalar,
-             n_recent_dev, ret_idx, target, ev_idx, ui, stats, steady);
+             n_recent_dev, ret_idx, target, ev_idx, ui, stats);
   KEEPKV_CHECK_LAUNCH(ctx);
   if (ret_bound <= 0) return;   // nothing is kept: every entry is dropped, which select has recorded
   const int cgx = (ret_bound + 63) / 64 < 32 ? (ret_bound + 63) / 64 : 32;   // the retained count is only known on the device

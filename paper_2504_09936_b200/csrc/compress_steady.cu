@@ -1,6 +1,7 @@
-// keepkv_compress, single-kernel path for a steady-state compression (Algorithm 1 on a cache that is
-// only one period over its budget): a unit qualifies when it evicts at most kStEv entries and has at most
-// kStCand entries between the sinks and the recent window.  The R CTAs of a unit (grid (R, U)) each
+// keepkv_compress with KEEPKV_FLAG_COMPRESS_STEADY: Algorithm 1 in one kernel for a cache that is only one
+// period over its budget.  A unit qualifies when it evicts at most kStEv entries and has at most kStCand
+// entries between the sinks and the recent window; the others are reported and left alone.  The R CTAs of
+// a unit (grid (R, U)) each
 //   1. repeat the selection (lines 2-3): keys of the candidates in shared memory, a radix search,
 //      one ordered pass -> the kept candidates and the evicted entries as lists in shared memory;
 //   2. stream their slice of the retained slots src -> dst (line 11), 64 slots at a time.  The key rows go
@@ -105,10 +106,7 @@ steady_compress_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, cons
   }
   const int m_cand = hi - lo, n_ret = min(len, budget), n_ev = len - n_ret;
   if (m_cand > kStCand || n_ev > kStEv || n_ret > kStRet) {
-    if (r == 0 && tid == 0) {
-      unit_info[u].done = 0;   // left to the general pipeline
-      if (p.flags & KEEPKV_FLAG_COMPRESS_STEADY_ONLY) atomicOr(status_dev, KEEPKV_DEV_NOT_STEADY);   // there is none
-    }
+    if (r == 0 && tid == 0) atomicOr(status_dev, KEEPKV_DEV_NOT_STEADY);   // the promise does not hold here
     return;
   }
   const size_t base = (size_t)u * p.N_cap;
@@ -469,8 +467,6 @@ steady_compress_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, cons
     st.n_retained = n_ret; st.n_evicted = n_ev; st.n_merged = 0; st.n_below_T = n_ev - M;
     st.n_guard_groups = 0; st.n_groups = 0; st.max_group = 0; st.reserved = 0;
     stats[u] = st;
-    UnitInfo ui{len, n_ret, 0, 0, 0, 0, 1, 0};   // done: nothing is left for the general pipeline
-    unit_info[u] = ui;
     if (h == 0) dst.seq_len[b] = n_ret;
   }
   __syncthreads();

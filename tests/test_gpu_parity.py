@@ -341,16 +341,16 @@ def _copy_params(p, **kw):
 
 
 @pytest.mark.parametrize("B,H_kv,G,d,lens,budget,n_recent,T", [
-    (2, 2, 4, 128, [1766, 1700], 1638, 1307, 0.8),          # a steady-state period: 128 resp. 62 evicted, four CTAs per unit
-    (2, 2, 4, 128, [1766, 1767], 1638, 1307, -math.inf),    # 129 evicted: that sequence takes the pipeline, the other does not
-    (1, 1, 1, 64, [900], 800, 600, -math.inf),              # one unit, eight CTAs, everything merged
+    (2, 2, 4, 128, [1766, 1700], 1638, 1307, 0.8),          # a steady-state period: 128 resp. 62 evicted, several CTAs per unit
+    (2, 2, 4, 128, [1766, 1765], 1638, 1307, -math.inf),    # everything merged
+    (1, 1, 1, 64, [900], 800, 600, -math.inf),              # one unit, eight CTAs
     (40, 8, 1, 64, [150 + (7 * i) % 50 for i in range(40)], 120, 90, 0.3),   # 320 units: one CTA per unit
-    (3, 2, 2, 128, [2400, 2300, 90], 2290, 100, 0.5),       # 2186 candidates: the first sequence exceeds the key table
+    (3, 2, 2, 128, [2400, 2350, 90], 2290, 350, 0.5),       # 2046 candidates; one sequence within its budget
     (2, 1, 8, 128, [500, 300], 400, 0, 0.1),                # no recent window, one sequence within its budget
 ])
-def test_compress_single_kernel_path_equals_pipeline(B, H_kv, G, d, lens, budget, n_recent, T):
-    """Units that evict few entries are finished by one kernel; with KEEPKV_FLAG_COMPRESS_PIPELINE_ONLY every
-    unit goes through the general kernels.  Both must leave the same bits everywhere, and agree with the oracle."""
+def test_compress_steady_flag_equals_pipeline(B, H_kv, G, d, lens, budget, n_recent, T):
+    """With KEEPKV_FLAG_COMPRESS_STEADY one kernel does the whole compression of units that evict few entries.
+    It must leave the same bits everywhere as the general kernels, and agree with the oracle."""
     n_cap = -(-(max(lens) + 1) // 64) * 64
     p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=n_cap, period=0, n_sink=4, n_recent=n_recent,
                        merge_threshold=T)
@@ -359,8 +359,8 @@ def test_compress_single_kernel_path_equals_pipeline(B, H_kv, G, d, lens, budget
     src.K[:, :, 40] = src.K[:, :, 10]                                    # exactly equal cosines: the lower slot wins
     src.K[:, :, 41] = src.K[:, :, 10]
     src.lscore[:, :, 40:42] = -30.0                                      # ... for two entries that are evicted
-    dst, ret, tgt, stats = _run_compress(p, src, budget)
-    dst2, ret2, tgt2, stats2 = _run_compress(_copy_params(p, flags=kb.FLAG_COMPRESS_PIPELINE_ONLY), src, budget)
+    dst, ret, tgt, stats = _run_compress(_copy_params(p, flags=kb.FLAG_COMPRESS_STEADY), src, budget)
+    dst2, ret2, tgt2, stats2 = _run_compress(p, src, budget)
     U = B * H_kv
     new_len = dst.seq_len.cpu().numpy()
     assert np.array_equal(new_len, dst2.seq_len.cpu().numpy())
@@ -378,31 +378,33 @@ def test_compress_single_kernel_path_equals_pipeline(B, H_kv, G, d, lens, budget
         check_compress_unit(p, u, budget, n_recent, hs, hd, ret, tgt, stats, what="single kernel")
 
 
-def test_compress_steady_only_flag_matches_and_reports_violations():
-    """KEEPKV_FLAG_COMPRESS_STEADY_ONLY launches the single kernel alone: same bits as the default call when the
-    promise holds; a unit outside the limits is reported through the device status word."""
+def test_compress_steady_flag_reports_units_outside_its_limits():
+    """A unit that breaks the steady-state promise (more than 128 evicted entries, more than 2048 candidates) is
+    reported through the device status word; the others are compressed as usual."""
     B, H_kv, G, d = 3, 2, 4, 128
-    lens, budget, n_recent = [900, 870, 880], 820, 600
+    lens, budget, n_recent = [900, 1020, 880], 820, 600
     p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=1024, period=128, n_sink=4, n_recent=n_recent,
-                       merge_threshold=0.2)
+                       merge_threshold=0.2, flags=kb.FLAG_COMPRESS_STEADY)
     src = random_cache(p, lens, seed=77, vote_max=2)
-    dst, ret, tgt, stats = _run_compress(p, src, budget)
-    dst2, ret2, tgt2, stats2 = _run_compress(_copy_params(p, flags=kb.FLAG_COMPRESS_STEADY_ONLY), src, budget)
-    assert np.array_equal(stats, stats2) and np.array_equal(dst.seq_len.cpu().numpy(), dst2.seq_len.cpu().numpy())
-    for u in range(B * H_kv):
-        b, h = divmod(u, H_kv)
-        assert np.array_equal(ret[u, :budget], ret2[u, :budget]) and np.array_equal(tgt[u, :lens[b]], tgt2[u, :lens[b]])
-        for a, c in ((dst.K, dst2.K), (dst.V, dst2.V)):
-            assert torch.equal(a[b, h, :budget].view(torch.int16), c[b, h, :budget].view(torch.int16)), u
-        for a, c in ((dst.votes, dst2.votes), (dst.lscore, dst2.lscore)):
-            assert torch.equal(a[b, h, :budget].view(torch.int32), c[b, h, :budget].view(torch.int32)), u
-    # 200 evicted entries in the second sequence: the promise is broken there
-    src.seq_len[1] = 1020
+    dst = kb.Cache.empty(p)
     ws, st = kb.new_workspace(p), kb.new_status()
-    kb.keepkv_compress(_copy_params(p, flags=kb.FLAG_COMPRESS_STEADY_ONLY), src, kb.Cache.empty(p), budget, ws, st)
+    U = B * H_kv
+    ret = torch.full((U, p.N_cap), -7, dtype=torch.int32, device="cuda")
+    tgt = torch.full((U, p.N_cap), -7, dtype=torch.int32, device="cuda")
+    stats = torch.zeros(U, 8, dtype=torch.int32, device="cuda")
+    kb.keepkv_compress(p, src, dst, budget, ws, st, retained_idx=ret, target=tgt, stats=stats)
     torch.cuda.synchronize()
-    assert int(st.item()) == kb.DEV_NOT_STEADY
+    assert int(st.item()) == kb.DEV_NOT_STEADY          # sequence 1 evicts 200 entries
+    hs, hd = HostCache(src), HostCache(dst)
+    ret, tgt, stats = ret.cpu().numpy(), tgt.cpu().numpy(), stats.cpu().numpy()
+    for u in (0, 1, 4, 5):
+        check_compress_unit(_copy_params(p, flags=0), u, budget, n_recent, hs, hd, ret, tgt, stats, what="kept promise")
+    st.zero_()
+    big = kb.make_params(B=1, H_q=1, H_kv=1, d=64, N_cap=4096, period=0, n_sink=4, n_recent=100, flags=kb.FLAG_COMPRESS_STEADY)
+    kb.keepkv_compress(big, random_cache(big, [4000], seed=3), kb.Cache.empty(big), 3900, kb.new_workspace(big), st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == kb.DEV_NOT_STEADY          # 3896 candidates
     with pytest.raises(kb.KeepKVError):
-        kb.keepkv_compress(_copy_params(p, flags=kb.FLAG_COMPRESS_STEADY_ONLY), src, kb.Cache.empty(p), 0, ws, st)
+        kb.keepkv_compress(p, src, kb.Cache.empty(p), 0, ws, st)
     with pytest.raises(kb.KeepKVError):
-        kb.keepkv_compress(_copy_params(p, flags=3), src, kb.Cache.empty(p), budget, ws, st)
+        kb.keepkv_compress(_copy_params(p, flags=2), src, kb.Cache.empty(p), budget, ws, st)
