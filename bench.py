@@ -3,7 +3,7 @@
 
 One "step" is one compression period of the steady-state decode loop of a workload
 (default C2, the Llama-3-8B-shaped layer): P x (append one token, decode attention with
-score update) followed by one compression (budget + P -> budget), for every one of
+score update; one keepkv_decode_step launch) followed by one compression (budget + P -> budget), for every one of
 `--layers` independent layer caches visited round-robin, so that no call finds its
 cache in L2.  value = decode tokens/s of one layer = B * P * layers / step time.
 
@@ -289,9 +289,8 @@ def run_ours(args, w, rank, world):
             n = 0
             for t in range(P):
                 for l in range(L):
-                    kb.keepkv_append(p, cur[l], kn_all[t + 1], vn_all[t + 1], st)
-                    kb.keepkv_decode_attention(p, cur[l], q_all[t + 1], out, None, True, ws, st)
-                    n += 2
+                    kb.keepkv_decode_step(p, cur[l], q_all[t + 1], kn_all[t + 1], vn_all[t + 1], out, None, True, ws, st)
+                    n += 1
             for l in range(L):
                 kb.keepkv_compress(p_inc, cur[l], oth[l], budget_arg, ws, st, n_recent_dev=nrec_arg,
                                    stats=None if stats_t is None else stats_t[l])
@@ -333,8 +332,7 @@ def run_ours(args, w, rank, world):
         load_period()
         for t in range(P // 2):              # a real half period with fresh tokens
             for l in range(L):
-                kb.keepkv_append(p, cur[l], kn_all[t + 1], vn_all[t + 1], st)
-                kb.keepkv_decode_attention(p, cur[l], q_all[t + 1], out, None, True, ws, st)
+                kb.keepkv_decode_step(p, cur[l], q_all[t + 1], kn_all[t + 1], vn_all[t + 1], out, None, True, ws, st)
         reps = 16
         gd = torch.cuda.CUDAGraph()
         stream.synchronize()
@@ -348,8 +346,7 @@ def run_ours(args, w, rank, world):
         # ---- compression alone (incremental, budget + P -> budget), as a graph of the L calls
         for t in range(P // 2, P):
             for l in range(L):
-                kb.keepkv_append(p, cur[l], kn_all[t + 1], vn_all[t + 1], st)
-                kb.keepkv_decode_attention(p, cur[l], q_all[t + 1], out, None, True, ws, st)
+                kb.keepkv_decode_step(p, cur[l], q_all[t + 1], kn_all[t + 1], vn_all[t + 1], out, None, True, ws, st)
         gc = torch.cuda.CUDAGraph()
         stream.synchronize()
         with torch.cuda.graph(gc, stream=stream):

@@ -130,6 +130,15 @@ int keepkv_decode_attention(const keepkv_params *p, const keepkv_cache *cache, c
                             float *lse_or_null, int update_scores, void *ws, size_t ws_bytes, int32_t *status_dev,
                             void *stream);
 
+/* One decode step on device buffers in ONE launch: keepkv_append of (k_new, v_new) followed by
+ * keepkv_decode_attention of q, with exactly their results (the attention sees the fresh entry; with
+ * update_scores its score estimate becomes its first observation; lengths grow by one; a sequence already
+ * at N_cap keeps its entries, attends to them only, and raises KEEPKV_DEV_APPEND_FULL).  Arguments as for
+ * those two calls. */
+int keepkv_decode_step(const keepkv_params *p, const keepkv_cache *cache, const void *q, const void *k_new,
+                       const void *v_new, void *out, float *lse_or_null, int update_scores, void *ws, size_t ws_bytes,
+                       int32_t *status_dev, void *stream);
+
 /* Eq. 8, first case: the score estimate at the end of prefill, from the last W prompt queries
  * (W = w + 1 <= 32).  q_window: bf16 [B, H_q, W, d], oldest query first; query k sits at position
  * seq_len[b] - W + k and, the prompt being causal, scores only the entries at or before it.  For every entry
@@ -165,7 +174,7 @@ int keepkv_compress(const keepkv_params *p, const keepkv_cache *src, const keepk
 
 /* One decode step driven from HOST memory (the call a serving loop makes): copies q_host,
  * k_new_host, v_new_host (pinned or pageable host memory, shapes as above) into the device
- * staging buffers q_dev/k_new_dev/v_new_dev, runs keepkv_append and keepkv_decode_attention
+ * staging buffers q_dev/k_new_dev/v_new_dev, runs keepkv_decode_step
  * (update_scores as given) and copies the result from out_dev into out_host, all enqueued on
  * `stream`; the caller synchronises the stream before reading out_host. */
 int keepkv_decode_step_host(const keepkv_params *p, const keepkv_cache *cache, const void *q_host,

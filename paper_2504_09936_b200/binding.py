@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkeepkv.so")
 
 EXPORTS = ("keepkv_workspace_bytes", "keepkv_workspace_init", "keepkv_append", "keepkv_decode_attention",
-           "keepkv_compress", "keepkv_prefill_scores", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_status_string", "keepkv_last_cuda_error",
+           "keepkv_decode_step", "keepkv_compress", "keepkv_prefill_scores", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_status_string", "keepkv_last_cuda_error",
            "keepkv_last_launch_count")
 
 
@@ -62,6 +62,7 @@ def lib() -> C.CDLL:
         l.keepkv_workspace_init.argtypes = [pp, vp, sz, vp]
         l.keepkv_append.argtypes = [pp, pc, vp, vp, vp, vp]
         l.keepkv_decode_attention.argtypes = [pp, pc, vp, vp, vp, C.c_int, vp, sz, vp, vp]
+        l.keepkv_decode_step.argtypes = [pp, pc, vp, vp, vp, vp, vp, C.c_int, vp, sz, vp, vp]
         l.keepkv_decode_attention_static.argtypes = [pp, pc, vp, vp, vp, C.c_int, vp, vp]
         l.keepkv_prefill_scores.argtypes = [pp, pc, vp, i32, vp, vp]
         l.keepkv_compress.argtypes = [pp, pc, pc, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
@@ -147,6 +148,13 @@ def keepkv_decode_attention(p, cache: Cache, q, out, lse, update_scores: bool, w
     _check(lib().keepkv_decode_attention(C.byref(p), C.byref(cache.c()), q.data_ptr(), out.data_ptr(), _ptr(lse),
                                          int(update_scores), ws.data_ptr(), ws.numel(), status.data_ptr(),
                                          _stream(stream)), "keepkv_decode_attention")
+
+
+def keepkv_decode_step(p, cache: Cache, q, k_new, v_new, out, lse, update_scores: bool, ws, status, stream=None):
+    """keepkv_append followed by keepkv_decode_attention in one launch."""
+    _check(lib().keepkv_decode_step(C.byref(p), C.byref(cache.c()), q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(),
+                                    out.data_ptr(), _ptr(lse), int(update_scores), ws.data_ptr(), ws.numel(),
+                                    status.data_ptr(), _stream(stream)), "keepkv_decode_step")
 
 
 def keepkv_decode_attention_static(p, cache: Cache, q, out, lse, update_scores: bool, status, stream=None):

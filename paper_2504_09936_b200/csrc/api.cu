@@ -16,10 +16,10 @@ WsLayout ws_layout(const keepkv_params &p) {
   const size_t U = (size_t)p.B * p.H_kv, N = (size_t)p.N_cap, G = (size_t)(p.H_q / p.H_kv);
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-  L.counters = take(U * 4);
+  L.counters = take((U + 1) * 4);
   L.part_pool = take((size_t)kDecMaxCtas * 2 * (16 + G * (size_t)p.d) * 4);
   L.decode_bytes = off;
-  L.counter_bytes = U * 4;
+  L.counter_bytes = (U + 1) * 4;
   L.unit_info = take(U * sizeof(UnitInfo));
   L.sched = take(4 * 4);
   size_t C = (2 * 148 + U - 1) / U;
@@ -113,7 +113,7 @@ int keepkv_workspace_init(const keepkv_params *p, void *ws, size_t ws_bytes, voi
   WsLayout L = ws_layout(*p);
   if (ws_bytes < L.total) return KEEPKV_ERR_WORKSPACE;
   LaunchCtx ctx{(cudaStream_t)stream, 0, cudaSuccess};
-  ctx.err = cudaMemsetAsync((char *)ws + L.counters, 0, (size_t)p->B * p->H_kv * 4, ctx.stream);
+  ctx.err = cudaMemsetAsync((char *)ws + L.counters, 0, L.counter_bytes, ctx.stream);
   return finish(ctx);
 }
 
@@ -140,6 +140,22 @@ int keepkv_decode_attention(const keepkv_params *p, const keepkv_cache *cache, c
   if (ws_bytes < L.total) return KEEPKV_ERR_WORKSPACE;
   LaunchCtx ctx{(cudaStream_t)stream, 0, cudaSuccess};
   launch_decode(*p, *cache, q, out, lse_or_null, update_scores, (char *)ws, L, status_dev, ctx);
+  return finish(ctx);
+}
+
+int keepkv_decode_step(const keepkv_params *p, const keepkv_cache *cache, const void *q, const void *k_new,
+                       const void *v_new, void *out, float *lse_or_null, int update_scores, void *ws, size_t ws_bytes,
+                       int32_t *status_dev, void *stream) {
+  int rc = validate(p);
+  if (rc) return rc;
+  if ((rc = validate_cache(cache))) return rc;
+  if (!q || !k_new || !v_new || !out || !ws || !status_dev || !aligned(q, 16) || !aligned(k_new, 16) ||
+      !aligned(v_new, 16) || !aligned(out, 16) || !aligned(ws, 256))
+    return KEEPKV_ERR_INVALID_ARG;
+  WsLayout L = ws_layout(*p);
+  if (ws_bytes < L.total) return KEEPKV_ERR_WORKSPACE;
+  LaunchCtx ctx{(cudaStream_t)stream, 0, cudaSuccess};
+  launch_decode(*p, *cache, q, out, lse_or_null, update_scores, (char *)ws, L, status_dev, ctx, k_new, v_new);
   return finish(ctx);
 }
 
@@ -209,9 +225,8 @@ int keepkv_decode_step_host(const keepkv_params *p, const keepkv_cache *cache, c
   cp(q_dev, q_host, qb, cudaMemcpyHostToDevice);
   cp(k_new_dev, k_new_host, kb, cudaMemcpyHostToDevice);
   cp(v_new_dev, v_new_host, kb, cudaMemcpyHostToDevice);
-  if (ctx.err == cudaSuccess) launch_append(*p, *cache, k_new_dev, v_new_dev, status_dev, ctx);
   if (ctx.err == cudaSuccess)
-    launch_decode(*p, *cache, q_dev, out_dev, nullptr, update_scores, (char *)ws, L, status_dev, ctx);
+    launch_decode(*p, *cache, q_dev, out_dev, nullptr, update_scores, (char *)ws, L, status_dev, ctx, k_new_dev, v_new_dev);
   if (ctx.err == cudaSuccess) cp(out_host, out_dev, qb, cudaMemcpyDeviceToHost);
   return finish(ctx);
 }
@@ -243,10 +258,8 @@ int keepkv_decode_step_host_layers(const keepkv_params *p, const keepkv_cache *c
   cp(k_new_dev, k_new_host, kb * n_layers, cudaMemcpyHostToDevice);
   cp(v_new_dev, v_new_host, kb * n_layers, cudaMemcpyHostToDevice);
   for (int l = 0; l < n_layers && ctx.err == cudaSuccess; ++l) {
-    launch_append(*p, caches_host[l], (const char *)k_new_dev + kb * l, (const char *)v_new_dev + kb * l, status_dev, ctx);
-    if (ctx.err == cudaSuccess)
-      launch_decode(*p, caches_host[l], (const char *)q_dev + qb * l, (char *)out_dev + qb * l, nullptr, update_scores,
-                    (char *)ws, L, status_dev, ctx);
+    launch_decode(*p, caches_host[l], (const char *)q_dev + qb * l, (char *)out_dev + qb * l, nullptr, update_scores,
+                  (char *)ws, L, status_dev, ctx, (const char *)k_new_dev + kb * l, (const char *)v_new_dev + kb * l);
   }
   if (ctx.err == cudaSuccess) cp(out_host, out_dev, qb * n_layers, cudaMemcpyDeviceToHost);
   return finish(ctx);

@@ -22,7 +22,7 @@ struct UnitInfo { int len, n_ret, n_ev, n_groups, n_keys, ticket, pad0, pad1; };
 
 // Byte offsets of the arrays kept in the caller's workspace.  U = B*H_kv, N = N_cap.
 struct WsLayout {
-  size_t counters;    // i32 [U]            split-KV arrival counters (zero between calls)
+  size_t counters;    // i32 [U + 1]        split-KV arrival counters per unit, finished CTAs of a step (zero between calls)
   size_t part_pool;   // f32 [kDecMaxCtas,2,16+G*d]  partial results of units cut across CTAs (two per CTA)
   size_t unit_info;   // UnitInfo [U]       len, n_ret, n_ev, n_groups of the running compression
   size_t sched;       // i32 [4]            column-chunk count the nomination kernel settled on
@@ -56,8 +56,10 @@ int finish_call(LaunchCtx &ctx);
 // launchers (each returns cudaSuccess or the launch error and bumps ctx.launches)
 void launch_append(const keepkv_params &p, const keepkv_cache &c, const void *k_new, const void *v_new,
                    int32_t *status_dev, LaunchCtx &ctx);
+// k_new / v_new: the step's token to append inside the same launch (keepkv_decode_step), or null
 void launch_decode(const keepkv_params &p, const keepkv_cache &c, const void *q, void *out, float *lse,
-                   int update_scores, char *ws, const WsLayout &L, int32_t *status_dev, LaunchCtx &ctx);
+                   int update_scores, char *ws, const WsLayout &L, int32_t *status_dev, LaunchCtx &ctx,
+                   const void *k_new = nullptr, const void *v_new = nullptr);
 void launch_compress(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
                      const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev, int32_t *ret_idx,
                      int32_t *target, keepkv_stats *stats, char *ws, const WsLayout &L, int32_t *status_dev,

@@ -18,6 +18,12 @@
 // split into a bf16 head (A rows 0-7) and a bf16 remainder (A rows 8-15), so that P.V keeps
 // fp32-level accuracy in one MMA.  The Eq. 8 update is done one entry per lane, from the logits the
 // warp exchanges through shared memory.
+//
+// keepkv_decode_step runs the same kernel with the step's new token (Eq. 2) folded in: lengths count the fresh
+// entry from the start; the warp that owns its row patches it into the tile it has just received (and stores
+// it to the cache), so that the attention sees it.  The new lengths are published when nobody reads the old
+// ones any more: every CTA copies the lengths into shared memory first and then signs off on a counter, and
+// the last one to sign off writes them (batches beyond kSeqCache sequences: the last CTA to finish does).
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -25,6 +31,7 @@ namespace keepkv {
 
 constexpr int kDecConsumers = 4;                  // warps per CTA
 constexpr int kDecThreads = 32 * kDecConsumers;   // 128 threads leave each of them up to 255 registers at two CTAs per SM
+constexpr int kSeqCache = 256;                    // sequence lengths a CTA keeps in shared memory
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -37,7 +44,7 @@ struct TileDesc {
   int c_first;    // first CTA that holds a segment of the unit
   int nparts;     // CTAs that hold a segment of the unit
   int u_next;     // unit of the next tile of this CTA's range when this tile ends its unit, else -1
-  int pad1;
+  int fresh;      // row inside the tile of the entry this call appends, -1 if the tile does not hold it
 };
 
 template <int D>
@@ -89,7 +96,8 @@ template <int D, int G>
 __global__ void __launch_bounds__(kDecThreads, 2)
 decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, keepkv_params p,
               keepkv_cache c, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *__restrict__ out,
-              float *__restrict__ lse, int update_scores, int *counters, PartRec<D, G> *pool, int32_t *status_dev) {
+              float *__restrict__ lse, int update_scores, int *counters, PartRec<D, G> *pool, int32_t *status_dev,
+              const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new) {
   using SL = DecSmem<D>;
   constexpr int S = SL::kStages;
   constexpr int KS = D / 16;   // k-steps of the QK^T product
@@ -99,7 +107,8 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   __shared__ int s_scan[8];
   __shared__ int s_start[4];   // b, h, tile of the first tile of this CTA's range
   __shared__ volatile int s_abort;
-  __shared__ int s_last;
+  __shared__ int s_last, s_finisher;
+  __shared__ int s_seq[kSeqCache];   // the lengths as they were when the kernel started
 
   // dynamic shared memory is only guaranteed 16-byte aligned: round up to the swizzle atom
   uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -121,11 +130,22 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   pdl_trigger();
 
   // ---- the tile list: every thread sums a block of consecutive sequences, a block scan gives the offsets
-  auto tiles_of = [&](int b) { return (max(0, min(c.seq_len[b], p.N_cap)) + kTile - 1) / kTile; };
+  // entries of sequence b this call attends to: with a token to append, the fresh entry counts
+  const bool cached = p.B <= kSeqCache;   // then every thread copies the lengths of its block of sequences below
+  auto old_len = [&](int b) { return cached ? s_seq[b] : c.seq_len[b]; };
+  auto len_of = [&](int b) {
+    int n = old_len(b);
+    if (k_new && n >= 0 && n < p.N_cap) ++n;
+    return max(0, min(n, p.N_cap));
+  };
+  auto tiles_of = [&](int b) { return (len_of(b) + kTile - 1) / kTile; };
   const int per = (p.B + kDecThreads - 1) / kDecThreads;
   const int b_lo = min(p.B, tid * per), b_hi = min(p.B, b_lo + per);
   int mine = 0;
-  for (int b = b_lo; b < b_hi; ++b) mine += tiles_of(b);
+  for (int b = b_lo; b < b_hi; ++b) {
+    if (cached) s_seq[b] = c.seq_len[b];   // read back by this thread here, by the others after the barrier below
+    mine += tiles_of(b);
+  }
   int incl = mine;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
@@ -157,12 +177,24 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     }
   }
   __syncthreads();
+  if (k_new && cached && tid == kDecThreads - 1) {
+    // every CTA signs off once it holds its copy of the lengths; the last one publishes the new ones (this thread
+    // is not the producer: its wait for the counter hides behind the first tile's flight)
+    if (atomicAdd(&counters[U], 1) == grid - 1) {
+      counters[U] = 0;   // ready for the next call
+      for (int b = 0; b < p.B; ++b) {
+        const int n = s_seq[b];
+        if (n >= 0 && n < p.N_cap) c.seq_len[b] = n + 1;
+        else atomicOr(status_dev, KEEPKV_DEV_APPEND_FULL);
+      }
+    }
+  }
 
   // ------------------------------------------------------------ producer state (thread 0)
   int pb = 0, ph = 0, ptile = 0, plen = 0, ptb = 1, pit = 0;
   if (tid == 0 && ntiles > 0) {
     pb = s_start[0]; ph = s_start[1]; ptile = s_start[2];
-    plen = max(0, min(c.seq_len[pb], p.N_cap));
+    plen = len_of(pb);
     ptb = (plen + kTile - 1) / kTile;
   }
   // Issues the copies of tile `pit` of the range (thread 0 only); false if the stage never came free.
@@ -178,7 +210,11 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     d.c_first = (int)(us / chunk);
     d.nparts = (int)((ue - 1) / chunk) - d.c_first + 1;
     d.u_next = -1;
-    d.pad1 = 0;
+    d.fresh = -1;
+    if (k_new) {
+      const int old = old_len(pb);   // the fresh entry goes to row `old` of the unit
+      if (old >= 0 && old < p.N_cap && old / kTile == ptile) d.fresh = old % kTile;
+    }
     const size_t ubase = (size_t)u * p.N_cap;
     const int row = (int)ubase + ptile * kTile;
     const int this_tile = ptile;
@@ -189,7 +225,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
         ph = 0;
         do {
           ++pb;
-          plen = max(0, min(c.seq_len[pb], p.N_cap));
+          plen = len_of(pb);
           ptb = (plen + kTile - 1) / kTile;
         } while (ptb == 0);
       }
@@ -229,7 +265,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     // sequences without entries: output 0, lse = -inf
     for (int u = cta; u < U; u += grid) {
       const int b = u / p.H_kv, h = u % p.H_kv;
-      if (c.seq_len[b] <= 0) {
+      if (len_of(b) <= 0) {
         for (int idx = ctid; idx < G * D; idx += 32 * kDecConsumers)
           out[((size_t)b * p.H_q + h * G) * D + idx] = __float2bfloat16_rn(0.f);
         if (lse && ctid < G) lse[(size_t)b * p.H_q + h * G + ctid] = -CUDART_INF_F;
@@ -280,6 +316,26 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       const int i_base = d.tile * kTile + r0;     // first entry of this warp's slice
       const int n_valid = d.len - i_base;         // entries of the slice that exist (may be <= 0 or >= 32)
       const bool mine = (it & 1) == pair;
+      const bool patch = mine && d.fresh >= r0 && d.fresh < r0 + 32;
+      if (patch) {
+        // Eq. 2 inside this call: the row of the fresh entry arrived with whatever the cache held; this warp,
+        // the only one to read it, overwrites it in the tile and in the cache (one vote, no score history)
+        constexpr int CH = D / 8;
+        const size_t e = (size_t)d.u * p.N_cap + d.tile * kTile + d.fresh;
+        const int half = lane >> 4, ch = lane & 15;
+        if (ch < CH) {
+          const uint4 val = (half ? v_new : k_new)[(size_t)d.u * CH + ch];
+          *reinterpret_cast<uint4 *>(smem + stage * SL::kStride + (half ? SL::kV : SL::kK) + swz(d.fresh, ch)) = val;
+          reinterpret_cast<uint4 *>(half ? c.V : c.K)[e * CH + ch] = val;
+        }
+        if (lane == 0) {
+          reinterpret_cast<float *>(smem + stage * SL::kStride + SL::kVotes)[d.fresh] = 1.0f;
+          reinterpret_cast<float *>(smem + stage * SL::kStride + SL::kLscore)[d.fresh] = -CUDART_INF_F;
+          c.votes[e] = 1.0f;
+          if (!update_scores) c.lscore[e] = -CUDART_INF_F;   // otherwise Eq. 8 below writes the first observation
+        }
+        __syncwarp();
+      }
       if (mine && n_valid > 0) {
         const bool ragged = n_valid < 32;
         if (ragged) {
@@ -396,7 +452,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
             mma_bf16(o[2 * np + 1], pa[ks][0], pa[ks][1], pa[ks][2], pa[ks][3], b2, b3);
           }
         }
-        if (ragged) fence_proxy_async_smem();   // the zeroed V rows precede the next TMA write
+        if (ragged || patch) fence_proxy_async_smem();   // the rows written here precede the next TMA write
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&empty_bar[stage]));   // this warp is done with the stage
@@ -571,6 +627,22 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   }
 
   __syncthreads();
+  if (k_new && !cached) {
+    // the new lengths are published by the last CTA to get here: every CTA has read the old ones for the last time
+    if (tid == 0) {
+      __threadfence();
+      s_finisher = atomicAdd(&counters[U], 1) == grid - 1;
+      if (s_finisher) counters[U] = 0;   // ready for the next call
+    }
+    __syncthreads();
+    if (s_finisher) {
+      for (int b = tid; b < p.B; b += kDecThreads) {
+        const int n = c.seq_len[b];
+        if (n >= 0 && n < p.N_cap) c.seq_len[b] = n + 1;
+        else atomicOr(status_dev, KEEPKV_DEV_APPEND_FULL);
+      }
+    }
+  }
   if (s_abort) {
     // give copies still in flight a bounded chance to land before the CTA's shared memory goes away
     if (tid == 0) {
@@ -584,7 +656,8 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
 // ---------------------------------------------------------------- host side
 template <int D, int G>
 static void launch_t(const keepkv_params &p, const keepkv_cache &c, const void *q, void *out, float *lse,
-                     int update_scores, char *ws, const WsLayout &L, int32_t *status_dev, LaunchCtx &ctx) {
+                     int update_scores, char *ws, const WsLayout &L, int32_t *status_dev, const void *k_new,
+                     const void *v_new, LaunchCtx &ctx) {
   using SL = DecSmem<D>;
   constexpr size_t smem_bytes = (size_t)SL::kBytes + 1024;
   static_assert(sizeof(PartRec<D, G>) == (16 + G * D) * 4, "partial record layout");
@@ -602,22 +675,24 @@ static void launch_t(const keepkv_params &p, const keepkv_cache &c, const void *
     return;
   }
   // two CTAs per SM, never more than tiles could exist or than the partial pool holds
-  const long long max_tiles = (long long)p.B * p.H_kv * (p.N_cap / kTile);
+  const long long max_tiles = (long long)p.B * p.H_kv * (p.N_cap / kTile);   // N_cap % 64 == 0: at least one
   long long grid = 2LL * sm_count();
   if (grid > kDecMaxCtas) grid = kDecMaxCtas;
   if (grid > max_tiles) grid = max_tiles;
   launch_pdl(decode_kernel<D, G>, dim3((unsigned)grid), dim3(kDecThreads), smem_bytes, ctx.stream,
       mapK, mapV, p, c, reinterpret_cast<const __nv_bfloat16 *>(q), reinterpret_cast<__nv_bfloat16 *>(out), lse,
       update_scores, reinterpret_cast<int *>(ws + L.counters), reinterpret_cast<PartRec<D, G> *>(ws + L.part_pool),
-      status_dev);
+      status_dev, reinterpret_cast<const uint4 *>(k_new), reinterpret_cast<const uint4 *>(v_new));
   KEEPKV_CHECK_LAUNCH(ctx);
 }
 
 void launch_decode(const keepkv_params &p, const keepkv_cache &c, const void *q, void *out, float *lse,
-                   int update_scores, char *ws, const WsLayout &L, int32_t *status_dev, LaunchCtx &ctx) {
+                   int update_scores, char *ws, const WsLayout &L, int32_t *status_dev, LaunchCtx &ctx, const void *k_new,
+                   const void *v_new) {
   const int G = p.H_q / p.H_kv;
 #define KEEPKV_DISPATCH(DD, GG) \
-  if (p.d == DD && G == GG) return launch_t<DD, GG>(p, c, q, out, lse, update_scores, ws, L, status_dev, ctx);
+  if (p.d == DD && G == GG) \
+    return launch_t<DD, GG>(p, c, q, out, lse, update_scores, ws, L, status_dev, k_new, v_new, ctx);
   KEEPKV_DISPATCH(128, 1) KEEPKV_DISPATCH(128, 2) KEEPKV_DISPATCH(128, 4) KEEPKV_DISPATCH(128, 8)
   KEEPKV_DISPATCH(64, 1) KEEPKV_DISPATCH(64, 2) KEEPKV_DISPATCH(64, 4) KEEPKV_DISPATCH(64, 8)
 #undef KEEPKV_DISPATCH

@@ -267,6 +267,67 @@ def test_decode_step_host_matches_separate_calls():
     assert list(c1.seq_len.cpu()) == [101, 201]
 
 
+@pytest.mark.parametrize("G,d,update", [(4, 128, True), (1, 64, True), (8, 128, False), (2, 64, True)])
+def test_decode_step_is_append_then_decode(G, d, update):
+    """keepkv_decode_step folds Eq. 2 into the attention launch: three steps in a row give the same bits as
+    keepkv_append + keepkv_decode_attention, for lengths at tile edges, an empty and a full sequence."""
+    H_kv, n_cap = 2, 256
+    lens = [0, 63, 64, 127, 128, 200, 255, 256, 1]
+    B = len(lens)
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=n_cap)
+    c1 = random_cache(p, lens, seed=G + d, vote_max=2, scored_frac=0.8)
+    c2 = kb.Cache(c1.K.clone(), c1.V.clone(), c1.votes.clone(), c1.lscore.clone(), c1.seq_len.clone())
+    ws, st1, st2 = kb.new_workspace(p), kb.new_status(), kb.new_status()
+    rng = np.random.default_rng(9)
+    mk = lambda *s: f32_to_dev_bf16(rng.standard_normal(s).astype(np.float32))
+    for step in range(3):
+        q, kn, vn = mk(B, H_kv * G, d), mk(B, H_kv, d), mk(B, H_kv, d)
+        o1, o2 = torch.empty_like(q), torch.empty_like(q)
+        l1 = torch.empty(B, H_kv * G, dtype=torch.float32, device="cuda")
+        l2 = torch.empty_like(l1)
+        kb.keepkv_decode_step(p, c1, q, kn, vn, o1, l1, update, ws, st1)
+        kb.keepkv_append(p, c2, kn, vn, st2)
+        kb.keepkv_decode_attention(p, c2, q, o2, l2, update, ws, st2)
+        torch.cuda.synchronize()
+        assert torch.equal(c1.seq_len, c2.seq_len), step
+        assert torch.equal(o1.view(torch.int16), o2.view(torch.int16)) and torch.equal(l1.view(torch.int32), l2.view(torch.int32)), step
+        n = c2.seq_len.cpu().numpy()
+        for b in range(B):
+            k = int(n[b])
+            for x, y in ((c1.K, c2.K), (c1.V, c2.V)):
+                assert torch.equal(x[b, :, :k].view(torch.int16), y[b, :, :k].view(torch.int16)), (step, b)
+            for x, y in ((c1.votes, c2.votes), (c1.lscore, c2.lscore)):
+                assert torch.equal(x[b, :, :k].view(torch.int32), y[b, :, :k].view(torch.int32)), (step, b)
+    assert list(c1.seq_len.cpu().numpy()) == [3, 66, 67, 130, 131, 203, 256, 256, 4]
+    assert int(st1.item()) == kb.DEV_APPEND_FULL and int(st2.item()) == kb.DEV_APPEND_FULL
+
+
+def test_decode_step_many_sequences():
+    """More sequences than a CTA caches lengths for: the new lengths are published by the last CTA to finish."""
+    B, H_kv, G, d, n_cap = 300, 1, 2, 64, 128
+    lens = [(37 * i) % 129 for i in range(B)]          # 0 .. 128, some full
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=n_cap)
+    c1 = random_cache(p, lens, seed=21)
+    c2 = kb.Cache(c1.K.clone(), c1.V.clone(), c1.votes.clone(), c1.lscore.clone(), c1.seq_len.clone())
+    ws, st1, st2 = kb.new_workspace(p), kb.new_status(), kb.new_status()
+    rng = np.random.default_rng(10)
+    mk = lambda *s: f32_to_dev_bf16(rng.standard_normal(s).astype(np.float32))
+    for step in range(2):
+        q, kn, vn = mk(B, H_kv * G, d), mk(B, H_kv, d), mk(B, H_kv, d)
+        o1, o2 = torch.empty_like(q), torch.empty_like(q)
+        kb.keepkv_decode_step(p, c1, q, kn, vn, o1, None, True, ws, st1)
+        kb.keepkv_append(p, c2, kn, vn, st2)
+        kb.keepkv_decode_attention(p, c2, q, o2, None, True, ws, st2)
+        torch.cuda.synchronize()
+        assert torch.equal(c1.seq_len, c2.seq_len) and torch.equal(o1.view(torch.int16), o2.view(torch.int16)), step
+    n = c2.seq_len.cpu().numpy()
+    for b in range(B):
+        k = int(n[b])
+        assert torch.equal(c1.K[b, :, :k].view(torch.int16), c2.K[b, :, :k].view(torch.int16)), b
+        assert torch.equal(c1.lscore[b, :, :k].view(torch.int32), c2.lscore[b, :, :k].view(torch.int32)), b
+    assert int(st1.item()) == int(st2.item()) == kb.DEV_APPEND_FULL
+
+
 def test_decode_step_host_layers_matches_per_layer_calls():
     p = kb.make_params(B=2, H_q=8, H_kv=2, d=128, N_cap=256)
     Lr = 3
