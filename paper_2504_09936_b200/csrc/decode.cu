@@ -7,6 +7,13 @@
 // finished by the last of those CTAs to arrive (one ticket per unit), in a fixed order, so results
 // are bit-reproducible.
 //
+// With a moderate number of units (a dozen to one per SM) the grid is launched as clusters of S CTAs, one
+// cluster per unit, S * units <= two CTAs per SM.  If the units are about equally long -- every steady-state
+// step -- a cluster splits its unit's tiles evenly, and the S partial results meet in distributed shared
+// memory instead of global memory: each CTA leaves its partial in its own shared memory, a cluster barrier,
+// each CTA folds 1/S of the outputs from its peers' memories (in rank order), a second barrier.  Ragged
+// batches fall back to the equal ranges over the whole list, whatever the launch shape.
+//
 // One CTA = 4 warps.  Thread 0 also walks the range as producer: per tile it issues TMA loads of the
 // K and V tiles (128-byte swizzled boxes), bulk copies of the tile's votes and lscore, and a small
 // descriptor, into a ring of shared-memory stages guarded by full/empty mbarriers, two tiles ahead
@@ -104,7 +111,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   constexpr int NT = D / 8;    // 8-channel n-tiles of the PV product
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[S], empty_bar[S];
-  __shared__ int s_scan[8];
+  __shared__ int s_scan[8], s_tbmax[4];
   __shared__ int s_start[4];   // b, h, tile of the first tile of this CTA's range
   __shared__ volatile int s_abort;
   __shared__ int s_last, s_finisher;
@@ -141,18 +148,22 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   auto tiles_of = [&](int b) { return (len_of(b) + kTile - 1) / kTile; };
   const int per = (p.B + kDecThreads - 1) / kDecThreads;
   const int b_lo = min(p.B, tid * per), b_hi = min(p.B, b_lo + per);
-  int mine = 0;
+  int mine = 0, tb_max = 0;
   for (int b = b_lo; b < b_hi; ++b) {
     if (cached) s_seq[b] = c.seq_len[b];   // read back by this thread here, by the others after the barrier below
-    mine += tiles_of(b);
+    const int tb = tiles_of(b);
+    mine += tb;
+    tb_max = max(tb_max, tb);
   }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) tb_max = max(tb_max, __shfl_xor_sync(0xffffffffu, tb_max, o));
   int incl = mine;
 #pragma unroll
   for (int o = 1; o < 32; o <<= 1) {
     const int y = __shfl_up_sync(0xffffffffu, incl, o);
     if (lane >= o) incl += y;
   }
-  if (lane == 31) s_scan[warp] = incl;
+  if (lane == 31) { s_scan[warp] = incl; s_tbmax[warp] = tb_max; }
   __syncthreads();
   int before = incl - mine, total_b = 0;
   for (int w = 0; w < kDecConsumers; ++w) {
@@ -161,9 +172,22 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   }
   const long long T = (long long)total_b * p.H_kv;
   const int chunk = (int)((T + grid - 1) / grid);
-  const long long g0 = min(T, (long long)cta * chunk), g1 = min(T, g0 + chunk);
+  // one cluster per unit, if the launch has them and no sequence is much longer than the average
+  const int csize = (int)cluster_nctarank(), crank = (int)cluster_ctarank();
+  tb_max = max(max(s_tbmax[0], s_tbmax[1]), max(s_tbmax[2], s_tbmax[3]));
+  const bool aligned = csize > 1 && grid == U * csize && total_b > 0 && (long long)tb_max * p.B * 4 <= 5LL * total_b;
+  long long g0 = min(T, (long long)cta * chunk), g1 = min(T, g0 + chunk);
+  int tb_unit = 0;   // aligned: tiles of this cluster's unit
+  if (aligned) {
+    const int ub = (cta / csize) / p.H_kv;
+    tb_unit = tiles_of(ub);
+    const int t_lo = (int)((long long)crank * tb_unit / csize), t_hi = (int)((long long)(crank + 1) * tb_unit / csize);
+    g0 = t_lo;   // only the tile count matters below
+    g1 = t_hi;
+    if (tid == 0 && t_hi > t_lo) { s_start[0] = ub; s_start[1] = (cta / csize) % p.H_kv; s_start[2] = t_lo; }
+  }
   const int ntiles = (int)(g1 - g0);
-  if (ntiles > 0 && (long long)before * p.H_kv <= g0 && g0 < (long long)(before + mine) * p.H_kv) {
+  if (!aligned && ntiles > 0 && (long long)before * p.H_kv <= g0 && g0 < (long long)(before + mine) * p.H_kv) {
     long long at = (long long)before * p.H_kv;
     for (int b = b_lo; b < b_hi; ++b) {
       const int tb = tiles_of(b);
@@ -209,6 +233,10 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     d.flags = ((it == 0 || ptile == 0) ? 1 : 0) | ((it == ntiles - 1 || ptile == ptb - 1) ? 2 : 0);
     d.c_first = (int)(us / chunk);
     d.nparts = (int)((ue - 1) / chunk) - d.c_first + 1;
+    if (aligned) {   // every CTA of the cluster holds a partial (possibly empty) unless the unit is a single tile
+      d.c_first = 0;
+      d.nparts = ptb == 1 ? 1 : csize;
+    }
     d.u_next = -1;
     d.fresh = -1;
     if (k_new) {
@@ -501,6 +529,10 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
               const size_t qo = (size_t)b * p.H_q + h * G + gg;
               out[qo * D + j] = __float2bfloat16_rn(Ls > 0.f ? a / Ls : 0.f);
               if (lse && j == 0) lse[qo] = Ls > 0.f ? (M + lg2f(Ls)) * kLn2 : -CUDART_INF_F;
+            } else if (aligned) {   // this CTA's partial stays in its shared memory (the ring is idle by now)
+              float *xr = reinterpret_cast<float *>(smem);
+              xr[16 + gg * D + j] = a;
+              if (j == 0) { xr[gg] = M; xr[8 + gg] = Ls; }
             } else {
               rec->acc[gg * D + j] = a;
               if (j == 0) { rec->m[gg] = M; rec->l[gg] = Ls; }
@@ -508,7 +540,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
           }
           asm volatile("bar.sync 1, 128;" ::: "memory");
         }
-        if (!whole) {
+        if (!whole && !aligned) {
           // ---- the last CTA of the unit to arrive merges the partials, in CTA order
           __threadfence();
           asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -627,6 +659,43 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   }
 
   __syncthreads();
+  if (aligned && tb_unit > 1) {
+    // ---- the cluster folds its unit's partials through distributed shared memory: [m[8], l[8], acc[G*D]] per CTA
+    float *xr = reinterpret_cast<float *>(smem);
+    if (ntiles == 0 && tid < 8) { xr[tid] = -CUDART_INF_F; xr[8 + tid] = 0.f; }   // no tiles here: an empty partial
+    cluster_sync_all();
+    const int u = cta / csize, b = u / p.H_kv, h = u % p.H_kv;
+    const int per_cta = G * D / csize;   // outputs this CTA folds
+    const uint32_t xr_addr = smem_u32(xr);
+    for (int k = tid; k < per_cta; k += kDecThreads) {
+      const int idx = crank * per_cta + k, gg = idx / D, j = idx % D;
+      float pm[8], pl[8], pa_[8];
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        pm[r] = -CUDART_INF_F; pl[r] = 0.f; pa_[r] = 0.f;
+        if (r < csize) {
+          const uint32_t ra = mapa_shared(xr_addr, (uint32_t)r);
+          pm[r] = ld_shared_cluster_f32(ra + gg * 4);
+          pl[r] = ld_shared_cluster_f32(ra + (8 + gg) * 4);
+          pa_[r] = ld_shared_cluster_f32(ra + (16 + idx) * 4);
+        }
+      }
+      float M = pm[0];
+#pragma unroll
+      for (int r = 1; r < 8; ++r) M = fmaxf(M, pm[r]);
+      float Ls = 0.f, a = 0.f;
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        const float f = pm[r] > -CUDART_INF_F ? ex2f(pm[r] - M) : 0.f;
+        Ls = fmaf(f, pl[r], Ls);
+        a = fmaf(f, pa_[r], a);
+      }
+      const size_t qo = (size_t)b * p.H_q + h * G + gg;
+      out[qo * D + j] = __float2bfloat16_rn(Ls > 0.f ? a / Ls : 0.f);
+      if (lse && j == 0) lse[qo] = Ls > 0.f ? (M + lg2f(Ls)) * kLn2 : -CUDART_INF_F;
+    }
+    cluster_sync_all();   // nobody leaves while a peer still reads its shared memory
+  }
   if (k_new && !cached) {
     // the new lengths are published by the last CTA to get here: every CTA has read the old ones for the last time
     if (tid == 0) {
@@ -678,6 +747,21 @@ static void launch_t(const keepkv_params &p, const keepkv_cache &c, const void *
   const long long max_tiles = (long long)p.B * p.H_kv * (p.N_cap / kTile);   // N_cap % 64 == 0: at least one
   long long grid = 2LL * sm_count();
   if (grid > kDecMaxCtas) grid = kDecMaxCtas;
+  // a dozen units to one per SM: one cluster per unit, as many CTAs per cluster as two per SM allow
+  const int U = p.B * p.H_kv;
+  int cs = 1;
+  if (U >= 12 && 2 * U <= grid && p.N_cap / kTile >= 2) {
+    cs = 8;
+    while (cs > 1 && (long long)U * cs > grid) cs >>= 1;
+  }
+  if (cs > 1) {
+    launch_pdl_cluster(decode_kernel<D, G>, dim3((unsigned)(U * cs)), dim3(kDecThreads), smem_bytes, ctx.stream, cs,
+        mapK, mapV, p, c, reinterpret_cast<const __nv_bfloat16 *>(q), reinterpret_cast<__nv_bfloat16 *>(out), lse,
+        update_scores, reinterpret_cast<int *>(ws + L.counters), reinterpret_cast<PartRec<D, G> *>(ws + L.part_pool),
+        status_dev, reinterpret_cast<const uint4 *>(k_new), reinterpret_cast<const uint4 *>(v_new));
+    KEEPKV_CHECK_LAUNCH(ctx);
+    return;
+  }
   if (grid > max_tiles) grid = max_tiles;
   launch_pdl(decode_kernel<D, G>, dim3((unsigned)grid), dim3(kDecThreads), smem_bytes, ctx.stream,
       mapK, mapV, p, c, reinterpret_cast<const __nv_bfloat16 *>(q), reinterpret_cast<__nv_bfloat16 *>(out), lse,

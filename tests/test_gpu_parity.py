@@ -53,6 +53,30 @@ def test_decode_small_shapes_ragged(G, d):
         assert np.array_equal(ls_after[u, n:], ls_before[u, n:], equal_nan=True)
 
 
+@pytest.mark.parametrize("B,H_kv,G,d,lens", [
+    (4, 4, 8, 128, [130, 128, 129, 131]),       # 16 units, clusters of 8, three tiles per unit: empty ranks
+    (8, 2, 4, 128, [1700 + i for i in range(8)]),   # 16 units, 27 tiles each
+    (16, 4, 1, 64, [64] * 16),                  # 64 units of exactly one tile: no exchange at all
+    (16, 4, 2, 64, [65 + 3 * i for i in range(16)]),   # 64 units, clusters of 4, two or three tiles
+    (37, 4, 4, 128, [300] * 36 + [0]),          # 148 units, clusters of 2, one empty sequence
+])
+def test_decode_one_cluster_per_unit(B, H_kv, G, d, lens):
+    """Batches of a dozen to 148 units with similar lengths: a thread-block cluster per unit, whose partial
+    results meet in distributed shared memory.  Same checks as for the split over the whole tile list."""
+    n_cap = -(-(max(lens) + 2) // 64) * 64
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=max(n_cap, 128), ema_alpha=0.9)
+    cache = random_cache(p, lens, seed=B + G + d, vote_max=4, scored_frac=0.6)
+    q = _q(p, 11)
+    hc = HostCache(cache)
+    out, lse = _run_decode(p, cache, q, True)
+    ls_after = to_f64(cache.lscore).reshape(B * H_kv, -1)
+    q64, o64, l64 = to_f64(q), to_f64(out), to_f64(lse)
+    for u in range(0, B * H_kv, max(1, B * H_kv // 24)):
+        check_decode_unit(p, u, hc, q64, o64, l64, ls_after, what=f"cluster G={G} d={d}")
+    out2, lse2 = _run_decode(p, cache, q, False)      # the estimate has moved, the attention has not
+    assert torch.equal(out.view(torch.int16), out2.view(torch.int16)) and torch.equal(lse.view(torch.int32), lse2.view(torch.int32))
+
+
 def test_decode_without_score_update_leaves_lscore():
     p = kb.make_params(B=2, H_q=8, H_kv=2, d=128, N_cap=256)
     cache = random_cache(p, [256, 100], seed=3)
