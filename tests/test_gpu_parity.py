@@ -54,14 +54,14 @@ def test_decode_small_shapes_ragged(G, d):
 
 
 @pytest.mark.parametrize("B,H_kv,G,d,lens", [
-    (4, 4, 8, 128, [130, 128, 129, 131]),       # 16 units, clusters of 8, three tiles per unit: empty ranks
-    (8, 2, 4, 128, [1700 + i for i in range(8)]),   # 16 units, 27 tiles each
+    (6, 4, 8, 128, [130, 128, 129, 131, 130, 129]),   # 24 units, clusters of 8, three tiles per unit: empty ranks
+    (6, 4, 4, 128, [1700 + i for i in range(6)]),   # 24 units, 27 tiles each
     (16, 4, 1, 64, [64] * 16),                  # 64 units of exactly one tile: no exchange at all
     (16, 4, 2, 64, [65 + 3 * i for i in range(16)]),   # 64 units, clusters of 4, two or three tiles
     (37, 4, 4, 128, [300] * 36 + [0]),          # 148 units, clusters of 2, one empty sequence
 ])
 def test_decode_one_cluster_per_unit(B, H_kv, G, d, lens):
-    """Batches of a dozen to 148 units with similar lengths: a thread-block cluster per unit, whose partial
+    """Batches of two dozen to 148 units with similar lengths: a thread-block cluster per unit, whose partial
     results meet in distributed shared memory.  Same checks as for the split over the whole tile list."""
     n_cap = -(-(max(lens) + 2) // 64) * 64
     p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=max(n_cap, 128), ema_alpha=0.9)
