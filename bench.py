@@ -459,7 +459,7 @@ def run_ours(args, w, rank, world):
     }
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
-            period_s, cores, desc, _, _ = oracle_period_time(w, w.U, 32)
+            period_s, cores, desc, _, _ = oracle_period_time(w, w.U, min(w.period, 128))
             line["cpu_baseline"] = {"value": w.B * P / period_s, "unit": UNIT, "cores": cores, "kind": "oracle",
                                     "sample": desc}
         print(json.dumps(line))
