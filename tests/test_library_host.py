@@ -64,3 +64,22 @@ def test_calls_reject_null_and_capacity_before_any_launch(lib):
     assert lib.keepkv_compress(C.byref(p), C.byref(fake), C.byref(fake2), None, 51, None, None, None, None, 256, 16,
                                256, None) == -4
     assert lib.keepkv_decode_attention(C.byref(p), C.byref(fake), 256, 256, None, 0, 256, 16, 256, None) == -4
+
+
+def test_flags_and_decode_step_arguments_are_checked_before_any_launch(lib):
+    fake = kb.keepkv_cache(256, 512, 768, 1024, 1280)      # non-null, aligned, never dereferenced
+    fake2 = kb.keepkv_cache(2560, 5120, 7680, 10240, 12800)
+    sz = C.c_size_t()
+    # unknown flag bits are rejected by every call that takes the parameters
+    bad = kb.make_params(B=1, H_q=8, H_kv=2, d=64, N_cap=576, period=32, flags=2)
+    assert lib.keepkv_workspace_bytes(C.byref(bad), C.byref(sz)) == -1
+    # the steady-state promise needs something to keep
+    st = kb.make_params(B=1, H_q=8, H_kv=2, d=64, N_cap=576, period=32, flags=kb.FLAG_COMPRESS_STEADY)
+    assert lib.keepkv_workspace_bytes(C.byref(st), C.byref(sz)) == 0
+    assert lib.keepkv_compress(C.byref(st), C.byref(fake), C.byref(fake2), None, 0, None, None, None, None, 256, 1 << 40,
+                               256, None) == -1
+    # keepkv_decode_step: null or misaligned token rows, short workspace
+    p = kb.make_params(B=1, H_q=8, H_kv=2, d=64, N_cap=576, period=32)
+    assert lib.keepkv_decode_step(C.byref(p), C.byref(fake), 256, None, 256, 256, None, 0, 256, 1 << 40, 256, None) == -1
+    assert lib.keepkv_decode_step(C.byref(p), C.byref(fake), 256, 264, 256, 256, None, 0, 256, 1 << 40, 256, None) == -1
+    assert lib.keepkv_decode_step(C.byref(p), C.byref(fake), 256, 256, 256, 256, None, 0, 256, 16, 256, None) == -4
