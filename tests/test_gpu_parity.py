@@ -212,6 +212,44 @@ def test_single_step_lossless_on_gpu():
     check_close(to_f64(lse1), to_f64(lse0), "lossless lse", ulps=None, max_abs=2e-2, mean_rel=1e-3)
 
 
+def test_periodic_lossless_protocol_on_gpu():
+    """The periodic mode of Section 1 through the library: the complete cache is kept aside and grows with
+    every step; every P steps it is scored by the current query (alpha = 0), compressed from scratch into
+    the working cache (T = -inf: everything merged) and the working cache must then reproduce the complete
+    cache's attention output for that query (Theorem 2, G = 1, to bf16 storage resolution).  Between two
+    compressions the steps run on the working cache."""
+    B, H, d, P, budget, n_cap = 2, 4, 128, 8, 96, 512
+    p = kb.make_params(B=B, H_q=H, H_kv=H, d=d, N_cap=n_cap, period=P, n_sink=4, n_recent=40, ema_alpha=0.0,
+                       merge_threshold=-math.inf, gamma_min=-math.inf, gamma_max=math.inf)
+    full = random_cache(p, [400, 250], seed=33, scored_frac=0.0, scale=0.3)
+    full.K.add_(0.5)       # logits near +1.4 for the constant query below: away from the rescale factor's singular point
+    ws, st = kb.new_workspace(p), kb.new_status()
+    rng = np.random.default_rng(34)
+    q = torch.full((B, H, d), 0.25, dtype=torch.bfloat16, device="cuda")
+    work = None
+    for period in range(3):
+        out_full, lse_full = _run_decode(p, full, q, True)             # scores of the complete cache for this query
+        work, ret, tgt, stats = _run_compress(p, full, budget)
+        assert np.all(stats[:, 2] == stats[:, 1])                       # every evicted entry merged
+        assert list(work.seq_len.cpu().numpy()) == [budget, budget]
+        out_work, lse_work = _run_decode(p, work, q, False)
+        check_close(to_f64(out_work), to_f64(out_full), f"period {period} out", ulps=None, max_abs=2e-2, mean_rel=2e-2)
+        check_close(to_f64(lse_work), to_f64(lse_full), f"period {period} lse", ulps=None, max_abs=2e-2, mean_rel=1e-3)
+        hw = HostCache(work)
+        n_full = full.seq_len.cpu().numpy()
+        for u in range(B * H):
+            assert hw.votes[u, :budget].sum() == n_full[u // H]         # Electoral Votes are conserved
+        for t in range(P):                                              # the steps between two compressions
+            kn = f32_to_dev_bf16((rng.standard_normal((B, H, d)) * 0.3 + 0.5).astype(np.float32))
+            vn = f32_to_dev_bf16(rng.standard_normal((B, H, d)).astype(np.float32))
+            o = torch.empty_like(q)
+            kb.keepkv_append(p, full, kn, vn, st)
+            kb.keepkv_decode_step(p, work, q, kn, vn, o, None, True, ws, st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        assert list(work.seq_len.cpu().numpy()) == [budget + P, budget + P]
+
+
 def test_c1_protocol_free_running():
     """Config C1 end to end: score the prompt, compress 512 -> 51, then 32 x (append, decode) on both
     sides independently; final compression checked teacher-forced."""
