@@ -364,6 +364,39 @@ def test_decode_step_is_append_then_decode(G, d, update):
     assert int(st1.item()) == kb.DEV_APPEND_FULL and int(st2.item()) == kb.DEV_APPEND_FULL
 
 
+def test_decode_step_one_cluster_per_unit():
+    """keepkv_decode_step on a batch that runs one cluster per unit (24 units), with lengths around tile edges so
+    that the fresh row opens a new tile for some sequences: same bits as append + decode, and the oracle's output."""
+    B, H_kv, G, d, n_cap = 6, 4, 4, 128, 256
+    lens = [127, 128, 129, 128, 127, 126]
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=n_cap)
+    c1 = random_cache(p, lens, seed=5, vote_max=3, scored_frac=0.7)
+    c2 = kb.Cache(c1.K.clone(), c1.V.clone(), c1.votes.clone(), c1.lscore.clone(), c1.seq_len.clone())
+    ws, st = kb.new_workspace(p), kb.new_status()
+    rng = np.random.default_rng(12)
+    mk = lambda *s: f32_to_dev_bf16(rng.standard_normal(s).astype(np.float32))
+    for step in range(3):
+        q, kn, vn = mk(B, H_kv * G, d), mk(B, H_kv, d), mk(B, H_kv, d)
+        o1, o2 = torch.empty_like(q), torch.empty_like(q)
+        l1 = torch.empty(B, H_kv * G, dtype=torch.float32, device="cuda")
+        l2 = torch.empty_like(l1)
+        kb.keepkv_decode_step(p, c1, q, kn, vn, o1, l1, True, ws, st)
+        kb.keepkv_append(p, c2, kn, vn, st)
+        hc = HostCache(c2)
+        kb.keepkv_decode_attention(p, c2, q, o2, l2, True, ws, st)
+        torch.cuda.synchronize()
+        assert torch.equal(c1.seq_len, c2.seq_len), step
+        assert torch.equal(o1.view(torch.int16), o2.view(torch.int16)) and torch.equal(l1.view(torch.int32), l2.view(torch.int32)), step
+        assert torch.equal(c1.K.view(torch.int16), c2.K.view(torch.int16)) and torch.equal(c1.votes, c2.votes), step
+        n = c2.seq_len.cpu().numpy()
+        for b in range(B):
+            assert torch.equal(c1.lscore[b, :, :n[b]].view(torch.int32), c2.lscore[b, :, :n[b]].view(torch.int32)), (step, b)
+        ls_after = to_f64(c1.lscore).reshape(B * H_kv, -1)
+        for u in range(0, B * H_kv, 5):
+            check_decode_unit(p, u, hc, to_f64(q), to_f64(o1), to_f64(l1), ls_after, what=f"step {step}")
+    assert int(st.item()) == 0
+
+
 def test_decode_step_many_sequences():
     """More sequences than a CTA caches lengths for: the new lengths are published by the last CTA to finish."""
     B, H_kv, G, d, n_cap = 300, 1, 2, 64, 128
