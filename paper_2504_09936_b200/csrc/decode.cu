@@ -686,9 +686,13 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       float Ls = 0.f, a = 0.f;
 #pragma unroll
       for (int r = 0; r < 8; ++r) {
-        const float f = pm[r] > -CUDART_INF_F ? ex2f(pm[r] - M) : 0.f;
-        Ls = fmaf(f, pl[r], Ls);
-        a = fmaf(f, pa_[r], a);
+        // a CTA without tiles published m = -inf and nothing else: its numerators are whatever its shared
+        // memory held (0 * NaN would poison the sum), so an empty partial is skipped, not weighted by zero
+        if (pm[r] > -CUDART_INF_F) {
+          const float f = ex2f(pm[r] - M);
+          Ls = fmaf(f, pl[r], Ls);
+          a = fmaf(f, pa_[r], a);
+        }
       }
       const size_t qo = (size_t)b * p.H_q + h * G + gg;
       out[qo * D + j] = __float2bfloat16_rn(Ls > 0.f ? a / Ls : 0.f);
