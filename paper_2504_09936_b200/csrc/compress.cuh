@@ -209,7 +209,11 @@ struct Top2 {
 };
 
 // Two trackers per thread, one for the even and one for the odd columns, so that the select chains of
-// neighbouring columns do not wait on each other; both share the lower of their cuts (kept in ta.cut).
+// neighbouring columns do not wait on each other.  Both share one cut (kept in ta.cut), taken from the larger of
+// their two bests: the row's final best is at least that, so a value below the cut cannot be within thr of it,
+// whichever list it would have gone to; what the two lists hold together still contains the row's two largest
+// values within thr of its best.  (A cut from the smaller best lets through everything between the two bests,
+// and with 32 rows per warp the warp-wide skip then hardly ever fires.)
 // a_i: accumulators, w_i: inverse norms of the four columns idx..idx+3.
 // TEST = false (the first tile of an item, where nearly every group holds a new candidate for some row):
 // all four columns are inserted without the skip test, so nothing but the select chains is on the
@@ -224,7 +228,7 @@ __device__ __forceinline__ void offer4(Top2 &ta, Top2 &tb, float a0, float a1, f
     if (!__any_sync(0xffffffffu, (int)s >= 0)) return;   // no lane has a value that is not below its cut
   }
   ta.insert(a0 * w.x, idx); tb.insert(a1 * w.y, idx + 1); ta.insert(a2 * w.z, idx + 2); tb.insert(a3 * w.w, idx + 3);
-  if (TEST) ta.cut = fminf(ta.best, tb.best) - ta.thr;
+  if (TEST) ta.cut = fmaxf(ta.best, tb.best) - ta.thr;
 }
 
 // ------------------------------------------------------------------ the interface's cosine

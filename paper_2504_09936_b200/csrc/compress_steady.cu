@@ -301,7 +301,7 @@ steady_compress_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, cons
         for (int k = 0; k < 32; k += 4)
           offer4<false>(top, topb, __uint_as_float(acc[k]), __uint_as_float(acc[k + 1]), __uint_as_float(acc[k + 2]),
                         __uint_as_float(acc[k + 3]), *reinterpret_cast<const float4 *>(ci + k), c0 + k);
-        top.cut = fminf(top.best, topb.best) - top.thr;
+        top.cut = fmaxf(top.best, topb.best) - top.thr;
       } else {
 #pragma unroll
         for (int k = 0; k < 32; k += 4)

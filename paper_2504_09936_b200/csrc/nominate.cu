@@ -342,7 +342,7 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
               if (t == it.t0) {   // cold trackers: insert everything
                 drain32(std::false_type{}, r0, cb);
                 drain32(std::false_type{}, r1, cb + 32);
-                if (jg == 1) top.cut = fminf(top.best, topb.best) - top.thr;
+                if (jg == 1) top.cut = fmaxf(top.best, topb.best) - top.thr;
               } else {
                 drain32(std::true_type{}, r0, cb);
                 drain32(std::true_type{}, r1, cb + 32);
