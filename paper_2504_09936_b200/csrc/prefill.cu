@@ -10,10 +10,12 @@
 //   warp 0     TMA producer: the unit's window queries (one box of W rows per head) when the unit
 //              changes, key tiles into a 3-stage ring;
 //   warp 1     one thread issues the MMAs into one of two accumulators and commits to the barriers;
-//   warps 2-9  drain (two warps per 32 entries, alternate heads, combined through shared memory): per
-//              entry a running max / weighted sum of 2^(x - max) over the visible queries
-//              (a prompt is causal: query k, at position len - W + k, scores only entries at or before
-//              it), then lscore = ln(sum / sum of the visible weights / G).
+//   warps 2-17 drain (four warps per 32 entries, heads g = w, w + 4 of the group for the w-th of them, combined
+//              through shared memory): per entry a running max / sum of 2^(x + log2 weight - max) over the
+//              visible queries (a prompt is causal: query k, at position len - W + k, scores only entries
+//              at or before it), then lscore = ln(sum / sum of the visible weights / G).  The logarithms
+//              of the window weights are kernel parameters, i.e. constant-bank operands of the multiply-add
+//              that scales the logit, so they cost neither registers nor instructions.
 // Every wait is bounded; one that runs out raises KEEPKV_DEV_TIMEOUT and the CTA winds down.
 #include "common.cuh"
 #include "ptx.cuh"
@@ -22,7 +24,8 @@ namespace keepkv {
 
 constexpr int kPfM = 128;        // entries per tile
 constexpr int kPfStages = 3;     // key-tile ring
-constexpr int kPfThreads = 320;  // producer, MMA issuer, eight drain warps (two per 32-lane quarter, alternate heads)
+constexpr int kPfDrainWarps = 16; // four per 32-lane quarter of tensor memory
+constexpr int kPfThreads = 32 * (2 + kPfDrainWarps);   // producer, MMA issuer, drain warps
 constexpr int kPfWmax = 32;      // window queries per head (columns reserved per head)
 constexpr float kPfLog2e = 1.4426950408889634f;
 constexpr float kPfLn2 = 0.6931471805599453f;
@@ -36,8 +39,8 @@ struct PfSmem {
   static constexpr int kA = 0;
   static constexpr int kB = kPfStages * kABytes;
   static constexpr int kWt = kB + kBBytes;                  // f32 [32] weights, f32 [33] their suffix sums (as ln)
-  static constexpr int kXchg = kWt + 512;                   // f32 [2 accumulators][128 entries][2]: the odd heads' (max, sum)
-  static constexpr int kBytes = kXchg + 2 * 128 * 2 * 4;
+  static constexpr int kXchg = kWt + 512;                   // float2 [2 accumulators][128 entries][4 warps]: (max, sum)
+  static constexpr int kBytes = kXchg + 2 * 128 * 4 * 8;
 };
 
 // Position in the global tile list: sequence, kv head, tile of the unit; next() moves to the next tile.
@@ -46,6 +49,9 @@ __device__ __forceinline__ float pf_ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+
+// log2 of the window weights alpha^(W-1-k), -inf for k >= W (and, with alpha = 0, for all but the last query)
+struct PfLogWeights { float c[kPfWmax]; };
 
 struct PfWalker {
   int b, h, tile, len, tb;
@@ -67,7 +73,7 @@ struct PfWalker {
 template <int D, int G>
 __global__ void __launch_bounds__(kPfThreads, 1)
 prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapQ,
-                      keepkv_params p, keepkv_cache c, int W, int32_t *status_dev) {
+                      keepkv_params p, keepkv_cache c, int W, const PfLogWeights lw, int32_t *status_dev) {
   using SL = PfSmem<D, G>;
   constexpr int KSTEPS = D / 16, NB = SL::kNB;
   constexpr uint32_t IDESC = umma_idesc_bf16(kPfM, NB);
@@ -94,7 +100,7 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
     for (int i = 0; i < kPfStages; ++i) { mbar_init(bar_a_full + 8 * i, 1); mbar_init(bar_a_empty + 8 * i, 1); }
     mbar_init(bar_b_full, 1);
     mbar_init(bar_b_empty, 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(bar_t_full + 8 * i, 1); mbar_init(bar_t_empty + 8 * i, 8); }
+    for (int i = 0; i < 2; ++i) { mbar_init(bar_t_full + 8 * i, 1); mbar_init(bar_t_empty + 8 * i, kPfDrainWarps); }
     mbar_init(bar_drain, 1);
     s_abort = 0;
     s_start[0] = p.B;
@@ -230,13 +236,11 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
     }
   } else {
     // ------------------------------------------------------------ drain: one entry per thread
-    const int quarter = warp & 3, half = (warp - 2) >> 2;       // half 0 takes the even heads, half 1 the odd ones
+    const int quarter = warp & 3, hq = (warp - 2) >> 2;         // this warp takes heads hq, hq + 4 of the group
+    const int g_last = hq < G ? hq + ((G - 1 - hq) / 4) * 4 : -1;   // its last head (none: it only keeps in step)
     const float scale2 = p.sm_scale * kPfLog2e;
     const float ln_G = logf((float)G);
-    float *xchg = reinterpret_cast<float *>(smem + SL::kXchg);
-    float wr[32];   // the window weights stay in registers
-#pragma unroll
-    for (int k = 0; k < 32; ++k) wr[k] = wt[k];
+    float2 *xchg = reinterpret_cast<float2 *>(smem + SL::kXchg);
     for (int it = 0; it < ntiles; ++it) {
       const int a = it & 1;
       int ok = 0;
@@ -246,59 +250,73 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
       const int row = quarter * 32 + lane;
       const int i = wk.tile * kPfM + row;                         // this thread's entry
       const int klo = min(32, max(0, i - wk.len + W));            // first window query that sees it
-      const bool full = W == kPfWmax && wk.tile * kPfM + kPfM - 1 - wk.len + W <= 0;   // whole tile sees every query
+      const bool full = wk.tile * kPfM + kPfM - 1 - wk.len + W <= 0;   // the whole tile is seen by every query
       const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + a * NB;
       float m = -CUDART_INF_F, S = 0.f;
-      constexpr int LAST = G >= 2 ? G - 2 : 0;   // last head index of half 0 (half 1: LAST + 1)
+      if (g_last < 0) {   // no head for this warp: the accumulator is not its business
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_t_empty + 8 * a);
+      }
 #pragma unroll 1
-      for (int g = half; g < G; g += 2) {
+      for (int g = hq; g < G; g += 4) {
         uint32_t r[32];
         tmem_ld_32x32(taddr + g * 32, r);
         tmem_ld_wait();
-        if (g >= LAST) {   // this warp's part of the accumulator is in registers: hand it back
+        if (g == g_last) {   // this warp's part of the accumulator is in registers: hand it back
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_t_empty + 8 * a);
         }
-        float x[32], mc = -CUDART_INF_F;
+        // y_k = log2 of (weight_k * score_k); queries k >= W carry weight 0 (log2 = -inf).  Two copies of the
+        // loop, chosen per tile: only the last tiles of a unit hold entries that some window queries do not see.
+        float y[32], mc = -CUDART_INF_F, mc2 = -CUDART_INF_F;
+        if (full) {
 #pragma unroll
-        for (int k = 0; k < 32; ++k) {
-          x[k] = __uint_as_float(r[k]) * scale2;
-          if (!full) x[k] = (k >= klo && k < W) ? x[k] : -CUDART_INF_F;
-          mc = fmaxf(mc, x[k]);
+          for (int k = 0; k < 32; k += 2) {
+            y[k] = fmaf(__uint_as_float(r[k]), scale2, lw.c[k]);
+            y[k + 1] = fmaf(__uint_as_float(r[k + 1]), scale2, lw.c[k + 1]);
+            mc = fmaxf(mc, y[k]);
+            mc2 = fmaxf(mc2, y[k + 1]);
+          }
+        } else {
+#pragma unroll
+          for (int k = 0; k < 32; k += 2) {
+            y[k] = k >= klo ? fmaf(__uint_as_float(r[k]), scale2, lw.c[k]) : -CUDART_INF_F;
+            y[k + 1] = k + 1 >= klo ? fmaf(__uint_as_float(r[k + 1]), scale2, lw.c[k + 1]) : -CUDART_INF_F;
+            mc = fmaxf(mc, y[k]);
+            mc2 = fmaxf(mc2, y[k + 1]);
+          }
         }
-        const float m_new = fmaxf(m, mc);
+        const float m_new = fmaxf(m, fmaxf(mc, mc2));
         if (m_new > -CUDART_INF_F) {
           S *= pf_ex2(m - m_new);   // m = -inf: S is 0 and stays 0
           float add0 = 0.f, add1 = 0.f;
 #pragma unroll
           for (int k = 0; k < 32; k += 2) {
-            add0 = fmaf(wr[k], pf_ex2(x[k] - m_new), add0);
-            add1 = fmaf(wr[k + 1], pf_ex2(x[k + 1] - m_new), add1);
+            add0 += pf_ex2(y[k] - m_new);
+            add1 += pf_ex2(y[k + 1] - m_new);
           }
           S += add0 + add1;
           m = m_new;
         }
       }
-      if (G == 1) {
-        if (half == 1) {   // a single head: nothing for the second warp of the quarter to read
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar_t_empty + 8 * a);
-        }
-      } else {
-        // the two warps of a quarter meet at a barrier of their own (64 threads)
-        float2 *x2 = reinterpret_cast<float2 *>(xchg) + a * 128 + row;
-        if (half == 1) *x2 = make_float2(m, S);
-        asm volatile("bar.sync %0, 64;" ::"r"(1 + quarter) : "memory");
-        if (half == 0) {
-          const float2 o = *x2;
-          const float mm = fmaxf(m, o.x);
-          if (mm > -CUDART_INF_F) S = S * pf_ex2(m - mm) + o.y * pf_ex2(o.x - mm);
-          m = mm;
+      if (G > 1) {
+        // the warps of a quarter meet at a barrier of their own (128 threads)
+        float2 *x2 = xchg + (a * 128 + row) * 4;
+        if (hq > 0 && hq < G) x2[hq] = make_float2(m, S);
+        asm volatile("bar.sync %0, 128;" ::"r"(1 + quarter) : "memory");
+        if (hq == 0) {
+#pragma unroll
+          for (int w = 1; w < (G < 4 ? G : 4); ++w) {
+            const float2 o = x2[w];
+            const float mm = fmaxf(m, o.x);
+            if (mm > -CUDART_INF_F) S = S * pf_ex2(m - mm) + o.y * pf_ex2(o.x - mm);
+            m = mm;
+          }
         }
       }
-      if (half == 0 && i < wk.len)
+      if (hq == 0 && i < wk.len)
         c.lscore[((size_t)(wk.b * p.H_kv + wk.h)) * p.N_cap + i] = (m + log2f(S)) * kPfLn2 - lnwsuf[klo] - ln_G;
       wk.next(p, c.seq_len, it + 1 < ntiles);
     }
@@ -340,8 +358,14 @@ static void launch_prefill_t(const keepkv_params &p, const keepkv_cache &c, cons
     if (ctx.err == cudaSuccess) ctx.err = cudaErrorInvalidValue;
     return;
   }
+  PfLogWeights lw;
+  for (int k = 0; k < kPfWmax; ++k) {
+    if (k >= W) lw.c[k] = -INFINITY;
+    else if (p.ema_alpha > 0.f) lw.c[k] = (float)(W - 1 - k) * log2f(p.ema_alpha);
+    else lw.c[k] = k == W - 1 ? 0.f : -INFINITY;
+  }
   launch_pdl(prefill_scores_kernel<D, G>, dim3(sm_count()), dim3(kPfThreads), smem_bytes, ctx.stream, mapK, mapQ, p, c,
-             W, status_dev);
+             W, lw, status_dev);
   KEEPKV_CHECK_LAUNCH(ctx);
 }
 
