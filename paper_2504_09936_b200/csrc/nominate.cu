@@ -324,13 +324,15 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
               }
               const int cb = jg * 64;
               const bool ragged = n_valid < cb + 64;   // columns past n_ret hold other rows' data
-              auto drain32 = [&](auto test, const uint32_t (&r)[32], int off) {
+              // `masked` is a compile-time flag: only the last tile of a row of tiles has columns to mask, and a
+              // run-time test inside the unrolled loop would be turned into selects that every group pays for
+              auto drain32 = [&](auto test, auto masked, const uint32_t (&r)[32], int off) {
 #pragma unroll
                 for (int i = 0; i < 32; i += 4) {
                   float4 iv = *reinterpret_cast<const float4 *>(inv_w + off + i);
                   float a0 = __uint_as_float(r[i]), a1 = __uint_as_float(r[i + 1]);
                   float a2 = __uint_as_float(r[i + 2]), a3 = __uint_as_float(r[i + 3]);
-                  if (ragged) {   // a masked column contributes -inf
+                  if (decltype(masked)::value) {   // a masked column contributes -inf
                     if (off + i >= n_valid) { a0 = -CUDART_INF_F; iv.x = 1.f; }
                     if (off + i + 1 >= n_valid) { a1 = -CUDART_INF_F; iv.y = 1.f; }
                     if (off + i + 2 >= n_valid) { a2 = -CUDART_INF_F; iv.z = 1.f; }
@@ -339,14 +341,21 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
                   offer4<decltype(test)::value>(top, topb, a0, a1, a2, a3, iv, c0 + off + i);
                 }
               };
-              if (t == it.t0) {   // cold trackers: insert everything
-                drain32(std::false_type{}, r0, cb);
-                drain32(std::false_type{}, r1, cb + 32);
-                if (jg == 1) top.cut = fmaxf(top.best, topb.best) - top.thr;
+              const bool cold = t == it.t0;   // cold lists: insert everything
+              if (cold && ragged) {
+                drain32(std::false_type{}, std::true_type{}, r0, cb);
+                drain32(std::false_type{}, std::true_type{}, r1, cb + 32);
+              } else if (cold) {
+                drain32(std::false_type{}, std::false_type{}, r0, cb);
+                drain32(std::false_type{}, std::false_type{}, r1, cb + 32);
+              } else if (ragged) {
+                drain32(std::true_type{}, std::true_type{}, r0, cb);
+                drain32(std::true_type{}, std::true_type{}, r1, cb + 32);
               } else {
-                drain32(std::true_type{}, r0, cb);
-                drain32(std::true_type{}, r1, cb + 32);
+                drain32(std::true_type{}, std::false_type{}, r0, cb);
+                drain32(std::true_type{}, std::false_type{}, r1, cb + 32);
               }
+              if (cold && jg == 1) top.cut = fmaxf(top.best, topb.best) - top.thr;
             }
           }
         }
