@@ -34,8 +34,8 @@ from paper_2504_09936_b200 import workloads as W  # noqa: E402
 
 METRIC = "decode tokens/s + compress GB/s, fraction of HBM roofline"
 # dram__bytes_read.sum + dram__bytes_write.sum of one steady-state decode launch of workload C2, from the ncu
-# capture summarised in profiles/decode_kernel_C2_steady.md (57.68 MB + 0.66 MB); None for other workloads
-DECODE_TRAFFIC_BYTES = 58.34e6
+# capture summarised in profiles/decode_kernel_C2_steady.md (57.68 MB + 0.61 MB); None for other workloads
+DECODE_TRAFFIC_BYTES = 58.29e6
 UNIT = "tokens/s"
 
 
