@@ -98,7 +98,7 @@ def lib() -> C.CDLL:
         _lib.okv_round_bf16.argtypes = [C.c_double]
         _lib.okv_cosine.restype = C.c_float
         _lib.okv_merge_group.restype = C.c_double
-        for n in ("okv_select", "okv_select_sorted", "okv_compress", "okv_append", "okv_num_threads"):
+        for n in ("okv_select", "okv_select_sorted", "okv_compress", "okv_compress_keyed", "okv_append", "okv_num_threads"):
             getattr(_lib, n).restype = C.c_int32
     return _lib
 
@@ -208,9 +208,11 @@ def merge_group(d: int, idx, K, V, votes, lscore):
     return dict(k_r=kr, v_r=vr, p_r=pr.value, lambda_r=lr.value, gamma=float(g), lambda_bar=lb.value)
 
 
-def compress(P: Params, budget: int, K, V, votes, lscore, sorted_select: bool = False):
+def compress(P: Params, budget: int, K, V, votes, lscore, sorted_select: bool = False, select_key=None):
     """Algorithm 1 end to end for one unit.  Returns a dict with the compacted cache
-    (K, V, votes, lscore: n_ret rows), ret_idx, target [len], gammas [n_ret], stats."""
+    (K, V, votes, lscore: n_ret rows), ret_idx, target [len], gammas [n_ret], stats.
+    select_key: optional fp32 importance scores [len] that replace kappa in the selection (Section 3.4:
+    any token selection may designate the retained and evicted sets)."""
     K, V, votes, lscore = _f64(K), _f64(V), _f64(votes), _f64(lscore)
     n, d = K.shape[0], P.d
     m = max(min(n, max(budget, 0)), 1)
@@ -220,9 +222,16 @@ def compress(P: Params, budget: int, K, V, votes, lscore, sorted_select: bool = 
     gam = np.empty(m, dtype=np.float64)
     st = _Stats()
     cp = P.c()
-    n_ret = lib().okv_compress(C.byref(cp), C.c_int32(n), C.c_int32(budget), _p(K), _p(V), _p(votes), _p(lscore),
-                               _p(dK), _p(dV), _p(dv), _p(dl), _pi(ret), _pi(target), _p(gam), C.byref(st),
-                               C.c_int32(int(sorted_select)))
+    if select_key is None:
+        n_ret = lib().okv_compress(C.byref(cp), C.c_int32(n), C.c_int32(budget), _p(K), _p(V), _p(votes), _p(lscore),
+                                   _p(dK), _p(dV), _p(dv), _p(dl), _pi(ret), _pi(target), _p(gam), C.byref(st),
+                                   C.c_int32(int(sorted_select)))
+    else:
+        key = np.ascontiguousarray(select_key, dtype=np.float32)
+        assert key.shape == (n,)
+        n_ret = lib().okv_compress_keyed(C.byref(cp), C.c_int32(n), C.c_int32(budget), _p(K), _p(V), _p(votes),
+                                         _p(lscore), _p(key, C.c_float), _p(dK), _p(dV), _p(dv), _p(dl), _pi(ret),
+                                         _pi(target), _p(gam), C.byref(st), C.c_int32(int(sorted_select)))
     return dict(K=dK[:n_ret], V=dV[:n_ret], votes=dv[:n_ret], lscore=dl[:n_ret], ret_idx=ret[:n_ret].copy(),
                 target=target[:n].copy(), gammas=gam[:n_ret],
                 stats={f: getattr(st, f) for f, _ in _Stats._fields_ if f != "pad_"})

@@ -373,16 +373,37 @@ double okv_merge_group(int d, int n, const int32_t *idx, const double *K, const 
  * ascending original index.  ret_idx[n_ret], target[len] (as in okv_match), gammas
  * [n_ret] (NaN where the slot had no group) are outputs; any of target/gammas/stats
  * may be NULL.  use_sorted_select picks the sort-based selection.  Returns n_ret. */
+/* select_key: NULL, or len importance scores supplied by the caller that replace kappa in the
+ * selection only (Section 3.4, "no specific constraints on ... token selection strategies"; Section
+ * 4.5 combines the merge with H2O's and PyramidInfer's selections): the retained and evicted sets
+ * come from the given scores, the merging pairs and the merge itself are unchanged. */
+int32_t okv_compress_keyed(const okv_params *P, int32_t len, int32_t budget, const double *K, const double *V,
+                           const double *votes, const double *lscore, const float *select_key, double *dK,
+                           double *dV, double *dvotes, double *dlscore, int32_t *ret_idx, int32_t *target_out,
+                           double *gammas, okv_stats *stats, int32_t use_sorted_select);
+
 int32_t okv_compress(const okv_params *P, int32_t len, int32_t budget, const double *K, const double *V,
                      const double *votes, const double *lscore, double *dK, double *dV, double *dvotes,
                      double *dlscore, int32_t *ret_idx, int32_t *target_out, double *gammas, okv_stats *stats,
                      int32_t use_sorted_select) {
+  return okv_compress_keyed(P, len, budget, K, V, votes, lscore, NULL, dK, dV, dvotes, dlscore, ret_idx, target_out,
+                            gammas, stats, use_sorted_select);
+}
+
+int32_t okv_compress_keyed(const okv_params *P, int32_t len, int32_t budget, const double *K, const double *V,
+                           const double *votes, const double *lscore, const float *select_key, double *dK,
+                           double *dV, double *dvotes, double *dlscore, int32_t *ret_idx, int32_t *target_out,
+                           double *gammas, okv_stats *stats, int32_t use_sorted_select) {
   const int d = P->d;
   const int L1 = len > 0 ? len : 1;
   float *kappa = (float *)malloc(sizeof(float) * (size_t)L1);
   int32_t *target = (int32_t *)malloc(sizeof(int32_t) * (size_t)L1);
   float *umax = (float *)malloc(sizeof(float) * (size_t)L1);
-  okv_kappa(len, votes, lscore, kappa);
+  if (select_key) {
+    for (int i = 0; i < len; ++i) kappa[i] = select_key[i];
+  } else {
+    okv_kappa(len, votes, lscore, kappa);
+  }
   int32_t n_ret = use_sorted_select ? okv_select_sorted(len, kappa, budget, P->n_sink, P->n_recent, ret_idx)
                                     : okv_select(len, kappa, budget, P->n_sink, P->n_recent, ret_idx);
   okv_match(P, len, K, n_ret, ret_idx, target, umax, NULL);

@@ -162,6 +162,42 @@ def test_selection_tie_keeps_lowest_index():
     assert list(O.select(kap, 3, 1, 1)) == [0, 1, 4]
 
 
+@pytest.mark.parametrize("seed", range(4))
+def test_compress_with_caller_supplied_selection_scores(seed):
+    """Section 3.4 / 4.5: any token selection may designate the retained and evicted sets.  With caller scores
+    the retained set is the numpy-sorted selection on those scores; the rest of Algorithm 1 is unchanged, so
+    (a) passing kappa itself as the scores reproduces the default compression exactly, and (b) the output equals
+    the default compression of a cache whose lscore makes kappa equal to the scores, wherever that substitution
+    does not touch the merge (no evicted entry merged: T above every cosine)."""
+    rng = RNG(300 + seed)
+    n, d, budget, n_sink, n_recent = int(rng.integers(40, 160)), 16, 24, 3, 9
+    K = O.round_bf16(rng.standard_normal((n, d)))
+    V = O.round_bf16(rng.standard_normal((n, d)))
+    votes = rng.integers(1, 4, n).astype(np.float64)
+    ls = rng.standard_normal(n)
+    key = np.abs(rng.standard_normal(n)).cumsum()[rng.permutation(n)].astype(np.float32)   # accumulated-attention-like
+    key[rng.integers(0, n, 5)] = key[rng.integers(0, n)]                                    # ties
+    P = O.Params(G=1, d=d, n_sink=n_sink, n_recent=n_recent, merge_threshold=0.3)
+    c = O.compress(P, budget, K, V, votes, ls, select_key=key)
+    assert np.array_equal(c["ret_idx"], _select_numpy(key, budget, n_sink, n_recent))
+    # (a) kappa as scores = default
+    c0 = O.compress(P, budget, K, V, votes, ls)
+    ck = O.compress(P, budget, K, V, votes, ls, select_key=O.kappa(votes, ls))
+    for f in ("ret_idx", "target", "K", "V", "votes", "lscore"):
+        assert np.array_equal(c0[f], ck[f], equal_nan=True), f
+    # (b) nothing merged: the scores only pick rows
+    P1 = O.Params(G=1, d=d, n_sink=n_sink, n_recent=n_recent, merge_threshold=1.5)
+    c1 = O.compress(P1, budget, K, V, votes, ls, select_key=key)
+    r = c1["ret_idx"]
+    assert np.all(c1["target"][np.setdiff1d(np.arange(n), r)] == -1)
+    assert np.array_equal(c1["K"], K[r]) and np.array_equal(c1["V"], V[r])
+    assert np.array_equal(c1["votes"], votes[r]) and np.array_equal(c1["lscore"], ls[r])
+    # merge targets depend only on the sets: wherever an entry was merged, it went where the matcher alone sends it
+    tgt, _, _ = O.match(P, K, c["ret_idx"])
+    merged = c["target"] >= 0
+    assert merged.any() and np.array_equal(c["target"][merged], np.asarray(tgt)[merged])
+
+
 def test_kappa_is_log_of_vote_weighted_score():
     votes = np.array([1.0, 2.0, 7.0])
     ls = np.array([0.25, -3.0, -np.inf])
