@@ -172,6 +172,17 @@ int keepkv_compress(const keepkv_params *p, const keepkv_cache *src, const keepk
                     int32_t *retained_idx_or_null, int32_t *target_or_null, keepkv_stats *stats_or_null, void *ws,
                     size_t ws_bytes, int32_t *status_dev, void *stream);
 
+/* keepkv_compress with the selection of step 1 driven by the caller's own importance scores (Section 3.4: the
+ * method puts no constraint on the token selection, the retained and evicted sets only designate the merging
+ * pairs; Section 4.5 combines it with H2O's accumulated attention and PyramidInfer's selection).
+ * select_score_or_null: fp32 [B, H_kv, N_cap], larger = more important, must not be NaN; it replaces kappa
+ * among the entries between the sinks and the recent window (equal scores -> lower index); votes and lscore
+ * still drive the merge of step 3.  NULL makes this keepkv_compress.  Everything else as there. */
+int keepkv_compress_scored(const keepkv_params *p, const keepkv_cache *src, const keepkv_cache *dst,
+                           const float *select_score_or_null, const int32_t *budget_dev, int32_t budget_scalar,
+                           const int32_t *n_recent_dev, int32_t *retained_idx_or_null, int32_t *target_or_null,
+                           keepkv_stats *stats_or_null, void *ws, size_t ws_bytes, int32_t *status_dev, void *stream);
+
 /* One decode step driven from HOST memory (the call a serving loop makes): copies q_host,
  * k_new_host, v_new_host (pinned or pageable host memory, shapes as above) into the device
  * staging buffers q_dev/k_new_dev/v_new_dev, runs keepkv_decode_step

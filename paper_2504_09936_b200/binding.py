@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkeepkv.so")
 
 EXPORTS = ("keepkv_workspace_bytes", "keepkv_workspace_init", "keepkv_append", "keepkv_decode_attention",
-           "keepkv_decode_step", "keepkv_compress", "keepkv_prefill_scores", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_status_string", "keepkv_last_cuda_error",
+           "keepkv_decode_step", "keepkv_compress", "keepkv_compress_scored", "keepkv_prefill_scores", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_status_string", "keepkv_last_cuda_error",
            "keepkv_last_launch_count")
 
 
@@ -66,6 +66,7 @@ def lib() -> C.CDLL:
         l.keepkv_decode_attention_static.argtypes = [pp, pc, vp, vp, vp, C.c_int, vp, vp]
         l.keepkv_prefill_scores.argtypes = [pp, pc, vp, i32, vp, vp]
         l.keepkv_compress.argtypes = [pp, pc, pc, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
+        l.keepkv_compress_scored.argtypes = [pp, pc, pc, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         l.keepkv_decode_step_host.argtypes = [pp, pc] + [vp] * 8 + [C.c_int, vp, sz, vp, vp]
         l.keepkv_decode_step_host_layers.argtypes = [pp, pc, i32] + [vp] * 8 + [C.c_int, vp, sz, vp, vp]
         _lib = l
@@ -180,6 +181,17 @@ def keepkv_compress(p, src: Cache, dst: Cache, budget, ws, status, n_recent_dev=
     _check(lib().keepkv_compress(C.byref(p), C.byref(src.c()), C.byref(dst.c()), bdev, bsc, _ptr(n_recent_dev),
                                  _ptr(retained_idx), _ptr(target), _ptr(stats), ws.data_ptr(), ws.numel(),
                                  status.data_ptr(), _stream(stream)), "keepkv_compress")
+
+
+def keepkv_compress_scored(p, src: Cache, dst: Cache, select_score, budget, ws, status, n_recent_dev=None,
+                           retained_idx=None, target=None, stats=None, stream=None):
+    """keepkv_compress with the caller's importance scores (fp32 CUDA tensor [B, H_kv, N_cap]) driving the selection."""
+    assert select_score.dtype == torch.float32 and select_score.is_contiguous()
+    bdev, bsc = (budget.data_ptr(), 0) if isinstance(budget, torch.Tensor) else (None, int(budget))
+    _check(lib().keepkv_compress_scored(C.byref(p), C.byref(src.c()), C.byref(dst.c()), select_score.data_ptr(), bdev,
+                                        bsc, _ptr(n_recent_dev), _ptr(retained_idx), _ptr(target), _ptr(stats),
+                                        ws.data_ptr(), ws.numel(), status.data_ptr(), _stream(stream)),
+           "keepkv_compress_scored")
 
 
 def keepkv_decode_step_host(p, cache: Cache, q_host, k_new_host, v_new_host, out_host, q_dev, k_new_dev, v_new_dev,

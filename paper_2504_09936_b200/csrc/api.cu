@@ -176,6 +176,14 @@ int keepkv_compress(const keepkv_params *p, const keepkv_cache *src, const keepk
                     const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
                     int32_t *retained_idx_or_null, int32_t *target_or_null, keepkv_stats *stats_or_null, void *ws,
                     size_t ws_bytes, int32_t *status_dev, void *stream) {
+  return keepkv_compress_scored(p, src, dst, nullptr, budget_dev, budget_scalar, n_recent_dev, retained_idx_or_null,
+                                target_or_null, stats_or_null, ws, ws_bytes, status_dev, stream);
+}
+
+int keepkv_compress_scored(const keepkv_params *p, const keepkv_cache *src, const keepkv_cache *dst,
+                           const float *select_score_or_null, const int32_t *budget_dev, int32_t budget_scalar,
+                           const int32_t *n_recent_dev, int32_t *retained_idx_or_null, int32_t *target_or_null,
+                           keepkv_stats *stats_or_null, void *ws, size_t ws_bytes, int32_t *status_dev, void *stream) {
   int rc = validate(p);
   if (rc) return rc;
   if ((rc = validate_cache(src))) return rc;
@@ -197,7 +205,8 @@ int keepkv_compress(const keepkv_params *p, const keepkv_cache *src, const keepk
   launch_compress(*p, *src, *dst, budget_dev, budget_scalar, n_recent_dev,
                   retained_idx_or_null ? retained_idx_or_null : (int32_t *)(w + L.ret_idx),
                   target_or_null ? target_or_null : (int32_t *)(w + L.target),
-                  stats_or_null ? stats_or_null : (keepkv_stats *)(w + L.stats), w, L, status_dev, ctx);
+                  stats_or_null ? stats_or_null : (keepkv_stats *)(w + L.stats), w, L, status_dev, ctx,
+                  select_score_or_null);
   return finish(ctx);
 }
 

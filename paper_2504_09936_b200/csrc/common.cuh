@@ -63,7 +63,7 @@ void launch_decode(const keepkv_params &p, const keepkv_cache &c, const void *q,
 void launch_compress(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
                      const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev, int32_t *ret_idx,
                      int32_t *target, keepkv_stats *stats, char *ws, const WsLayout &L, int32_t *status_dev,
-                     LaunchCtx &ctx);
+                     LaunchCtx &ctx, const float *select_key = nullptr);
 // tcgen05 similarity search: for every evicted key the two largest cosines over the retained keys
 void launch_nominate(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst, const int32_t *ev_idx,
                      const UnitInfo *unit_info, const float *inv_norm, int32_t *sched, float4 *nom_v, int32_t *nom_si,

@@ -20,7 +20,7 @@ constexpr int kWarpSelectMax = 2048;   // candidate sets up to this size are sea
 __global__ void __launch_bounds__(1024)
 select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int32_t *budget_dev, int budget_scalar,
               const int32_t *n_recent_dev, int32_t *ret_idx, int32_t *target, int32_t *ev_idx, UnitInfo *unit_info,
-              keepkv_stats *stats) {
+              keepkv_stats *stats, const float *__restrict__ select_key) {
   extern __shared__ uint32_t keys[];
   __shared__ int hist[256];
   __shared__ int warp_tot[32];
@@ -49,10 +49,8 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
   const int nthr = min((int)blockDim.x, max(128, ((len + 3) / 4 + 31) & ~31)), nw = nthr >> 5;
   if (tid >= nthr) return;
   for (int i = tid; i < len; i += nthr) {
-    const float pv = src.votes[base + i], ls = src.lscore[base + i];
-    // kappa = ln p + lscore in fp64, rounded once to fp32 (p = 1 needs no logarithm)
-    const float kappa = (pv == 1.0f) ? ls : (float)(log((double)pv) + (double)ls);
-    keys[i] = ordered_key(kappa);
+    // the caller's scores where given, else kappa = ln p + lscore
+    keys[i] = select_key ? ordered_key(select_key[base + i]) : kappa_key(src.votes[base + i], src.lscore[base + i]);
   }
   __syncthreads();
 
@@ -466,7 +464,7 @@ template <int D>
 static void launch_compress_t(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
                               const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
                               int32_t *ret_idx, int32_t *target, keepkv_stats *stats, char *ws, const WsLayout &L,
-                              int32_t *status_dev, LaunchCtx &ctx) {
+                              int32_t *status_dev, const float *select_key, LaunchCtx &ctx) {
   const int U = p.B * p.H_kv;
   UnitInfo *ui = reinterpret_cast<UnitInfo *>(ws + L.unit_info);
   int32_t *sched = reinterpret_cast<int32_t *>(ws + L.sched);
@@ -491,11 +489,11 @@ static void launch_compress_t(const keepkv_params &p, const keepkv_cache &src, c
   }
   if (p.flags & KEEPKV_FLAG_COMPRESS_STEADY) {   // the caller vouches for every unit: one kernel does it all
     launch_compress_steady(p, src, dst, budget_dev, budget_scalar, n_recent_dev, ret_idx, target, stats, ws, L, status_dev,
-                           ctx);
+                           select_key, ctx);
     return;
   }
   launch_pdl(select_kernel, dim3(U), dim3(512), sel_smem, ctx.stream, p, src, dst.seq_len, budget_dev, budget_scalar,
-             n_recent_dev, ret_idx, target, ev_idx, ui, stats);
+             n_recent_dev, ret_idx, target, ev_idx, ui, stats, select_key);
   KEEPKV_CHECK_LAUNCH(ctx);
   if (ret_bound <= 0) return;   // nothing is kept: every entry is dropped, which select has recorded
   const int cgx = (ret_bound + 63) / 64 < 32 ? (ret_bound + 63) / 64 : 32;   // the retained count is only known on the device
@@ -517,13 +515,13 @@ static void launch_compress_t(const keepkv_params &p, const keepkv_cache &src, c
 void launch_compress(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
                      const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev, int32_t *ret_idx,
                      int32_t *target, keepkv_stats *stats, char *ws, const WsLayout &L, int32_t *status_dev,
-                     LaunchCtx &ctx) {
+                     LaunchCtx &ctx, const float *select_key) {
   if (p.d == 128)
     launch_compress_t<128>(p, src, dst, budget_dev, budget_scalar, n_recent_dev, ret_idx, target, stats, ws, L,
-                           status_dev, ctx);
+                           status_dev, select_key, ctx);
   else
     launch_compress_t<64>(p, src, dst, budget_dev, budget_scalar, n_recent_dev, ret_idx, target, stats, ws, L,
-                          status_dev, ctx);
+                          status_dev, select_key, ctx);
 }
 
 }  // namespace keepkv

@@ -359,6 +359,6 @@ __device__ __forceinline__ void merge_group(const keepkv_params &p, const keepkv
 void launch_compress_steady(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
                             const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
                             int32_t *ret_idx, int32_t *target, keepkv_stats *stats, char *ws, const WsLayout &L,
-                            int32_t *status_dev, LaunchCtx &ctx);
+                            int32_t *status_dev, const float *select_key, LaunchCtx &ctx);
 
 }  // namespace keepkv

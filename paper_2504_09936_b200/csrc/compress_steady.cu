@@ -60,7 +60,8 @@ template <int D>
 __global__ void __launch_bounds__(kStThreads, 2)
 steady_compress_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_t *budget_dev, int budget_scalar,
                        const int32_t *n_recent_dev, int32_t *ret_idx, int32_t *target, UnitInfo *unit_info, float4 *nom_v,
-                       int32_t *nom_si, int C_max, int *counters, keepkv_stats *stats, int32_t *status_dev) {
+                       int32_t *nom_si, int C_max, int *counters, keepkv_stats *stats, int32_t *status_dev,
+                       const float *__restrict__ select_key) {
   using SL = StSmem<D>;
   constexpr int KSTEPS = D / 16;          // k-steps of the similarity product
   constexpr int CH = D / 8;               // 16-byte chunks of a row
@@ -173,7 +174,9 @@ steady_compress_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, cons
   if (early) { issue_keys(t0); issue_keys(t0 + 1); issue_keys(t0 + 2); load_values(t0); }
 
   // ---- selection (lines 2-3)
-  for (int i = tid; i < m_cand; i += kStThreads) keys[i] = kappa_key(src.votes[base + lo + i], src.lscore[base + lo + i]);
+  for (int i = tid; i < m_cand; i += kStThreads)   // the caller's scores where given, else kappa = ln p + lscore
+    keys[i] = select_key ? ordered_key(select_key[base + lo + i])
+                         : kappa_key(src.votes[base + lo + i], src.lscore[base + lo + i]);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -483,7 +486,7 @@ template <int D>
 static void launch_steady_t(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
                             const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
                             int32_t *ret_idx, int32_t *target, keepkv_stats *stats, char *ws, const WsLayout &L,
-                            int32_t *status_dev, LaunchCtx &ctx) {
+                            int32_t *status_dev, const float *select_key, LaunchCtx &ctx) {
   using SL = StSmem<D>;
   const int U = p.B * p.H_kv;
   constexpr size_t smem_bytes = (size_t)SL::kBytes + 1024;   // slack to align the swizzled tiles
@@ -500,20 +503,20 @@ static void launch_steady_t(const keepkv_params &p, const keepkv_cache &src, con
   launch_pdl(steady_compress_kernel<D>, dim3(R, U), dim3(kStThreads), smem_bytes, ctx.stream, p, src, dst,
              budget_dev, budget_scalar, n_recent_dev, ret_idx, target, reinterpret_cast<UnitInfo *>(ws + L.unit_info),
              reinterpret_cast<float4 *>(ws + L.nom_v), reinterpret_cast<int32_t *>(ws + L.nom_si), L.nom_chunks,
-             reinterpret_cast<int *>(ws + L.counters), stats, status_dev);
+             reinterpret_cast<int *>(ws + L.counters), stats, status_dev, select_key);
   KEEPKV_CHECK_LAUNCH(ctx);
 }
 
 void launch_compress_steady(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
                             const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
                             int32_t *ret_idx, int32_t *target, keepkv_stats *stats, char *ws, const WsLayout &L,
-                            int32_t *status_dev, LaunchCtx &ctx) {
+                            int32_t *status_dev, const float *select_key, LaunchCtx &ctx) {
   if (p.d == 128)
     launch_steady_t<128>(p, src, dst, budget_dev, budget_scalar, n_recent_dev, ret_idx, target, stats, ws, L, status_dev,
-                         ctx);
+                         select_key, ctx);
   else
     launch_steady_t<64>(p, src, dst, budget_dev, budget_scalar, n_recent_dev, ret_idx, target, stats, ws, L, status_dev,
-                        ctx);
+                        select_key, ctx);
 }
 
 }  // namespace keepkv

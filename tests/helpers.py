@@ -140,13 +140,14 @@ def check_decode_unit(p, u, hc: HostCache, q64, out_gpu64, lse_gpu, lscore_after
 
 
 def check_compress_unit(p, u, budget, n_recent, hc_src: HostCache, hc_dst: HostCache, ret_idx, target, stats=None,
-                        what="", sorted_select=True):
+                        what="", sorted_select=True, select_key=None):
     """Teacher-forced staged check of one unit of a compress call: the oracle is fed the same source
     state; index sets and merge targets must match exactly, tensors within the bf16 rules."""
     P = oracle_params(p, n_recent=n_recent)
     K, V, votes, ls = hc_src.unit(u)
     n = K.shape[0]
-    ref = O.compress(P, budget, K, V, votes, ls, sorted_select=sorted_select)
+    ref = O.compress(P, budget, K, V, votes, ls, sorted_select=sorted_select,
+                     select_key=None if select_key is None else select_key[u, :n])
     m = len(ref["ret_idx"])
     b = u // p.H_kv
     assert int(hc_dst.seq_len[b]) == m, f"{what} u={u}: new seq_len {hc_dst.seq_len[b]} != {m}"

@@ -564,3 +564,38 @@ def test_compress_steady_flag_reports_units_outside_its_limits():
         kb.keepkv_compress(p, src, kb.Cache.empty(p), 0, ws, st)
     with pytest.raises(kb.KeepKVError):
         kb.keepkv_compress(_copy_params(p, flags=2), src, kb.Cache.empty(p), budget, ws, st)
+
+
+@pytest.mark.parametrize("flags", [0, kb.FLAG_COMPRESS_STEADY])
+def test_compress_with_caller_supplied_selection_scores(flags):
+    """keepkv_compress_scored: the caller's importance scores (here an accumulated-attention-like positive
+    score with ties) pick the retained set; the merge is unchanged.  Both compression paths, against the oracle."""
+    B, H_kv, G, d = 3, 2, 2, 128
+    lens, budget, n_recent = [330, 300, 256], 256, 100
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=384, period=0, n_sink=4, n_recent=n_recent,
+                       merge_threshold=0.1, flags=flags)
+    src = random_cache(p, lens, seed=91, vote_max=3)
+    rng = np.random.default_rng(92)
+    U = B * H_kv
+    key = np.abs(rng.standard_normal((U, p.N_cap))).cumsum(axis=1)
+    key = np.take_along_axis(key, rng.permuted(np.tile(np.arange(p.N_cap), (U, 1)), axis=1), axis=1).astype(np.float32)
+    key[:, 20:26] = key[:, 20:21]                                         # equal scores: the lower index is kept first
+    key_dev = torch.from_numpy(key).cuda().view(B, H_kv, p.N_cap)
+    dst = kb.Cache.empty(p)
+    ws, st = kb.new_workspace(p), kb.new_status()
+    ret = torch.full((U, p.N_cap), -7, dtype=torch.int32, device="cuda")
+    tgt = torch.full((U, p.N_cap), -7, dtype=torch.int32, device="cuda")
+    stats = torch.zeros(U, 8, dtype=torch.int32, device="cuda")
+    kb.keepkv_compress_scored(p, src, dst, key_dev, budget, ws, st, retained_idx=ret, target=tgt, stats=stats)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    hs, hd = HostCache(src), HostCache(dst)
+    ret, tgt, stats = ret.cpu().numpy(), tgt.cpu().numpy(), stats.cpu().numpy()
+    n_full = 0
+    for u in range(U):
+        _, full = check_compress_unit(p, u, budget, n_recent, hs, hd, ret, tgt, stats, what="scored", select_key=key)
+        n_full += full
+    assert n_full >= U - 1
+    # and the scores did change the outcome: the default selection keeps a different set
+    dst0, ret0, _, _ = _run_compress(p, src, budget)
+    assert not np.array_equal(ret0[0, :budget], ret[0, :budget])
