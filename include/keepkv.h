@@ -16,8 +16,9 @@
  *
  * Conventions
  *  - Every pointer is DEVICE memory owned by the caller unless its name ends in
- *    `_host`.  The library allocates nothing, holds no state between calls and
- *    never synchronises: each call validates its arguments on the host, enqueues
+ *    `_host`.  The library allocates nothing, holds no state between calls
+ *    (one exception: the built-in scratch array of keepkv_decode_attention_static)
+ *    and never synchronises: each call validates its arguments on the host, enqueues
  *    kernels on `stream` (a cudaStream_t passed as void*) and returns at once.
  *  - Return value: KEEPKV_OK or a negative keepkv_status.  Nothing is enqueued
  *    when a negative value is returned, except for KEEPKV_ERR_CUDA (a launch
@@ -66,7 +67,7 @@ typedef struct keepkv_params {
   int32_t n_recent;         /* entries always kept at the back  (App. B.3: recent window)      */
   float sm_scale;           /* 1/sqrt(d) of Eq. 3                                              */
   float ema_alpha;          /* alpha of Eq. 8, in [0,1); 0 makes the estimate the last score   */
-  float merge_threshold;    /* T of Algorithm 1 line 5 (paper: 0.8); -INFINITY merges always   */
+  float merge_threshold;    /* T of Algorithm 1, arg-max and threshold step (paper: 0.8); -INFINITY merges always   */
   float gamma_min;          /* a group is merged only if gamma_min < gamma <= gamma_max, gamma */
   float gamma_max;          /* the key rescale factor of Eq. A.3; (-INF, +INF) = paper as is   */
   int32_t flags;            /* KEEPKV_FLAG_* bits, normally 0                                  */
@@ -113,8 +114,8 @@ int keepkv_workspace_init(const keepkv_params *p, void *ws, size_t ws_bytes, voi
 
 /* Eq. 2.  For every sequence b and kv head h, writes k_new[b,h,:], v_new[b,h,:] (bf16 [B,H_kv,d])
  * to row seq_len[b], sets that entry's votes to 1 (Section 3.3.1: p initialised to 1) and its
- * lscore to -INFINITY, then increments seq_len[b].  A sequence already at N_cap is left
- * unchanged and KEEPKV_DEV_APPEND_FULL is raised in *status_dev. */
+ * lscore to -INFINITY, then increments seq_len[b].  A sequence already at N_cap (or whose
+ * seq_len[b] is negative) is left unchanged and KEEPKV_DEV_APPEND_FULL is raised in *status_dev. */
 int keepkv_append(const keepkv_params *p, const keepkv_cache *cache, const void *k_new, const void *v_new,
                   int32_t *status_dev, void *stream);
 
@@ -124,7 +125,9 @@ int keepkv_append(const keepkv_params *p, const keepkv_cache *cache, const void 
  * sequence, whose output is 0).
  * update_scores != 0 also advances Eq. 8 for every entry read: the kv head's score at this step
  * is the mean over its G query heads of e^{l_i}; lscore <- ln(alpha e^{lscore} + (1-alpha) score),
- * or ln(score) for an entry never scored before (per-entry bias correction) or when alpha = 0.
+ * or ln(score) for an entry never scored before or when alpha = 0: the first observed score
+ * initialises the state, which equals Eq. 8's bias correction S/(1 - alpha^n) counted from the entry's
+ * first observation at n = 1 only (from n = 2 on the plain recursion is used, not the corrected form).
  * This is the "attention scores s^t" input of Algorithm 1, produced without materialising them. */
 int keepkv_decode_attention(const keepkv_params *p, const keepkv_cache *cache, const void *q, void *out,
                             float *lse_or_null, int update_scores, void *ws, size_t ws_bytes, int32_t *status_dev,
@@ -155,14 +158,14 @@ int keepkv_prefill_scores(const keepkv_params *p, const keepkv_cache *cache, con
  * budget_scalar; likewise n_recent_dev[b] / p->n_recent):
  *   1. key kappa_i = fp32(ln p_i + lscore_i); retained set = first n_sink, last n_recent and the
  *      largest kappa among the rest, equal keys -> lower index; everything else is evicted
- *      (Algorithm 1 lines 2-3; App. B.3).  If the budget is below n_sink + n_recent the recent
+ *      (Algorithm 1, selection step; App. B.3).  If the budget is below n_sink + n_recent the recent
  *      window shrinks first.  len <= budget: plain ordered copy.
  *   2. each evicted key takes the retained key of highest cosine similarity as its target,
  *      equal values -> lower slot, and is merged only if that cosine exceeds merge_threshold
- *      (lines 4-5).  The cosine is the fp32 value dot/(sqrtf(n_e)*sqrtf(n_c)) with dot and the
+ *      (Algorithm 1, similarity and arg-max steps).  The cosine is the fp32 value dot/(sqrtf(n_e)*sqrtf(n_c)) with dot and the
  *      squared norms accumulated by fused multiply-add from 0 over channels 0..d-1.
  *   3. every retained entry with members is rewritten by Eq. A.3 using exp(lscore) as score
- *      estimate: v_r, k_r, p_r = sum of votes, lscore_r = ln(sum p s / sum p) (lines 7-10).
+ *      estimate: v_r, k_r, p_r = sum of votes, lscore_r = ln(sum p s / sum p) (Algorithm 1, merge step).
  *   4. dst holds the retained entries in ascending source order, dst.seq_len[b] = min(len, b_b).
  * Optional outputs: retained_idx_or_null i32 [B, H_kv, N_cap] (first seq_len entries valid: source
  * index of each dst row); target_or_null i32 [B, H_kv, N_cap] (per source entry: dst slot it was
@@ -209,9 +212,12 @@ int keepkv_decode_step_host_layers(const keepkv_params *p, const keepkv_cache *c
  * of KEEPKV_STATIC_SCRATCH_BYTES inside the library image; every GPU that loads the library holds
  * it until the process exits.  The call allocates and frees nothing.
  *  - Arguments as keepkv_decode_attention, without ws / ws_bytes; inputs and outputs stay the caller's.
- *  - Shapes whose decode scratch (4 bytes per unit, U = B*H_kv, plus a pool of 1024 partial results of
- *    (16 + G*d) floats, each rounded up to 256-byte pieces) exceeds the array are refused with
- *    KEEPKV_ERR_WORKSPACE before anything is enqueued; G = 8, d = 128 leaves room for 900 000 units.
+ *  - Shapes whose decode scratch exceeds the array are refused with KEEPKV_ERR_WORKSPACE before
+ *    anything is enqueued.  The exact rule, with U = B*H_kv and align256(x) = x rounded up to a multiple
+ *    of 256:  align256(4*(U+1)) + align256(1024*(16 + G*d)*4) <= KEEPKV_STATIC_SCRATCH_BYTES
+ *    (G = 8, d = 128: the pool takes 4 259 840 bytes, which leaves room for 1 032 191 units).
+ *  - Every call clears the 4*(U+1) bytes of arrival counters with a cudaMemsetAsync on `stream` before its
+ *    kernel (3.6 MB at the largest admissible U; a few hundred bytes for ordinary batches).
  *  - The first call on each device looks up the array's device address; make that call outside any
  *    stream capture, with the device current that `stream` belongs to.
  *  - All calls on one GPU share the array and find in it whatever the previous call left: the call

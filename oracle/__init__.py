@@ -182,7 +182,7 @@ def cosine(ke, kc):
 
 
 def match(P: Params, K, ret_idx):
-    """Algorithm 1 lines 4-5.  Returns (target [len] int32, umax [len] f32, second [len] f32)."""
+    """Algorithm 1, similarity and arg-max steps.  Returns (target [len] int32, umax [len] f32, second [len] f32)."""
     K = _f64(K)
     ret_idx = np.ascontiguousarray(ret_idx, dtype=np.int32)
     n = K.shape[0]

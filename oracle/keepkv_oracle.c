@@ -23,7 +23,7 @@
  * EMA estimate of s_i (Eq. 8), G query heads sharing one kv head.
  *
  * Parity unpinned (the paper prints nothing that fixes them; they are readings
- * stated in the design notes): the GQA score reduction (mean over the group),
+ * fixed by this oracle): the GQA score reduction (mean over the group),
  * first-observation initialisation of the EMA, the sink/recent/heavy split of the
  * selection, the gamma guard, and the ascending order of the compacted cache.
  */
@@ -44,7 +44,7 @@ typedef struct {
   int32_t pad_;
   double sm_scale;          /* 1/sqrt(d), Eq. 3                                     */
   double ema_alpha;         /* alpha of Eq. 8                                       */
-  double merge_threshold;   /* T of Algorithm 1 line 5; -inf merges always          */
+  double merge_threshold;   /* T of Algorithm 1, arg-max and threshold step; -inf merges always          */
   double gamma_min;         /* guard on the key rescale factor: merge iff           */
   double gamma_max;         /*   gamma_min < gamma <= gamma_max and |lambda_bar|>=1e-6 */
 } okv_params;
@@ -275,7 +275,7 @@ int32_t okv_select_sorted(int32_t len, const float *kappa, int32_t budget, int32
   return n;
 }
 
-/* -------------------------------------------- Algorithm 1 lines 4-5: match */
+/* -------------------------------------------- Algorithm 1, similarity and arg-max steps: match */
 
 /* The fixed fp32 recipe for cosine similarity: sequential fused multiply-adds
  * from 0.0f over j = 0..d-1 for the dot product and both squared norms, then

@@ -11,7 +11,7 @@ __global__ void __launch_bounds__(128) append_kernel(keepkv_params p, keepkv_cac
   pdl_wait();
   pdl_trigger();
   const int pos = c.seq_len[b];
-  if (pos >= p.N_cap) {
+  if (pos < 0 || pos >= p.N_cap) {   // full, or a length that is not one: skipped and reported, never written
     if (threadIdx.x == 0) atomicOr(status_dev, KEEPKV_DEV_APPEND_FULL);
     return;
   }

@@ -1,12 +1,12 @@
 // keepkv_compress: Algorithm 1 of the paper, out of place, one (sequence, kv-head) unit at a time.
-//   select   -> retained / evicted sets from the key kappa = ln p + lscore       (lines 2-3)
-//   compact  -> retained rows copied to dst in ascending source order            (line 11)
-//   nominate -> three best cosines of every evicted key over the retained keys,
-//               on the tensor cores (nominate.cu)                                (line 4)
-//   resolve  -> arg-max and threshold of line 5, decided in the interface's fixed fp32
+//   select   -> retained / evicted sets from the key kappa = ln p + lscore       (Algorithm 1, selection step)
+//   compact  -> retained rows copied to dst in ascending source order            (Algorithm 1, insertion step)
+//   nominate -> two best cosines of every evicted key over the retained keys,
+//               on the tensor cores (nominate.cu)                                (Algorithm 1, similarity step)
+//   resolve  -> arg-max and threshold of Algorithm 1, decided in the interface's fixed fp32
 //               arithmetic wherever the tensor-core ranking is too close to call; members
 //               of each retained slot sorted into groups                         (many-to-one, App. A.2)
-//   merge    -> Eq. A.3 with the EMA estimate as score                           (lines 7-10)
+//   merge    -> Eq. A.3 with the EMA estimate as score                           (Algorithm 1, merge step)
 #include "compress.cuh"
 
 namespace keepkv {

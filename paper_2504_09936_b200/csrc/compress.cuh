@@ -273,11 +273,15 @@ __device__ __forceinline__ void merge_group(const keepkv_params &p, const keepkv
   const __nv_bfloat16 *sK = reinterpret_cast<const __nv_bfloat16 *>(src.K) + base * D;
   const __nv_bfloat16 *sV = reinterpret_cast<const __nv_bfloat16 *>(src.V) + base * D;
 
-  float ka[EPL], va[EPL], lbar = 0.f, L, Ps;
+  // The group's scalars are evaluated in fp64: L = LSE(a) - ln(sum p) and lambda_bar cancel to almost nothing
+  // when the members' log-scores sit near zero, and gamma = L / lambda_bar then carries whatever relative error
+  // they have into every channel of the merged key (an fp32 L of 1e-5 is off by a percent).  A handful of
+  // double-precision logarithms per group cost nothing next to the rows it loads; the row sums stay fp32.
+  float ka[EPL], va[EPL];
+  double lbar = 0.0, L, Ps;
 #pragma unroll
   for (int e = 0; e < EPL; ++e) { ka[e] = 0.f; va[e] = 0.f; }
-  auto accumulate = [&](int i, float om, float lsi) {
-    lbar = fmaf(om, lsi, lbar);
+  auto accumulate = [&](int i, float om) {
     if constexpr (EPL == 4) {
       const uint2 kk = *reinterpret_cast<const uint2 *>(sK + (size_t)i * D + lane * 4);
       const uint2 vv = *reinterpret_cast<const uint2 *>(sV + (size_t)i * D + lane * 4);
@@ -292,42 +296,62 @@ __device__ __forceinline__ void merge_group(const keepkv_params &p, const keepkv
       va[0] = fmaf(om, bf16_lo(vv), va[0]); va[1] = fmaf(om, bf16_hi(vv), va[1]);
     }
   };
+  auto wsum_d = [](double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+  };
+  auto wmax_d = [](double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+  };
+  const double NEG_INF = -CUDART_INF;
   if (n < 32) {
     // the usual case: lane 0 holds the target, lane t the t-th member, so that their votes and scores are
     // fetched together and the row loads of the accumulation do not wait on one another
     const int idx = lane == 0 ? ci : (lane <= n ? member(lane - 1) : -1);
     const float pv = idx >= 0 ? votes[idx] : 0.f, lsv = idx >= 0 ? ls[idx] : 0.f;
-    const float a = idx >= 0 ? logf(pv) + lsv : -CUDART_INF_F;
-    const float M = warp_max(a);
-    const float Z = warp_sum(idx >= 0 ? expf(a - M) : 0.f);
-    Ps = warp_sum(pv);
-    const float Lam = M + logf(Z);
-    L = Lam - logf(Ps);
-    const float om = idx >= 0 ? expf(a - Lam) : 0.f;
+    const double a = idx >= 0 ? log((double)pv) + (double)lsv : NEG_INF;
+    const double M = wmax_d(a);
+    const double Z = wsum_d(idx >= 0 ? exp(a - M) : 0.0);
+    Ps = wsum_d((double)pv);
+    const double Lam = M + log(Z);
+    L = Lam - log(Ps);
+    const double omd = idx >= 0 ? exp(a - Lam) : 0.0;
+    lbar = wsum_d(omd * (double)lsv);
+    const float om = (float)omd;
 #pragma unroll 4
-    for (int t = 0; t <= n; ++t)
-      accumulate(__shfl_sync(0xffffffffu, idx, t), __shfl_sync(0xffffffffu, om, t), __shfl_sync(0xffffffffu, lsv, t));
+    for (int t = 0; t <= n; ++t) accumulate(__shfl_sync(0xffffffffu, idx, t), __shfl_sync(0xffffffffu, om, t));
   } else {
-    const float a_c = logf(votes[ci]) + ls[ci];
-    float M = a_c;
-    for (int t = lane; t < n; t += 32) { const int e = member(t); M = fmaxf(M, logf(votes[e]) + ls[e]); }
-    M = warp_max(M);
-    float Z = 0.f;
-    Ps = 0.f;
-    if (lane == 0) { Z = expf(a_c - M); Ps = votes[ci]; }
-    for (int t = lane; t < n; t += 32) { const int e = member(t); Z += expf(logf(votes[e]) + ls[e] - M); Ps += votes[e]; }
-    Z = warp_sum(Z);
-    Ps = warp_sum(Ps);
-    const float Lam = M + logf(Z);
-    L = Lam - logf(Ps);
+    const double a_c = log((double)votes[ci]) + (double)ls[ci];
+    double M = a_c;
+    for (int t = lane; t < n; t += 32) { const int e = member(t); M = fmax(M, log((double)votes[e]) + (double)ls[e]); }
+    M = wmax_d(M);
+    double Z = 0.0;
+    Ps = 0.0;
+    if (lane == 0) { Z = exp(a_c - M); Ps = (double)votes[ci]; }
+    for (int t = lane; t < n; t += 32) {
+      const int e = member(t);
+      Z += exp(log((double)votes[e]) + (double)ls[e] - M);
+      Ps += (double)votes[e];
+    }
+    Z = wsum_d(Z);
+    Ps = wsum_d(Ps);
+    const double Lam = M + log(Z);
+    L = Lam - log(Ps);
+    // every lane walks all members (the rows are spread over the lanes by channel), so lambda_bar is summed per lane
     for (int t = -1; t < n; ++t) {
       const int i = t < 0 ? ci : member(t);
-      const float lsi = ls[i];
-      accumulate(i, expf(logf(votes[i]) + lsi - Lam), lsi);
+      const double lsi = (double)ls[i];
+      const double omd = exp(log((double)votes[i]) + lsi - Lam);
+      lbar += omd * lsi;
+      accumulate(i, (float)omd);
     }
   }
-  const float gamma = L / lbar;
-  const bool ok = gamma > p.gamma_min && gamma <= p.gamma_max && fabsf(lbar) >= 1e-6f;
+  const double gamma_d = L / lbar;
+  const float gamma = (float)gamma_d;
+  const bool ok = gamma_d > (double)p.gamma_min && gamma_d <= (double)p.gamma_max && fabs(lbar) >= 1e-6;
   if (!ok) {
     // guard: the members are dropped after all and the target keeps the row copied by compaction
     for (int t = lane; t < n; t += 32) target_u[member(t)] = -1;
@@ -347,8 +371,8 @@ __device__ __forceinline__ void merge_group(const keepkv_params &p, const keepkv
     *reinterpret_cast<uint32_t *>(dV + lane * 2) = pack_bf16(va[0], va[1]);
   }
   if (lane == 0) {
-    dst.votes[base + c] = Ps;
-    dst.lscore[base + c] = L;
+    dst.votes[base + c] = (float)Ps;
+    dst.lscore[base + c] = (float)L;
     atomicAdd(&st->n_merged, n);
     atomicAdd(&st->n_groups, 1);
     atomicMax(&st->max_group, n);

@@ -2,18 +2,18 @@
 // period over its budget.  A unit qualifies when it evicts at most kStEv entries and has at most kStCand
 // entries between the sinks and the recent window; the others are reported and left alone.  The R CTAs of
 // a unit (grid (R, U)) each
-//   1. repeat the selection (lines 2-3): keys of the candidates in shared memory, a radix search,
+//   1. repeat the selection (Algorithm 1, selection step): keys of the candidates in shared memory, a radix search,
 //      one ordered pass -> the kept candidates and the evicted entries as lists in shared memory;
-//   2. stream their slice of the retained slots src -> dst (line 11), 64 slots at a time.  The key rows go
+//   2. stream their slice of the retained slots src -> dst (Algorithm 1, insertion step), 64 slots at a time.  The key rows go
 //      global -> shared by cp.async into a ring of 128-byte-swizzled tiles, three tiles ahead of their use (a
 //      slice that lies in the recent window does not depend on the selection and starts before it), and are
 //      stored to dst from there; values pass through registers.  The key tiles are the B operand of a tcgen05.mma (M = 128 evicted keys, staged once as A operand; N = 64; fp32
-//      accumulators in tensor memory, double-buffered) that one thread issues per tile (line 4).  All eight
+//      accumulators in tensor memory, double-buffered) that one thread issues per tile (Algorithm 1, similarity step).  All eight
 //      warps drain the accumulator of the previous tile with tcgen05.ld while the next product runs: a thread
 //      owns one evicted row and half of the columns and keeps the row's two best cosines with their slots;
 //   3. leave their two best per row in the workspace; the last CTA of the unit to arrive folds them, settles
-//      arg-max and threshold (line 5) with the interface's exact fp32 chain wherever the tensor-core ranking is
-//      closer than kRankEps, sorts the entries to merge into groups and merges them (Eq. A.3, lines 7-10).
+//      arg-max and threshold (Algorithm 1, arg-max and threshold step) with the interface's exact fp32 chain wherever the tensor-core ranking is
+//      closer than kRankEps, sorts the entries to merge into groups and merges them (Eq. A.3; Algorithm 1, merge step).
 // Decisions, and therefore all outputs, are the same bits as the general pipeline's (compress.cu).
 // Every wait on the tensor core is bounded; one that runs out raises KEEPKV_DEV_TIMEOUT and the CTA goes on
 // without further products (its unit's result is then unspecified), frees its tensor memory and returns.
@@ -89,7 +89,7 @@ steady_compress_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, cons
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   pdl_wait();
   pdl_trigger();
-  // ---- the sets of Algorithm 1 lines 2-3, exactly as the general selection defines them
+  // ---- the sets of Algorithm 1, selection step, exactly as the general selection defines them
   const int len = max(0, min(src.seq_len[b], p.N_cap));
   int budget = budget_dev ? budget_dev[b] : budget_scalar;
   budget = max(0, min(budget, p.N_cap));
@@ -173,7 +173,7 @@ steady_compress_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, cons
   const bool early = t0 * kStN >= lo + n_heavy;
   if (early) { issue_keys(t0); issue_keys(t0 + 1); issue_keys(t0 + 2); load_values(t0); }
 
-  // ---- selection (lines 2-3)
+  // ---- selection (Algorithm 1, selection step)
   for (int i = tid; i < m_cand; i += kStThreads)   // the caller's scores where given, else kappa = ln p + lscore
     keys[i] = select_key ? ordered_key(select_key[base + lo + i])
                          : kappa_key(src.votes[base + lo + i], src.lscore[base + lo + i]);
@@ -231,7 +231,7 @@ steady_compress_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, cons
   top.init(0.f);
   topb.init(0.f);
   {
-    // The copy (line 11) of tile t, whose keys have landed in their stage and whose values are in vr, with the
+    // The copy (Algorithm 1, insertion step) of tile t, whose keys have landed in their stage and whose values are in vr, with the
     // per-slot records and the inverse norms the product ranks with.
     auto copy_tile = [&](int t) {
       const uint8_t *st = st_smem + SL::kRing + ((t - t0) % S) * SL::kStageBytes;
@@ -405,7 +405,7 @@ steady_compress_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, cons
     }
   }
 
-  // ---- line 5: arg-max and threshold; the interface's exact arithmetic where the ranking is too close to call
+  // ---- Algorithm 1, arg-max and threshold step: arg-max and threshold; the interface's exact arithmetic where the ranking is too close to call
   float *ke_s = reinterpret_cast<float *>(st_smem + SL::kKe), *kc_s = reinterpret_cast<float *>(st_smem + SL::kKc);
   int *qs = reinterpret_cast<int *>(st_smem + SL::kQ);
   int *q_tid = qs, *q_e = qs + kStEv, *q_kind = qs + 2 * kStEv, *q_a = qs + 3 * kStEv, *q_b = qs + 4 * kStEv,
@@ -473,7 +473,7 @@ steady_compress_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, cons
     if (h == 0) dst.seq_len[b] = n_ret;
   }
   __syncthreads();
-  // ---- lines 7-10: one warp per group
+  // ---- Algorithm 1, merge step: one warp per group
   for (int gi = warp; gi < n_groups; gi += kStWarps) {
     const int beg = ghead[gi], n = ghead[gi + 1] - beg;
     const int c = (int)(skey[beg] >> 16);

@@ -1,7 +1,7 @@
-// Similarity search of keepkv_compress (Algorithm 1 line 4: U = cosineSimilarity(K_e, K_c)) on the
+// Similarity search of keepkv_compress (Algorithm 1, similarity step: U = cosineSimilarity(K_e, K_c)) on the
 // 5th-generation tensor cores.  The cosine matrix is never stored: for every evicted key the kernel
 // keeps the two largest cosines over the retained keys and their slots, which is all the arg-max
-// of line 5 needs.  The values found here only *rank* candidates; wherever the
+// of Algorithm 1 needs.  The values found here only *rank* candidates; wherever the
 // ranking is closer than the accumulation error allows, the caller re-evaluates the candidates in
 // the fixed fp32 arithmetic the interface defines (see resolve_kernel in compress.cu).
 //

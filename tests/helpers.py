@@ -140,9 +140,15 @@ def check_decode_unit(p, u, hc: HostCache, q64, out_gpu64, lse_gpu, lscore_after
 
 
 def check_compress_unit(p, u, budget, n_recent, hc_src: HostCache, hc_dst: HostCache, ret_idx, target, stats=None,
-                        what="", sorted_select=True, select_key=None):
+                        what="", sorted_select=True, select_key=None, max_tolerated=0):
     """Teacher-forced staged check of one unit of a compress call: the oracle is fed the same source
-    state; index sets and merge targets must match exactly, tensors within the bf16 rules."""
+    state; index sets and merge targets must match exactly, tensors within the bf16 rules.
+
+    The only tolerated difference is a group whose rescale factor sits on the edge of the gamma guard
+    in the oracle (within 1e-3 relative): the two sides may then disagree on whether that ONE slot is
+    merged, so the targets of its members and the row of that slot are excused.  Every other slot is
+    still compared.  Returns (oracle result, number of excused source entries); more than
+    `max_tolerated` of them fail the check."""
     P = oracle_params(p, n_recent=n_recent)
     K, V, votes, ls = hc_src.unit(u)
     n = K.shape[0]
@@ -152,25 +158,31 @@ def check_compress_unit(p, u, budget, n_recent, hc_src: HostCache, hc_dst: HostC
     b = u // p.H_kv
     assert int(hc_dst.seq_len[b]) == m, f"{what} u={u}: new seq_len {hc_dst.seq_len[b]} != {m}"
     assert np.array_equal(ret_idx[u, :m], ref["ret_idx"]), f"{what} u={u}: retained set differs"
-    # merge targets: exact, except where the oracle's guard sits on its edge or its top cosines tie
     tg, tr = target[u, :n], ref["target"]
-    if not np.array_equal(tg, tr):
-        _, umax, second = O.match(P, K, ref["ret_idx"])
-        diff = np.nonzero(tg != tr)[0]
-        gam = ref["gammas"]
-        for e in diff:
-            near_tie = abs(float(umax[e]) - float(second[e])) < 1e-5 or abs(float(umax[e]) - P.merge_threshold) < 1e-6
-            slots = [s for s in (tg[e], tr[e]) if s >= 0]
-            edge = any(np.isfinite(gam[s]) and (min(abs(gam[s] - P.gamma_min), abs(gam[s] - P.gamma_max))
-                                                 < 1e-3 * max(1.0, abs(gam[s]))) for s in slots)
-            assert near_tie or edge, f"{what} u={u}: target of entry {e}: gpu {tg[e]} oracle {tr[e]}"
-        return ref, False   # tensors of affected slots may legitimately differ: skip tensor check
+    excused_slots = set()
+    diff = np.nonzero(tg != tr)[0]
+    gam = ref["gammas"]
+    for e in diff:
+        slots = [int(s) for s in (tg[e], tr[e]) if s >= 0]
+        # the entry's target itself must agree wherever both sides name one: only "merged or not" may differ
+        assert len(slots) == 1 or slots[0] == slots[1], f"{what} u={u}: target of entry {e}: gpu {tg[e]} oracle {tr[e]}"
+        s = slots[0] if slots else -1
+        edge = s >= 0 and np.isfinite(gam[s]) and (min(abs(gam[s] - P.gamma_min), abs(gam[s] - P.gamma_max))
+                                                   < 1e-3 * max(1.0, abs(gam[s])))
+        assert edge, f"{what} u={u}: target of entry {e}: gpu {tg[e]} oracle {tr[e]} (not on the guard's edge)"
+        excused_slots.add(s)
+    n_tol = int(len(diff))
+    assert n_tol <= max_tolerated, f"{what} u={u}: {n_tol} entries excused by the guard edge (> {max_tolerated})"
+    keep = np.ones(m, dtype=bool)
+    keep[list(excused_slots)] = False
     dK, dV, dvotes, dls = hc_dst.unit(u)
-    assert np.array_equal(dvotes, ref["votes"]), f"{what} u={u}: votes differ"
-    check_close(dK, ref["K"], f"{what} K u={u}")
-    check_close(dV, ref["V"], f"{what} V u={u}")
-    check_close(dls, ref["lscore"], f"{what} lscore u={u}", ulps=None, max_abs=1e-4, mean_rel=1e-5)
+    assert np.array_equal(dvotes[keep], ref["votes"][keep]), f"{what} u={u}: votes differ"
+    check_close(dK[keep], ref["K"][keep], f"{what} K u={u}")
+    check_close(dV[keep], ref["V"][keep], f"{what} V u={u}")
+    check_close(dls[keep], ref["lscore"][keep], f"{what} lscore u={u}", ulps=None, max_abs=1e-4, mean_rel=1e-5)
     if stats is not None:
-        for f in ("n_retained", "n_evicted", "n_merged", "n_below_T", "n_guard_groups", "n_groups", "max_group"):
+        exact = ("n_retained", "n_evicted") if n_tol else ("n_retained", "n_evicted", "n_merged", "n_below_T",
+                                                           "n_guard_groups", "n_groups", "max_group")
+        for f in exact:
             assert int(stats[u][kb.STATS_FIELDS.index(f)]) == ref["stats"][f], (what, u, f, stats[u], ref["stats"])
-    return ref, True
+    return ref, n_tol

@@ -238,3 +238,128 @@ def test_largest_capacity():
     dst, ret, tgt, stats = _compress(p, cache, 160)
     check_compress_unit(p, 0, 160, p.n_recent, src, UnitView(dst, [0]), ret, tgt, stats, what="largest capacity compress")
     assert int(st.item()) == 0
+
+
+# ---------------------------------------------------------------------------------------------------
+# The remaining workloads at their stated shapes, in the launch configuration the benchmark times:
+# capacity, parameters, per-sequence budgets and the steady-state flag exactly as bench.py sets them.
+# Every stage runs on ALL units through the library; a few sampled units are compared with the oracle,
+# teacher-forced (the oracle is fed the library's state before the stage).
+
+def _with_fresh_row(view: UnitView, units, kn64, vn64, H_kv):
+    """The view of a cache after Eq. 2 appended (kn, vn) to every sampled unit: what the attention of a
+    keepkv_decode_step call must see."""
+    out = UnitView.__new__(UnitView)
+    out.H = view.H
+    out.seq_len = view.seq_len + 1
+    out._u = {}
+    for u in units:
+        b, h = divmod(u, H_kv)
+        n = int(view.seq_len[b])
+        K, V, p, ls = (a.copy() for a in view._u[u])
+        K[n], V[n], p[n], ls[n] = kn64[b, h], vn64[b, h], 1.0, -math.inf
+        out._u[u] = (K, V, p, ls)
+    return out
+
+
+def _protocol_at_stated_shape(name, units, layer=0):
+    w = W.CONFIGS[name]
+    P_ = w.period
+    n_cap = -(-(w.N + P_) // 64) * 64                     # as bench.py
+    p = workload_params(w, n_cap=n_cap)
+    cache = workload_cache(w, n_cap=n_cap, layer=layer)
+    lens = cache.seq_len.cpu().numpy()
+    bud = np.array([w.budget(int(n)) for n in lens], dtype=np.int32)
+    nrec = np.array([w.n_recent(int(x)) for x in bud], dtype=np.int32)
+    ragged = bool(np.any(bud != bud[0]))
+    steady = P_ <= 128 and int(np.max(bud + P_ - w.n_sink - nrec)) <= 2048 and int(np.max(bud)) <= 16384
+    budget_arg = torch.from_numpy(bud).cuda() if ragged else int(bud[0])
+    nrec_arg = torch.from_numpy(nrec).cuda() if ragged else None
+    p_inc = workload_params(w, n_cap=n_cap, flags=kb.FLAG_COMPRESS_STEADY if steady else 0)
+    ws, st = kb.new_workspace(p), kb.new_status()
+    U = w.U
+    q_all, kn_all, vn_all = W.make_step_inputs(w, layer, 0, P_ + 1)
+    out = torch.empty(w.B, w.H_q, w.d, dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty(w.B, w.H_q, dtype=torch.float32, device="cuda")
+    Por = oracle_params(p)
+
+    def compress(pp, src, stage):
+        dst = kb.Cache.empty(p)
+        ret = torch.full((U, n_cap), -7, dtype=torch.int32, device="cuda")
+        tgt = torch.full((U, n_cap), -7, dtype=torch.int32, device="cuda")
+        stats = torch.zeros(U, 8, dtype=torch.int32, device="cuda")
+        before = UnitView(src, units)
+        kb.keepkv_compress(pp, src, dst, budget_arg, ws, st, n_recent_dev=nrec_arg, retained_idx=ret, target=tgt,
+                           stats=stats)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0, f"{name} {stage}: status {int(st.item())}"
+        assert dst.seq_len.cpu().numpy().tolist() == np.minimum(bud, src.seq_len.cpu().numpy()).tolist()
+        after = UnitView(dst, units)
+        ret, tgt, stats = ret.cpu().numpy(), tgt.cpu().numpy(), stats.cpu().numpy()
+        for u in units:
+            bb = u // w.H_kv
+            # a handful of entries may sit in a group on the edge of the gamma guard; everything else is exact
+            check_compress_unit(p, u, int(bud[bb]), int(nrec[bb]), before, after, ret, tgt, stats,
+                                what=f"{name} {stage}", max_tolerated=8)
+        return dst
+
+    # ---- Eq. 8, first case: scores at the end of prefill from a 32-query window
+    Wq = 32
+    qwin = bits_to_dev(q_all[1:1 + Wq]).permute(1, 2, 0, 3).contiguous()         # [B, H_q, W, d]
+    before = UnitView(cache, units)
+    kb.keepkv_prefill_scores(p, cache, qwin, st)
+    torch.cuda.synchronize()
+    q64 = to_f64(qwin)
+    for u in units:
+        b, h = divmod(u, w.H_kv)
+        K = before.unit(u)[0]
+        qu = np.ascontiguousarray(q64[b, h * w.G:(h + 1) * w.G].transpose(1, 0, 2))
+        ref = O.prefill_scores(Por, qu, K)
+        check_close(to_f64(cache.lscore[b, h, :len(ref)]), ref, f"{name} prefill scores u={u}", ulps=None,
+                    max_abs=1e-3, mean_rel=1e-4)
+    # ---- step 0 on the whole prompt (Eq. 6 + Eq. 8)
+    before = UnitView(cache, units)
+    q0 = bits_to_dev(q_all[0])
+    kb.keepkv_decode_attention(p, cache, q0, out, lse, True, ws, st)
+    torch.cuda.synchronize()
+    _check_decode(p, before, units, q0, out, cache.lscore, f"{name} step 0", lse=lse)
+    # ---- first compression: prompt -> budget (general pipeline)
+    cur = compress(p, cache, "first compression")
+    del cache
+    # ---- one period of decode steps (append folded into the attention launch, as the benchmark runs it)
+    for t in range(1, P_ + 1):
+        if t == P_:
+            torch.cuda.synchronize()
+            before = UnitView(cur, units)
+        q = bits_to_dev(q_all[t])
+        kb.keepkv_decode_step(p, cur, q, bits_to_dev(kn_all[t]), bits_to_dev(vn_all[t]), out, lse, True, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0 and cur.seq_len.cpu().numpy().tolist() == (bud + P_).tolist()
+    seen = _with_fresh_row(before, units, to_f64(bits_to_dev(kn_all[P_])), to_f64(bits_to_dev(vn_all[P_])), w.H_kv)
+    _check_decode(p, seen, units, q, out, cur.lscore, f"{name} last step of the period", lse=lse)
+    # ---- steady-state compression: budget + P -> budget (one kernel where the benchmark uses it)
+    compress(p_inc, cur, "steady-state compression")
+    return steady
+
+
+def test_c3_stated_shape_sampled_units():
+    """Workload C3: 16 sequences x 32 heads (G = 1), 4096-entry prompts, budget 410, period 64, drifting
+    queries: prompt scoring, step 0, first compression 4096 -> 410 on all 512 units, 64 decode steps, the
+    steady-state compression 474 -> 410; units of the first, a middle and the last sequence checked."""
+    assert _protocol_at_stated_shape("C3", [0, 5 * 32 + 17, 511]) is True
+
+
+def test_c4_stated_shape_sampled_unit():
+    """Workload C4 (one of its 32 layers): 2 sequences x 8 kv heads (G = 4, d = 128), 32768-entry prompts,
+    budget 3277, period 256: the similarity search runs 13 column tiles in chunks over 29 491 evicted rows
+    per unit, several CTAs resolve a unit, the steady-state compression takes the general pipeline."""
+    assert _protocol_at_stated_shape("C4", [11], layer=3) is False
+
+
+def test_c5_stated_shape_sampled_units():
+    """Workload C5: 64 sequences x 8 kv heads (G = 8), ragged prompts of 4096-16384 entries, per-sequence
+    budgets (10 %) and recent windows, period 128; a head of the longest and one of the shortest sequence."""
+    w = W.CONFIGS["C5"]
+    lens = W.seq_lens(w, 0)
+    b_long, b_short = int(np.argmax(lens)), int(np.argmin(lens))
+    assert _protocol_at_stated_shape("C5", [b_long * 8 + 3, b_short * 8 + 6]) is True

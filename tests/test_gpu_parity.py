@@ -123,6 +123,26 @@ def test_append_equation_2_and_full_cache_flag():
         assert np.array_equal(after.K[4 + h], before.K[4 + h]) and np.array_equal(after.votes[4 + h], before.votes[4 + h])
 
 
+def test_append_skips_a_negative_length():
+    """A length that is not one (here -3, as an uninitialised buffer might hold) is reported like a full
+    sequence and nothing of that sequence is written; the other sequence is appended normally."""
+    p = kb.make_params(B=2, H_q=4, H_kv=2, d=64, N_cap=64)
+    cache = random_cache(p, [5, 7], seed=4)
+    cache.seq_len[0] = -3
+    snap = [t.clone() for t in (cache.K, cache.V, cache.votes, cache.lscore)]
+    rng = np.random.default_rng(1)
+    kn = f32_to_dev_bf16(rng.standard_normal((2, 2, 64)).astype(np.float32))
+    vn = f32_to_dev_bf16(rng.standard_normal((2, 2, 64)).astype(np.float32))
+    st = kb.new_status()
+    kb.keepkv_append(p, cache, kn, vn, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == kb.DEV_APPEND_FULL and cache.seq_len.tolist() == [-3, 8]
+    for before, after in zip(snap, (cache.K, cache.V, cache.votes, cache.lscore)):
+        assert torch.equal(before[0].view(torch.int16) if before.dtype == torch.bfloat16 else before[0].view(torch.int32),
+                           after[0].view(torch.int16) if after.dtype == torch.bfloat16 else after[0].view(torch.int32))
+    assert torch.equal(cache.K[1, :, 7].view(torch.int16), kn[1].view(torch.int16)) and torch.all(cache.votes[1, :, 7] == 1)
+
+
 def _run_compress(p, src, budget, n_recent_dev=None):
     dst = kb.Cache.empty(p)
     ws = kb.new_workspace(p)
@@ -152,11 +172,14 @@ def test_compress_staged_parity(d, G, T, guard):
     budget = 70
     dst, ret, tgt, stats = _run_compress(p, src, budget)
     hs, hd = HostCache(src), HostCache(dst)
-    n_full = 0
+    n_excused = 0
     for u in range(B * H_kv):
-        _, full = check_compress_unit(p, u, budget, p.n_recent, hs, hd, ret, tgt, stats, what=f"T={T}")
-        n_full += full
-    assert n_full >= B * H_kv - 1
+        # a group on the edge of the gamma guard may legitimately go either way: at most one such group in the
+        # whole batch, everything else exact
+        _, n_tol = check_compress_unit(p, u, budget, p.n_recent, hs, hd, ret, tgt, stats, what=f"T={T}",
+                                       max_tolerated=40 if guard else 0)
+        n_excused += 1 if n_tol else 0
+    assert n_excused <= 1
 
 
 def test_compress_ragged_budgets_and_copy_through():
@@ -591,11 +614,8 @@ def test_compress_with_caller_supplied_selection_scores(flags):
     assert int(st.item()) == 0
     hs, hd = HostCache(src), HostCache(dst)
     ret, tgt, stats = ret.cpu().numpy(), tgt.cpu().numpy(), stats.cpu().numpy()
-    n_full = 0
     for u in range(U):
-        _, full = check_compress_unit(p, u, budget, n_recent, hs, hd, ret, tgt, stats, what="scored", select_key=key)
-        n_full += full
-    assert n_full >= U - 1
+        check_compress_unit(p, u, budget, n_recent, hs, hd, ret, tgt, stats, what="scored", select_key=key)
     # and the scores did change the outcome: the default selection keeps a different set
     dst0, ret0, _, _ = _run_compress(p, src, budget)
     assert not np.array_equal(ret0[0, :budget], ret[0, :budget])

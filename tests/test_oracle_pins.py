@@ -207,7 +207,7 @@ def test_kappa_is_log_of_vote_weighted_score():
     assert abs(float(k[1]) - (math.log(2.0) - 3.0)) < 1e-6
 
 
-# ------------------------------------------------- Algorithm 1 lines 4-5: match
+# ------------------------------------------------- Algorithm 1, similarity and arg-max steps: match
 
 def test_match_agrees_with_fp64_cosine_away_from_ties():
     rng = RNG(7)
