@@ -227,6 +227,15 @@ int keepkv_decode_step_host_layers(const keepkv_params *p, const keepkv_cache *c
 int keepkv_decode_attention_static(const keepkv_params *p, const keepkv_cache *cache, const void *q, void *out,
                                    float *lse_or_null, int update_scores, int32_t *status_dev, void *stream);
 
+/* Test hook, not for production use: process-wide settings of the decode launches that follow (keepkv_decode_attention,
+ * keepkv_decode_step, their host and static variants).  spin_limit > 0 replaces the number of polls after which a
+ * bounded wait inside the kernel gives up (0 restores the default).  withhold_tile >= 0 makes every CTA announce
+ * the tile at that position of its tile sequence without ever issuing its copies, so that the wait for it runs out with
+ * nothing in flight: the call then returns normally, KEEPKV_DEV_TIMEOUT is raised in *status_dev and the outputs of
+ * that call are unspecified; -1 restores normal operation.  This is how the kernels' timeout path is exercised
+ * without faulting or hanging a GPU. */
+int keepkv_debug_decode(int spin_limit, int withhold_tile);
+
 /* Human-readable name of a keepkv_status. */
 const char *keepkv_status_string(int status);
 

@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkeepkv.so")
 
 EXPORTS = ("keepkv_workspace_bytes", "keepkv_workspace_init", "keepkv_append", "keepkv_decode_attention",
-           "keepkv_decode_step", "keepkv_compress", "keepkv_compress_scored", "keepkv_prefill_scores", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_status_string", "keepkv_last_cuda_error",
+           "keepkv_decode_step", "keepkv_compress", "keepkv_compress_scored", "keepkv_prefill_scores", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_debug_decode", "keepkv_status_string", "keepkv_last_cuda_error",
            "keepkv_last_launch_count")
 
 
@@ -64,6 +64,7 @@ def lib() -> C.CDLL:
         l.keepkv_decode_attention.argtypes = [pp, pc, vp, vp, vp, C.c_int, vp, sz, vp, vp]
         l.keepkv_decode_step.argtypes = [pp, pc, vp, vp, vp, vp, vp, C.c_int, vp, sz, vp, vp]
         l.keepkv_decode_attention_static.argtypes = [pp, pc, vp, vp, vp, C.c_int, vp, vp]
+        l.keepkv_debug_decode.argtypes = [C.c_int, C.c_int]
         l.keepkv_prefill_scores.argtypes = [pp, pc, vp, i32, vp, vp]
         l.keepkv_compress.argtypes = [pp, pc, pc, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         l.keepkv_compress_scored.argtypes = [pp, pc, pc, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
@@ -212,6 +213,11 @@ def keepkv_decode_step_host_layers(p, caches, q_host, k_new_host, v_new_host, ou
                                                 k_new_dev.data_ptr(), v_new_dev.data_ptr(), out_dev.data_ptr(),
                                                 int(update_scores), ws.data_ptr(), ws.numel(), status.data_ptr(),
                                                 _stream(stream)), "keepkv_decode_step_host_layers")
+
+
+def keepkv_debug_decode(spin_limit: int = 0, withhold_tile: int = -1):
+    """Test hook: bounded-wait poll count and a tile position whose copies are withheld (see the header)."""
+    _check(lib().keepkv_debug_decode(int(spin_limit), int(withhold_tile)), "keepkv_debug_decode")
 
 
 def last_launch_count() -> int:

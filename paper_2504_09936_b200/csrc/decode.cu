@@ -31,6 +31,8 @@
 // it to the cache), so that the attention sees it.  The new lengths are published when nobody reads the old
 // ones any more: every CTA copies the lengths into shared memory first and then signs off on a counter, and
 // the last one to sign off writes them (batches beyond kSeqCache sequences: the last CTA to finish does).
+#include <mutex>
+
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -92,6 +94,13 @@ __device__ __forceinline__ float lg2f(float x) {
   return y;
 }
 
+// Bounded wait with a caller-chosen number of polls.
+__device__ __forceinline__ bool mbar_wait_n(uint32_t bar, uint32_t parity, int limit) {
+  for (int it = 0; it < limit; ++it)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+
 // One partial result of a unit: running maxima (base-2 exponents), sums and numerators of its G heads.
 template <int D, int G>
 struct PartRec {
@@ -104,7 +113,7 @@ __global__ void __launch_bounds__(kDecThreads, 2)
 decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, keepkv_params p,
               keepkv_cache c, const __nv_bfloat16 *__restrict__ q, __nv_bfloat16 *__restrict__ out,
               float *__restrict__ lse, int update_scores, int *counters, PartRec<D, G> *pool, int32_t *status_dev,
-              const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new) {
+              const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new, int spin_limit, int withhold) {
   using SL = DecSmem<D>;
   constexpr int S = SL::kStages;
   constexpr int KS = D / 16;   // k-steps of the QK^T product
@@ -114,11 +123,13 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   __shared__ int s_scan[8], s_tbmax[4];
   __shared__ int s_start[4];   // b, h, tile of the first tile of this CTA's range
   __shared__ volatile int s_abort;
+  __shared__ volatile int s_issued, s_stop;   // tiles the producer has handed over; first tile that never will be
   __shared__ int s_last, s_finisher;
   __shared__ int s_seq[kSeqCache];   // the lengths as they were when the kernel started
 
   // dynamic shared memory is only guaranteed 16-byte aligned: round up to the swizzle atom
-  uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  // (the offset is added to the array itself, so that the compiler still knows every derived pointer as shared memory)
+  uint8_t *smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
   const uint32_t smem_base = smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int cta = blockIdx.x, grid = gridDim.x;
@@ -127,6 +138,8 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   if (tid == 0) {
     for (int i = 0; i < S; ++i) { mbar_init(smem_u32(&full_bar[i]), 1); mbar_init(smem_u32(&empty_bar[i]), kDecConsumers); }
     s_abort = 0;
+    s_issued = 0;
+    s_stop = 0x7fffffff;
     s_start[0] = p.B;
     mbar_fence_init();
     fence_proxy_async_smem();
@@ -224,7 +237,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
   // Issues the copies of tile `pit` of the range (thread 0 only); false if the stage never came free.
   auto issue_tile = [&]() -> bool {
     const int it = pit, stage = it % S;
-    if (!mbar_wait(smem_u32(&empty_bar[stage]), ((it / S) & 1) ^ 1)) return false;
+    if (!mbar_wait_n(smem_u32(&empty_bar[stage]), ((it / S) & 1) ^ 1, spin_limit)) return false;
     const long long cur = g0 + it;
     const int u = pb * p.H_kv + ph;
     const long long us = cur - ptile, ue = us + ptb;
@@ -263,6 +276,12 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     *reinterpret_cast<TileDesc *>(st + SL::kDesc) = d;
     const uint32_t bar = smem_u32(&full_bar[stage]);
     const uint32_t dst = smem_base + stage * SL::kStride;
+    if (it == withhold) {   // test hook: the tile is announced, its copies are never issued
+      ++pit;
+      __threadfence_block();
+      s_issued = pit;
+      return true;
+    }
     mbar_expect_tx(bar, SL::kTxBytes);
 #pragma unroll
     for (int sub = 0; sub < SL::kSub; ++sub) {
@@ -272,11 +291,13 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     bulk_load_1d(dst + SL::kVotes, c.votes + ubase + (size_t)this_tile * kTile, kTile * 4, bar);
     bulk_load_1d(dst + SL::kLscore, c.lscore + ubase + (size_t)this_tile * kTile, kTile * 4, bar);
     ++pit;
+    __threadfence_block();
+    s_issued = pit;   // the descriptor of every tile below pit is in place
     return true;
   };
   if (tid == 0)
     while (pit < ntiles && pit < S - 1)
-      if (!issue_tile()) { s_abort = 1; break; }
+      if (!issue_tile()) { s_stop = pit; s_abort = 1; break; }
 
   {
     // ------------------------------------------------------------ the arithmetic
@@ -322,19 +343,31 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
     float m_run = -CUDART_INF_F, l_run = 0.f;   // running max (base-2 exponent) and per-thread partial sum of head g
+    bool dead = false;                          // a bounded wait ran out: no more waiting, no more arithmetic
 
     for (int it = 0; it < ntiles; ++it) {
       const int stage = it % S;
       // keep the ring S-1 tiles ahead: the stage of tile it-1 is free once all four warps have left it
-      if (tid == 0 && pit < ntiles && pit <= it + S - 1 && !s_abort)
-        if (!issue_tile()) s_abort = 1;
+      if (tid == 0 && pit < ntiles && pit <= it + S - 1 && s_stop > pit)
+        if (!issue_tile()) { s_stop = pit; s_abort = 1; }
       __syncwarp();
-      {
-        // A tile that never arrives stops all four warps at this same iteration (none can be past it,
-        // none is held at a combine barrier that needs this warp), so leaving the loop here is safe.
+      if (!dead) {
         int ok = 0;
-        if (lane == 0) ok = !s_abort && mbar_wait(smem_u32(&full_bar[stage]), (it / S) & 1);
-        if (!__shfl_sync(0xffffffffu, ok, 0)) { s_abort = 1; break; }
+        if (lane == 0) ok = !s_abort && mbar_wait_n(smem_u32(&full_bar[stage]), (it / S) & 1, spin_limit);
+        if (!__shfl_sync(0xffffffffu, ok, 0)) { s_abort = 1; dead = true; }
+      }
+      if (dead) {
+        // A wait ran out (here or in another warp): the kernel's result is lost, but its barriers are not.  The warp
+        // walks the rest of its range without waiting for data and without arithmetic, so that it still meets the
+        // others at every barrier of the combines; it only makes sure that the descriptor it acts on exists, and
+        // all four warps stop at the same tile if the producer gave up.
+        int go = 1;
+        if (lane == 0) {
+          int polls = 0;
+          while (s_issued <= it && s_stop > it && polls < spin_limit) { ++polls; __nanosleep(64); }
+          go = s_issued > it;
+        }
+        if (!__shfl_sync(0xffffffffu, go, 0)) break;
       }
       const uint32_t st = smem_base + stage * SL::kStride;
       const uint8_t *stp = smem + stage * SL::kStride;
@@ -343,7 +376,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
 
       const int i_base = d.tile * kTile + r0;     // first entry of this warp's slice
       const int n_valid = d.len - i_base;         // entries of the slice that exist (may be <= 0 or >= 32)
-      const bool mine = (it & 1) == pair;
+      const bool mine = (it & 1) == pair && !dead;
       const bool patch = mine && d.fresh >= r0 && d.fresh < r0 + 32;
       if (patch) {
         // Eq. 2 inside this call: the row of the fresh entry arrived with whatever the cache held; this warp,
@@ -720,13 +753,41 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     // give copies still in flight a bounded chance to land before the CTA's shared memory goes away
     if (tid == 0) {
       atomicOr(status_dev, KEEPKV_DEV_TIMEOUT);
-      for (int i = 0; i < S; ++i) { mbar_wait(smem_u32(&full_bar[i]), 0); mbar_wait(smem_u32(&full_bar[i]), 1); }
+      for (int i = 0; i < S; ++i) { mbar_wait_n(smem_u32(&full_bar[i]), 0, spin_limit); mbar_wait_n(smem_u32(&full_bar[i]), 1, spin_limit); }
     }
     __syncthreads();
   }
 }
 
 // ---------------------------------------------------------------- host side
+// What a test may change: the number of polls of a bounded wait, and one position of every CTA's tile range
+// that the producer announces without issuing its copies, so that the consumers' wait for it runs out with
+// nothing in flight (keepkv_debug_decode in the header).
+static int g_dbg_spin = kSpinLimit;
+static int g_dbg_withhold = -1;
+void decode_debug(int spin_limit, int withhold) {
+  g_dbg_spin = spin_limit > 0 ? spin_limit : kSpinLimit;
+  g_dbg_withhold = withhold;
+}
+
+// Tensor maps are a function of (base pointer, rows, D): a serving loop calls with the same few caches over and
+// over, so the encoded maps are kept in a small table instead of being rebuilt by the driver on every launch.
+struct MapKey { const void *base; uint64_t rows; int D; };
+static bool cached_rows_map(CUtensorMap *out, void *base, uint64_t rows, int D) {
+  constexpr int N = 64;
+  static MapKey keys[N];
+  static CUtensorMap maps[N];
+  static int used = 0, next = 0;
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  for (int i = 0; i < used; ++i)
+    if (keys[i].base == base && keys[i].rows == rows && keys[i].D == D) { *out = maps[i]; return true; }
+  if (!make_bf16_rows_map(out, base, rows, D, kTile)) return false;
+  const int slot = used < N ? used++ : (next++ % N);
+  keys[slot] = MapKey{base, rows, D};
+  maps[slot] = *out;
+  return true;
+}
 template <int D, int G>
 static void launch_t(const keepkv_params &p, const keepkv_cache &c, const void *q, void *out, float *lse,
                      int update_scores, char *ws, const WsLayout &L, int32_t *status_dev, const void *k_new,
@@ -743,7 +804,7 @@ static void launch_t(const keepkv_params &p, const keepkv_cache &c, const void *
   }
   CUtensorMap mapK, mapV;
   const uint64_t rows = (uint64_t)p.B * p.H_kv * p.N_cap;
-  if (!make_bf16_rows_map(&mapK, c.K, rows, D, kTile) || !make_bf16_rows_map(&mapV, c.V, rows, D, kTile)) {
+  if (!cached_rows_map(&mapK, c.K, rows, D) || !cached_rows_map(&mapV, c.V, rows, D)) {
     if (ctx.err == cudaSuccess) ctx.err = cudaErrorInvalidValue;
     return;
   }
@@ -786,7 +847,7 @@ static void launch_t(const keepkv_params &p, const keepkv_cache &c, const void *
     launch_pdl_cluster(decode_kernel<D, G>, dim3((unsigned)(U * cs)), dim3(kDecThreads), smem_bytes, ctx.stream, cs,
         mapK, mapV, p, c, reinterpret_cast<const __nv_bfloat16 *>(q), reinterpret_cast<__nv_bfloat16 *>(out), lse,
         update_scores, reinterpret_cast<int *>(ws + L.counters), reinterpret_cast<PartRec<D, G> *>(ws + L.part_pool),
-        status_dev, reinterpret_cast<const uint4 *>(k_new), reinterpret_cast<const uint4 *>(v_new));
+        status_dev, reinterpret_cast<const uint4 *>(k_new), reinterpret_cast<const uint4 *>(v_new), g_dbg_spin, g_dbg_withhold);
     KEEPKV_CHECK_LAUNCH(ctx);
     return;
   }
@@ -794,7 +855,7 @@ static void launch_t(const keepkv_params &p, const keepkv_cache &c, const void *
   launch_pdl(decode_kernel<D, G>, dim3((unsigned)grid), dim3(kDecThreads), smem_bytes, ctx.stream,
       mapK, mapV, p, c, reinterpret_cast<const __nv_bfloat16 *>(q), reinterpret_cast<__nv_bfloat16 *>(out), lse,
       update_scores, reinterpret_cast<int *>(ws + L.counters), reinterpret_cast<PartRec<D, G> *>(ws + L.part_pool),
-      status_dev, reinterpret_cast<const uint4 *>(k_new), reinterpret_cast<const uint4 *>(v_new));
+      status_dev, reinterpret_cast<const uint4 *>(k_new), reinterpret_cast<const uint4 *>(v_new), g_dbg_spin, g_dbg_withhold);
   KEEPKV_CHECK_LAUNCH(ctx);
 }
 
@@ -811,3 +872,8 @@ void launch_decode(const keepkv_params &p, const keepkv_cache &c, const void *q,
 }
 
 }  // namespace keepkv
+
+extern "C" int keepkv_debug_decode(int spin_limit, int withhold_tile) {
+  keepkv::decode_debug(spin_limit, withhold_tile);
+  return KEEPKV_OK;
+}

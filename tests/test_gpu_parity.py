@@ -619,3 +619,41 @@ def test_compress_with_caller_supplied_selection_scores(flags):
     # and the scores did change the outcome: the default selection keeps a different set
     dst0, ret0, _, _ = _run_compress(p, src, budget)
     assert not np.array_equal(ret0[0, :budget], ret[0, :budget])
+
+
+@pytest.mark.parametrize("B,H_kv,n,withhold,expect_timeout", [
+    (1, 1, 300, 0, True),      # one unit of five tiles on five CTAs, one tile each: every CTA loses its only tile
+    (1, 1, 300, 2, False),     # no CTA has a third tile: nothing is withheld, the call is a normal one
+    (2, 4, 2560, 1, True),     # 320 tiles on 160 CTAs: the first tile of a range is processed, the second never comes
+])
+def test_decode_bounded_wait_runs_out_and_the_next_call_is_normal(B, H_kv, n, withhold, expect_timeout):
+    """Failure detection without a fault: through the library's test hook the producer of every CTA announces
+    one tile of its range but never issues its copies (nothing is in flight, nothing lands later), with the
+    poll limit of the bounded waits cut to a few thousand.  The call must return, raise KEEPKV_DEV_TIMEOUT in
+    the status word and leave the context usable: the next, normal call gives the oracle's result."""
+    G, d = 4, 128
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=-(-n // 64) * 64, ema_alpha=0.9)
+    cache = random_cache(p, [n] * B, seed=8, vote_max=3, scored_frac=0.5)
+    snap = cache.lscore.clone()
+    q = _q(p, 3)
+    ws, st = kb.new_workspace(p), kb.new_status()
+    out = torch.empty_like(q)
+    lse = torch.empty(B, p.H_q, dtype=torch.float32, device="cuda")
+    try:
+        kb.keepkv_debug_decode(spin_limit=4096, withhold_tile=withhold)
+        kb.keepkv_decode_attention(p, cache, q, out, lse, False, ws, st)
+        torch.cuda.synchronize()                 # returns: no wait inside the kernel is unbounded
+    finally:
+        kb.keepkv_debug_decode(0, -1)
+    assert int(st.item()) == (kb.DEV_TIMEOUT if expect_timeout else 0)
+    assert torch.equal(cache.lscore.view(torch.int32), snap.view(torch.int32))
+    # a following normal call (the arrival counters of a lost call are in an unknown state: a fresh workspace)
+    st.zero_()
+    ws = kb.new_workspace(p)
+    hc = HostCache(cache)
+    kb.keepkv_decode_attention(p, cache, q, out, lse, True, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    ls_after = to_f64(cache.lscore).reshape(B * H_kv, -1)
+    for u in range(B * H_kv):
+        check_decode_unit(p, u, hc, to_f64(q), to_f64(out), to_f64(lse), ls_after, what="after a timeout")
