@@ -98,7 +98,8 @@ def lib() -> C.CDLL:
         _lib.okv_round_bf16.argtypes = [C.c_double]
         _lib.okv_cosine.restype = C.c_float
         _lib.okv_merge_group.restype = C.c_double
-        for n in ("okv_select", "okv_select_sorted", "okv_compress", "okv_compress_keyed", "okv_append", "okv_num_threads"):
+        for n in ("okv_select", "okv_select_sorted", "okv_compress", "okv_compress_keyed", "okv_merge_similar", "okv_append",
+                  "okv_num_threads"):
             getattr(_lib, n).restype = C.c_int32
     return _lib
 
@@ -232,6 +233,27 @@ def compress(P: Params, budget: int, K, V, votes, lscore, sorted_select: bool = 
         n_ret = lib().okv_compress_keyed(C.byref(cp), C.c_int32(n), C.c_int32(budget), _p(K), _p(V), _p(votes),
                                          _p(lscore), _p(key, C.c_float), _p(dK), _p(dV), _p(dv), _p(dl), _pi(ret),
                                          _pi(target), _p(gam), C.byref(st), C.c_int32(int(sorted_select)))
+    return dict(K=dK[:n_ret], V=dV[:n_ret], votes=dv[:n_ret], lscore=dl[:n_ret], ret_idx=ret[:n_ret].copy(),
+                target=target[:n].copy(), gammas=gam[:n_ret],
+                stats={f: getattr(st, f) for f, _ in _Stats._fields_ if f != "pad_"})
+
+
+def merge_similar(P: Params, K, V, votes, lscore):
+    """Prefill merge-first policy (Section 3.4; App. B, Table 3) for one unit: entries whose most similar other
+    key exceeds T are merged into that (earlier) entry; nothing else is evicted.  Returns the same dict as
+    compress(): the merged cache (n_ret rows), ret_idx, target [len] (slot for a member, -1 guard, -2 kept),
+    gammas, stats."""
+    K, V, votes, lscore = _f64(K), _f64(V), _f64(votes), _f64(lscore)
+    n, d = K.shape[0], P.d
+    m = max(n, 1)
+    dK = np.zeros((m, d)); dV = np.zeros((m, d)); dv = np.zeros(m); dl = np.zeros(m)
+    ret = np.empty(m, dtype=np.int32)
+    target = np.empty(m, dtype=np.int32)
+    gam = np.empty(m, dtype=np.float64)
+    st = _Stats()
+    cp = P.c()
+    n_ret = lib().okv_merge_similar(C.byref(cp), C.c_int32(n), _p(K), _p(V), _p(votes), _p(lscore), _p(dK), _p(dV),
+                                    _p(dv), _p(dl), _pi(ret), _pi(target), _p(gam), C.byref(st))
     return dict(K=dK[:n_ret], V=dV[:n_ret], votes=dv[:n_ret], lscore=dl[:n_ret], ret_idx=ret[:n_ret].copy(),
                 target=target[:n].copy(), gammas=gam[:n_ret],
                 stats={f: getattr(st, f) for f, _ in _Stats._fields_ if f != "pad_"})

@@ -25,7 +25,8 @@
  * Parity unpinned (the paper prints nothing that fixes them; they are readings
  * fixed by this oracle): the GQA score reduction (mean over the group),
  * first-observation initialisation of the EMA, the sink/recent/heavy split of the
- * selection, the gamma guard, and the ascending order of the compacted cache.
+ * selection, the gamma guard, the ascending order of the compacted cache, and the pairing
+ * rule of the prefill merge-first policy (earlier entry is the target, a target is never a member).
  */
 #include <math.h>
 #include <stdint.h>
@@ -130,8 +131,11 @@ void okv_decode(const okv_params *P, int32_t len, const double *q, const double 
  * raw exponential scores, kept as a logarithm:  sigma_i = ln((1/G) sum_g exp l_{g,i}).
  * Recursive case of Eq. 8 in the log domain:
  *   lscore_i <- ln( alpha * exp(lscore_i) + (1-alpha) * exp(sigma_i) ),
- * an entry that has never been scored (lscore = -inf) takes sigma_i itself (this is
- * the bias correction of Eq. 8 applied per entry at its first observation);
+ * an entry that has never been scored (lscore = -inf) takes sigma_i itself: the first
+ * observed score initialises the state.  That equals Eq. 8's bias-corrected estimate
+ * S / (1 - alpha^n), counted from the entry's first observation, at n = 1 only; from the
+ * second observation on this is the plain recursion (0.9 s_1 + 0.1 s_2 at alpha = 0.9),
+ * not the corrected form ((0.9 s_1 + s_2) / 1.9).  A reading, not the printed formula;
  * alpha = 0 gives lscore_i = sigma_i. */
 void okv_score_update(const okv_params *P, int32_t len, const double *q, const double *K, double *lscore) {
   const int G = P->G;
@@ -460,6 +464,107 @@ int32_t okv_compress_keyed(const okv_params *P, int32_t len, int32_t budget, con
   if (target_out) memcpy(target_out, target, sizeof(int32_t) * (size_t)len);
   if (stats) *stats = st;
   free(kappa); free(target); free(umax); free(members); free(kr); free(vr);
+  return n_ret;
+}
+
+/* --------------------------- Section 3.4 / App. B.3: prefill "merge first, then evict" */
+
+/* The prefill merge policy of Section 3.4 (App. B, Table 3): before any eviction, entries whose keys are similar
+ * enough are merged with each other; the eviction strategy is applied afterwards (okv_compress with
+ * merge_threshold = +inf evicts without merging).  The paper states the idea only; this is the reading:
+ *   1. every entry e looks for its most similar OTHER entry, c(e) = argmax_{i != e} cos(k_e, k_i) (the fixed fp32
+ *      cosine of okv_cosine, equal values -> lowest i), U_e the maximum;
+ *   2. e wants to merge iff U_e > T and c(e) < e: of two entries the earlier one is the target, so a mutual pair
+ *      merges the later into the earlier;
+ *   3. no entry is both target and member: if c(e) itself wants to merge (into a still earlier entry), e stays as it
+ *      is.  The members of a target c form its group K'_e (with c) and are merged by Eq. (A.3) with the score
+ *      estimates, exactly as in okv_compress, including the guard on the rescale factor: a group the guard rejects
+ *      loses its members, the target stays as it was (the outcome of the guard everywhere in this oracle);
+ *   4. the result holds every entry that is not a member, in ascending original order; nothing else is evicted.
+ * Outputs as okv_compress: dst arrays (n_ret rows), ret_idx [n_ret], target [len] (slot of the target for a
+ * member, -1 for a member whose group the guard rejected, -2 for an entry that is kept), gammas [n_ret], stats
+ * (n_evicted counts the members, n_below_T stays 0).  Returns n_ret. */
+int32_t okv_merge_similar(const okv_params *P, int32_t len, const double *K, const double *V, const double *votes,
+                          const double *lscore, double *dK, double *dV, double *dvotes, double *dlscore,
+                          int32_t *ret_idx, int32_t *target_out, double *gammas, okv_stats *stats) {
+  const int d = P->d;
+  const int L1 = len > 0 ? len : 1;
+  const float T = (float)P->merge_threshold;
+  float *nrm = (float *)malloc(sizeof(float) * (size_t)L1);
+  int32_t *partner = (int32_t *)malloc(sizeof(int32_t) * (size_t)L1);
+  unsigned char *wants = (unsigned char *)calloc((size_t)L1, 1), *member = (unsigned char *)calloc((size_t)L1, 1);
+  int32_t *slot_of = (int32_t *)malloc(sizeof(int32_t) * (size_t)L1);
+  int32_t *target = (int32_t *)malloc(sizeof(int32_t) * (size_t)L1);
+  for (int i = 0; i < len; ++i) nrm[i] = sqrtf(dot_chain(K + (size_t)i * d, K + (size_t)i * d, d));
+  /* 1, 2: the most similar other entry */
+  for (int e = 0; e < len; ++e) {
+    float best = -INFINITY;
+    int bi = -1;
+    for (int i = 0; i < len; ++i) {
+      if (i == e) continue;
+      float u = dot_chain(K + (size_t)e * d, K + (size_t)i * d, d) / (nrm[e] * nrm[i]);
+      if (u > best) { best = u; bi = i; }
+    }
+    partner[e] = bi;
+    wants[e] = (bi >= 0 && best > T && bi < e) ? 1 : 0;
+  }
+  /* 3: a target must stay */
+  for (int e = 0; e < len; ++e) member[e] = (wants[e] && !wants[partner[e]]) ? 1 : 0;
+  /* 4: kept entries, ascending */
+  int n_ret = 0;
+  for (int i = 0; i < len; ++i) {
+    slot_of[i] = -1;
+    if (!member[i]) { slot_of[i] = n_ret; ret_idx[n_ret++] = i; }
+  }
+  for (int e = 0; e < len; ++e) target[e] = member[e] ? slot_of[partner[e]] : -2;
+
+  okv_stats st;
+  memset(&st, 0, sizeof st);
+  st.n_retained = n_ret;
+  st.n_evicted = len - n_ret;
+  int32_t *members = (int32_t *)malloc(sizeof(int32_t) * (size_t)(L1 + 1));
+  double *kr = (double *)malloc(sizeof(double) * (size_t)d);
+  double *vr = (double *)malloc(sizeof(double) * (size_t)d);
+  for (int c = 0; c < n_ret; ++c) {
+    int ci = ret_idx[c];
+    int n = 0;
+    for (int e = 0; e < len; ++e)
+      if (e == ci || target[e] == c) members[n++] = e;
+    if (gammas) gammas[c] = NAN;
+    int merged = 0;
+    if (n > 1) {
+      st.n_groups++;
+      double pr, lr, lbar;
+      double gamma = okv_merge_group(d, n, members, K, V, votes, lscore, kr, vr, &pr, &lr, &lbar);
+      if (gammas) gammas[c] = gamma;
+      if (gamma > P->gamma_min && gamma <= P->gamma_max && fabs(lbar) >= 1e-6) {
+        for (int j = 0; j < d; ++j) {
+          dK[(size_t)c * d + j] = store_kv(P, kr[j]);
+          dV[(size_t)c * d + j] = store_kv(P, vr[j]);
+        }
+        dvotes[c] = store_f32(P, pr);
+        dlscore[c] = store_f32(P, lr);
+        merged = 1;
+        st.n_merged += n - 1;
+        if (n - 1 > st.max_group) st.max_group = n - 1;
+      } else {
+        st.n_guard_groups++;
+        for (int t = 0; t < n; ++t)
+          if (members[t] != ci) target[members[t]] = -1;
+      }
+    }
+    if (!merged) {
+      for (int j = 0; j < d; ++j) {
+        dK[(size_t)c * d + j] = K[(size_t)ci * d + j];
+        dV[(size_t)c * d + j] = V[(size_t)ci * d + j];
+      }
+      dvotes[c] = votes[ci];
+      dlscore[c] = lscore[ci];
+    }
+  }
+  if (target_out) memcpy(target_out, target, sizeof(int32_t) * (size_t)len);
+  if (stats) *stats = st;
+  free(nrm); free(partner); free(wants); free(member); free(slot_of); free(target); free(members); free(kr); free(vr);
   return n_ret;
 }
 

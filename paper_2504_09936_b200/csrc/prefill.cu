@@ -241,11 +241,17 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
     const float scale2 = p.sm_scale * kPfLog2e;
     const float ln_G = logf((float)G);
     float2 *xchg = reinterpret_cast<float2 *>(smem + SL::kXchg);
+    // A wait that runs out (here or in another warp) ends the warp's work but not its walk: it goes through the
+    // rest of the tiles without waiting and without reading the accumulators, so that the warps of its quarter
+    // still meet at their barrier on every tile.
+    bool dead = false;
     for (int it = 0; it < ntiles; ++it) {
       const int a = it & 1;
-      int ok = 0;
-      if (lane == 0) ok = !s_abort && mbar_wait(bar_t_full + 8 * a, (it >> 1) & 1);
-      if (!__shfl_sync(0xffffffffu, ok, 0)) { s_abort = 1; break; }
+      if (!dead) {
+        int ok = 0;
+        if (lane == 0) ok = !s_abort && mbar_wait(bar_t_full + 8 * a, (it >> 1) & 1);
+        if (!__shfl_sync(0xffffffffu, ok, 0)) { s_abort = 1; dead = true; }
+      }
       tc_fence_after();
       const int row = quarter * 32 + lane;
       const int i = wk.tile * kPfM + row;                         // this thread's entry
@@ -253,13 +259,13 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
       const bool full = wk.tile * kPfM + kPfM - 1 - wk.len + W <= 0;   // the whole tile is seen by every query
       const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + a * NB;
       float m = -CUDART_INF_F, S = 0.f;
-      if (g_last < 0) {   // no head for this warp: the accumulator is not its business
+      if (g_last < 0 || dead) {   // no head for this warp (or no data any more): the accumulator is not its business
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_t_empty + 8 * a);
       }
 #pragma unroll 1
-      for (int g = hq; g < G; g += 4) {
+      for (int g = dead ? G : hq; g < G; g += 4) {
         uint32_t r[32];
         tmem_ld_32x32(taddr + g * 32, r);
         tmem_ld_wait();
@@ -316,7 +322,7 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
           }
         }
       }
-      if (hq == 0 && i < wk.len)
+      if (hq == 0 && i < wk.len && !dead)
         c.lscore[((size_t)(wk.b * p.H_kv + wk.h)) * p.N_cap + i] = (m + log2f(S)) * kPfLn2 - lnwsuf[klo] - ln_G;
       wk.next(p, c.seq_len, it + 1 < ntiles);
     }

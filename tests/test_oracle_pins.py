@@ -573,3 +573,158 @@ def test_windowed_init_respects_causality_and_constant_scores():
     # a prompt shorter than the window: the queries before position 0 do not exist
     short = O.prefill_scores(P, qw, K[:3])
     assert np.allclose(short, O.prefill_scores(P, qw[-3:], K[:3]), atol=1e-12)
+
+
+# ------------------------------------------------ Section 3.4 / App. B Table 3: prefill merge-first policy
+
+def _clustered_keys(rng, n, d, n_clusters, spread):
+    """Keys that come in clusters of near-duplicates (cosine well above any threshold inside a cluster, near zero
+    between clusters), in random order: the structure the merge-first policy exists for."""
+    centers = rng.standard_normal((n_clusters, d)) * 3.0
+    which = rng.integers(0, n_clusters, n)
+    return centers[which] + spread * rng.standard_normal((n, d)), which
+
+
+def _brute_force_merge_first(K, T):
+    """The pairing rule written out with numpy in fp64: partner = most similar other entry (lowest index on
+    exactly equal cosines), an entry wants to merge iff its best cosine exceeds T and the partner is earlier, and
+    it is merged only if that partner does not itself want to merge."""
+    n = K.shape[0]
+    Kn = K / np.linalg.norm(K, axis=1, keepdims=True)
+    U = Kn @ Kn.T
+    np.fill_diagonal(U, -np.inf)
+    partner = np.argmax(U, axis=1)
+    best = U[np.arange(n), partner]
+    wants = (best > T) & (partner < np.arange(n))
+    member = wants & ~wants[partner]
+    return partner, best, member
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_merge_first_pairing_rule_against_brute_force(seed):
+    """Which entries are merged into which: the oracle's fixed-fp32-cosine decisions against an fp64 numpy
+    restatement of the rule, on inputs whose margins are far from both the ties and the threshold."""
+    rng = RNG(700 + seed)
+    n, d = int(rng.integers(20, 90)), int(rng.choice([8, 16, 64]))
+    K, _ = _clustered_keys(rng, n, d, n_clusters=int(rng.integers(3, 9)), spread=0.6)
+    V = rng.standard_normal((n, d))
+    votes = rng.integers(1, 4, n).astype(float); ls = rng.standard_normal(n) + 1.5
+    T = 0.9
+    partner, best, member = _brute_force_merge_first(K, T)
+    srt = np.sort(np.where(np.eye(n, dtype=bool), -np.inf, (K / np.linalg.norm(K, axis=1, keepdims=True)) @ (K / np.linalg.norm(K, axis=1, keepdims=True)).T), axis=1)
+    if np.min(srt[:, -1] - srt[:, -2]) < 2e-6 or np.min(np.abs(best - T)) < 2e-6:
+        pytest.skip("a near tie: fp32 and fp64 may legitimately order it differently")
+    P = O.Params(G=1, d=d, merge_threshold=T, gamma_min=-np.inf, gamma_max=np.inf)
+    r = O.merge_similar(P, K, V, votes, ls)
+    kept = np.nonzero(~member)[0]
+    assert np.array_equal(r["ret_idx"], kept)
+    slot_of = -np.ones(n, dtype=int); slot_of[kept] = np.arange(len(kept))
+    want_target = np.where(member, slot_of[partner], -2)
+    assert np.array_equal(r["target"], want_target)
+    assert member.sum() > 0 and r["stats"]["n_merged"] == member.sum() and r["stats"]["n_evicted"] == member.sum()
+    # no entry is both a target and a member
+    assert not np.any(member[partner[member]])
+
+
+def test_merge_first_chain_and_mutual_pair():
+    """Hand-built cases of the rule.  Keys a, b, c at angles 0, 0.3, 0.65: b's best partner is a (cos .955 against
+    .939), c's best partner is b (.939 against .796).  b merges into a; c's partner is itself merged away, so c
+    stays.  A mutual pair merges the later entry into the earlier one."""
+    d = 4
+    def unit(theta):
+        return np.array([math.cos(theta), math.sin(theta), 0.0, 0.0])
+    far = np.array([0.0, 0.0, 1.0, 0.0]); far2 = np.array([0.0, 0.0, 0.0, 1.0])
+    K = np.stack([unit(0.0), unit(0.3), unit(0.65), far, far2 * 2.0, far2 * 0.5])
+    V = np.arange(6 * d, dtype=float).reshape(6, d)
+    P = O.Params(G=1, d=d, merge_threshold=0.9, gamma_min=-np.inf, gamma_max=np.inf)
+    r = O.merge_similar(P, K, V, np.ones(6), np.full(6, 1.0))
+    # entry 1 -> 0 (cos .955 > T, partner earlier).  entry 2's best partner is 1 (cos .939 > T), which is merged away: 2 stays.
+    # entries 4, 5 are parallel (cos 1): a mutual pair, 5 merges into 4.  entry 3 has no similar neighbour.
+    assert list(r["ret_idx"]) == [0, 2, 3, 4]
+    assert list(r["target"]) == [-2, 0, -2, -2, -2, 3]
+    assert list(r["votes"]) == [2.0, 1.0, 1.0, 2.0]
+    # equal scores: omega = 1/2 each, gamma = 1 (the merged score equals the members' common score)
+    assert np.allclose(r["K"][0], 0.5 * (K[0] + K[1])) and np.allclose(r["V"][3], 0.5 * (V[4] + V[5]))
+    assert np.array_equal(r["K"][1], K[2]) and np.array_equal(r["K"][2], K[3])
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_merge_first_is_lossless_for_the_current_query_and_conserves_votes(seed):
+    """Theorem 2 applies to every group the policy forms: with s_hat = s^t (alpha = 0, G = 1) the attention output
+    and its denominator are unchanged by the merge, whatever the vote counts; and since nothing is evicted, the
+    votes of the cache are conserved (p_r = sum of the members' votes)."""
+    rng = RNG(800 + seed)
+    n, d = 60, 16
+    K, _ = _clustered_keys(rng, n, d, n_clusters=5, spread=0.08)
+    q = rng.standard_normal((1, d)) * 0.3
+    V = rng.standard_normal((n, d))
+    votes = rng.integers(1, 5, n).astype(float)
+    P = O.Params(G=1, d=d, ema_alpha=0.0, merge_threshold=0.8, gamma_min=-np.inf, gamma_max=np.inf)
+    ls = O.score_update(P, q, K, np.full(n, -np.inf))       # lscore = this step's logits
+    o0, lse0 = O.decode(P, q, K, V, votes)
+    r = O.merge_similar(P, K, V, votes, ls)
+    assert r["stats"]["n_merged"] > 10
+    if np.nanmax(np.abs(r["gammas"])) > 1e6:
+        pytest.skip("group with lambda_bar ~ 0: the printed formula is singular there")
+    o1, lse1 = O.decode(P, q, r["K"], r["V"], r["votes"])
+    assert np.max(np.abs(o1 - o0)) < 1e-9 and abs(lse1[0] - lse0[0]) < 1e-9
+    assert r["votes"].sum() == votes.sum()
+
+
+def test_merge_first_degenerate_cases():
+    """T = +inf merges nothing (an ordered copy); exact duplicates collapse onto their first occurrence with the
+    key and value unchanged (Lemma 1) and the votes added; a single entry and an empty unit pass through."""
+    rng = RNG(9)
+    n, d = 10, 8
+    K = rng.standard_normal((n, d)); V = rng.standard_normal((n, d)); votes = np.arange(1, n + 1, dtype=float)
+    ls = rng.standard_normal(n)
+    r = O.merge_similar(O.Params(G=1, d=d, merge_threshold=np.inf), K, V, votes, ls)
+    assert np.array_equal(r["K"], K) and np.array_equal(r["votes"], votes) and list(r["target"]) == [-2] * n
+    K2 = np.vstack([K, K[3], K[3], K[7]]); V2 = np.vstack([V, V[3], V[3], V[7]])
+    ls2 = np.r_[ls, ls[3], ls[3], ls[7]]
+    r = O.merge_similar(O.Params(G=1, d=d, merge_threshold=0.99, gamma_min=-np.inf, gamma_max=np.inf), K2, V2,
+                        np.ones(n + 3), ls2)
+    assert list(r["ret_idx"]) == list(range(n)) and list(r["target"][n:]) == [3, 3, 7]
+    assert np.allclose(r["K"][3], K[3], atol=1e-12) and np.allclose(r["V"][7], V[7], atol=1e-12)
+    assert list(r["votes"]) == [1, 1, 1, 3, 1, 1, 1, 2, 1, 1]
+    one = O.merge_similar(O.Params(G=1, d=d), K[:1], V[:1], votes[:1], ls[:1])
+    assert one["stats"]["n_retained"] == 1 and np.array_equal(one["K"], K[:1])
+    none = O.merge_similar(O.Params(G=1, d=d), K[:0], V[:0], votes[:0], ls[:0])
+    assert none["stats"]["n_retained"] == 0
+
+
+def test_merge_first_then_evict_keeps_what_evict_first_loses():
+    """The point of the policy (App. B, Table 3): with the same budget, merging similar entries before the
+    eviction keeps the votes of near-duplicates that an eviction without merging discards.  Pure eviction is
+    okv_compress with T = +inf."""
+    rng = RNG(10)
+    n, d, budget = 80, 16, 20
+    K, which = _clustered_keys(rng, n, d, n_clusters=6, spread=0.05)
+    V = rng.standard_normal((n, d)); votes = np.ones(n); ls = rng.standard_normal(n) * 0.3 + 2.0
+    Pm = O.Params(G=1, d=d, n_sink=0, n_recent=0, merge_threshold=0.9)
+    Pe = O.Params(G=1, d=d, n_sink=0, n_recent=0, merge_threshold=np.inf)
+    first = O.merge_similar(Pm, K, V, votes, ls)
+    then = O.compress(Pe, budget, first["K"], first["V"], first["votes"], first["lscore"])
+    plain = O.compress(Pe, budget, K, V, votes, ls)
+    assert then["stats"]["n_merged"] == 0 and plain["stats"]["n_merged"] == 0
+    assert plain["votes"].sum() == budget                       # eviction alone keeps one vote per kept entry
+    assert then["votes"].sum() > 2 * budget                     # merge-first kept whole clusters
+
+
+def test_first_observation_initialisation_is_not_the_bias_corrected_mean_after_step_one():
+    """What the EMA reading is and is not (Eq. 8).  An entry's first observed score initialises its state, which
+    coincides with the bias-corrected estimate S_n / (1 - alpha^n) counted from the entry's first observation at
+    n = 1.  At n = 2 the two differ: the oracle holds alpha s_1 + (1 - alpha) s_2, the corrected form would be
+    (alpha s_1 + s_2) / (1 + alpha)."""
+    d, alpha = 4, 0.9
+    P = O.Params(G=1, d=d, ema_alpha=alpha)
+    K = np.array([[1.0, 0.0, 0.0, 0.0]])
+    q1 = np.array([[2.0, 0.0, 0.0, 0.0]]); q2 = np.array([[-1.0, 0.0, 0.0, 0.0]])
+    s1, s2 = math.exp(2.0 / math.sqrt(d)), math.exp(-1.0 / math.sqrt(d))
+    ls = O.score_update(P, q1, K, np.array([-np.inf]))
+    assert math.isclose(math.exp(ls[0]), s1, rel_tol=1e-12)                      # n = 1: both readings agree
+    ls = O.score_update(P, q2, K, ls)
+    plain = alpha * s1 + (1 - alpha) * s2
+    corrected = ((1 - alpha) * (alpha * s1 + s2)) / (1 - alpha ** 2)
+    assert math.isclose(math.exp(ls[0]), plain, rel_tol=1e-12)
+    assert abs(plain - corrected) / corrected > 0.05                             # ... and here they do not
