@@ -67,7 +67,7 @@ typedef struct keepkv_params {
   int32_t n_recent;         /* entries always kept at the back  (App. B.3: recent window)      */
   float sm_scale;           /* 1/sqrt(d) of Eq. 3                                              */
   float ema_alpha;          /* alpha of Eq. 8, in [0,1); 0 makes the estimate the last score   */
-  float merge_threshold;    /* T of Algorithm 1, arg-max and threshold step (paper: 0.8); -INFINITY merges always   */
+  float merge_threshold;    /* T of Algorithm 1 (paper: 0.8); -INFINITY merges always, +INFINITY never (evict only) */
   float gamma_min;          /* a group is merged only if gamma_min < gamma <= gamma_max, gamma */
   float gamma_max;          /* the key rescale factor of Eq. A.3; (-INF, +INF) = paper as is   */
   int32_t flags;            /* KEEPKV_FLAG_* bits, normally 0                                  */
@@ -185,6 +185,31 @@ int keepkv_compress_scored(const keepkv_params *p, const keepkv_cache *src, cons
                            const float *select_score_or_null, const int32_t *budget_dev, int32_t budget_scalar,
                            const int32_t *n_recent_dev, int32_t *retained_idx_or_null, int32_t *target_or_null,
                            keepkv_stats *stats_or_null, void *ws, size_t ws_bytes, int32_t *status_dev, void *stream);
+
+/* Prefill compression with the merge policy of Section 3.4 (App. B, Table 3): "merge first, then evict".  Before any
+ * eviction, entries of the prompt whose keys are similar enough are merged with each other; the eviction strategy
+ * (the selection of keepkv_compress, without any further merging) is applied to the result.
+ * `cache` holds the prompt on entry and the compressed cache on return; `scratch` is a second buffer of the same
+ * shape (a serving loop's ping-pong partner) whose contents are destroyed.  Per unit, with len = cache.seq_len[b]:
+ *   1. every entry e takes its most cosine-similar OTHER entry c(e) (the fixed fp32 cosine of keepkv_compress, equal
+ *      values -> lower index);
+ *   2. e is merged into c(e) iff that cosine exceeds merge_threshold, c(e) lies before e in the cache, and c(e) is
+ *      not itself merged into an earlier entry (the earlier of two entries is the target; no entry is both target
+ *      and member; the paper states the policy, not the pairing rule: this is the library's reading);
+ *   3. every target is rewritten by Eq. A.3 over its members (votes add up), with the gamma guard of
+ *      keepkv_compress: a group the guard rejects loses its members and the target stays as it was;
+ *   4. the entries that were not merged away, in source order, form the merged prompt; it is cut to the budget by
+ *      step 1 of keepkv_compress (sinks, recent window, largest kappa; kappa from the merged votes and scores),
+ *      the evicted entries are dropped.  Because the heads of a sequence share seq_len, the budget of a sequence is
+ *      capped by the length of its shortest merged head: cache.seq_len[b] = min(budget_b, min over heads).
+ * Optional outputs: retained_idx_or_null i32 [B, H_kv, N_cap] (source index, in the prompt, of each row of the
+ * result); stats_or_null [B * H_kv] (n_retained = new length, n_evicted = len - n_retained, n_merged / n_groups /
+ * n_guard_groups / max_group of the merge pass, n_below_T = 0).  The similarity search compares all pairs of a
+ * unit's entries: 2 len^2 d flop per unit, on the tensor cores. */
+int keepkv_compress_merge_first(const keepkv_params *p, const keepkv_cache *cache, const keepkv_cache *scratch,
+                                const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
+                                int32_t *retained_idx_or_null, keepkv_stats *stats_or_null, void *ws, size_t ws_bytes,
+                                int32_t *status_dev, void *stream);
 
 /* One decode step driven from HOST memory (the call a serving loop makes): copies q_host,
  * k_new_host, v_new_host (pinned or pageable host memory, shapes as above) into the device

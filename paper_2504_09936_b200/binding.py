@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkeepkv.so")
 
 EXPORTS = ("keepkv_workspace_bytes", "keepkv_workspace_init", "keepkv_append", "keepkv_decode_attention",
-           "keepkv_decode_step", "keepkv_compress", "keepkv_compress_scored", "keepkv_prefill_scores", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_debug_decode", "keepkv_status_string", "keepkv_last_cuda_error",
+           "keepkv_decode_step", "keepkv_compress", "keepkv_compress_scored", "keepkv_compress_merge_first", "keepkv_prefill_scores", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_debug_decode", "keepkv_status_string", "keepkv_last_cuda_error",
            "keepkv_last_launch_count")
 
 
@@ -68,6 +68,7 @@ def lib() -> C.CDLL:
         l.keepkv_prefill_scores.argtypes = [pp, pc, vp, i32, vp, vp]
         l.keepkv_compress.argtypes = [pp, pc, pc, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         l.keepkv_compress_scored.argtypes = [pp, pc, pc, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
+        l.keepkv_compress_merge_first.argtypes = [pp, pc, pc, vp, i32, vp, vp, vp, vp, sz, vp, vp]
         l.keepkv_decode_step_host.argtypes = [pp, pc] + [vp] * 8 + [C.c_int, vp, sz, vp, vp]
         l.keepkv_decode_step_host_layers.argtypes = [pp, pc, i32] + [vp] * 8 + [C.c_int, vp, sz, vp, vp]
         _lib = l
@@ -193,6 +194,17 @@ def keepkv_compress_scored(p, src: Cache, dst: Cache, select_score, budget, ws, 
                                         bsc, _ptr(n_recent_dev), _ptr(retained_idx), _ptr(target), _ptr(stats),
                                         ws.data_ptr(), ws.numel(), status.data_ptr(), _stream(stream)),
            "keepkv_compress_scored")
+
+
+def keepkv_compress_merge_first(p, cache: Cache, scratch: Cache, budget, ws, status, n_recent_dev=None,
+                                retained_idx=None, stats=None, stream=None):
+    """Prefill compression, merge-first policy (Section 3.4): similar entries of the prompt are merged with each
+    other, then the selection cuts the result to the budget.  In place on `cache`; `scratch` is destroyed."""
+    bdev, bsc = (budget.data_ptr(), 0) if isinstance(budget, torch.Tensor) else (None, int(budget))
+    _check(lib().keepkv_compress_merge_first(C.byref(p), C.byref(cache.c()), C.byref(scratch.c()), bdev, bsc,
+                                             _ptr(n_recent_dev), _ptr(retained_idx), _ptr(stats), ws.data_ptr(),
+                                             ws.numel(), status.data_ptr(), _stream(stream)),
+           "keepkv_compress_merge_first")
 
 
 def keepkv_decode_step_host(p, cache: Cache, q_host, k_new_host, v_new_host, out_host, q_dev, k_new_dev, v_new_dev,

@@ -38,6 +38,9 @@ WsLayout ws_layout(const keepkv_params &p) {
   L.grp_key = take(U * Np2 * 4);
   L.grp_head = take(U * N * 4);
   L.stats = take(U * sizeof(keepkv_stats));
+  L.stats2 = take(U * sizeof(keepkv_stats));
+  L.unit_len = take(U * 4);
+  L.eff_budget = take((size_t)p.B * 4);
   L.total = off;
   return L;
 }
@@ -207,6 +210,32 @@ int keepkv_compress_scored(const keepkv_params *p, const keepkv_cache *src, cons
                   target_or_null ? target_or_null : (int32_t *)(w + L.target),
                   stats_or_null ? stats_or_null : (keepkv_stats *)(w + L.stats), w, L, status_dev, ctx,
                   select_score_or_null);
+  return finish(ctx);
+}
+
+int keepkv_compress_merge_first(const keepkv_params *p, const keepkv_cache *cache, const keepkv_cache *scratch,
+                                const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
+                                int32_t *retained_idx_or_null, keepkv_stats *stats_or_null, void *ws, size_t ws_bytes,
+                                int32_t *status_dev, void *stream) {
+  int rc = validate(p);
+  if (rc) return rc;
+  if ((rc = validate_cache(cache))) return rc;
+  if ((rc = validate_cache(scratch))) return rc;
+  if (cache->K == scratch->K || cache->V == scratch->V || cache->votes == scratch->votes ||
+      cache->lscore == scratch->lscore || cache->seq_len == scratch->seq_len)
+    return KEEPKV_ERR_INVALID_ARG;
+  if (!ws || !status_dev || !aligned(ws, 256)) return KEEPKV_ERR_INVALID_ARG;
+  if ((long long)p->B * p->H_kv > kMaxUnits) return KEEPKV_ERR_UNSUPPORTED;
+  if (p->flags & KEEPKV_FLAG_COMPRESS_STEADY) return KEEPKV_ERR_INVALID_ARG;   // a prompt is not a steady-state cache
+  if (!budget_dev) {
+    if (budget_scalar < 0) return KEEPKV_ERR_INVALID_ARG;
+    if (budget_scalar > p->N_cap || (long long)budget_scalar + p->period > p->N_cap) return KEEPKV_ERR_CAPACITY;
+  }
+  WsLayout L = ws_layout(*p);
+  if (ws_bytes < L.total) return KEEPKV_ERR_WORKSPACE;
+  LaunchCtx ctx{(cudaStream_t)stream, 0, cudaSuccess};
+  launch_compress_merge_first(*p, *cache, *scratch, budget_dev, budget_scalar, n_recent_dev, retained_idx_or_null,
+                              stats_or_null, (char *)ws, L, status_dev, ctx);
   return finish(ctx);
 }
 

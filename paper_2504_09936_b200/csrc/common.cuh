@@ -35,6 +35,9 @@ struct WsLayout {
   size_t grp_key;     // u32 [U,Npow2]      (slot << 16 | evicted position) of merged entries, sorted
   size_t grp_head;    // i32 [U,N]          position in grp_key where each group starts
   size_t stats;       // keepkv_stats [U]   used when the caller passes no stats array
+  size_t stats2;      // keepkv_stats [U]   merge-first: statistics of the merge pass
+  size_t unit_len;    // i32 [U]            merge-first: entries of each unit after the merge pass
+  size_t eff_budget;  // i32 [B]            merge-first: budget of each sequence, capped by its shortest head
   size_t total;
   size_t decode_bytes;   // the leading part that keepkv_decode_attention uses (counters and partials)
   size_t counter_bytes;  // size of the counters array
@@ -67,7 +70,12 @@ void launch_compress(const keepkv_params &p, const keepkv_cache &src, const keep
 // tcgen05 similarity search: for every evicted key the two largest cosines over the retained keys
 void launch_nominate(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst, const int32_t *ev_idx,
                      const UnitInfo *unit_info, const float *inv_norm, int32_t *sched, float4 *nom_v, int32_t *nom_si,
-                     int nom_chunks, int32_t *status_dev, LaunchCtx &ctx);
+                     int nom_chunks, int32_t *status_dev, LaunchCtx &ctx, int self_mask = 0);
+// Section 3.4, prefill merge-first policy (compress.cu): cache -> scratch (merge) -> cache (eviction)
+void launch_compress_merge_first(const keepkv_params &p, const keepkv_cache &cache, const keepkv_cache &scratch,
+                                 const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
+                                 int32_t *ret_idx_out, keepkv_stats *stats_out, char *ws, const WsLayout &L,
+                                 int32_t *status_dev, LaunchCtx &ctx);
 void launch_prefill_scores(const keepkv_params &p, const keepkv_cache &c, const void *q_window, int W,
                            int32_t *status_dev, LaunchCtx &ctx);
 int sm_count();

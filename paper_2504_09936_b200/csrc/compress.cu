@@ -20,7 +20,7 @@ constexpr int kWarpSelectMax = 2048;   // candidate sets up to this size are sea
 __global__ void __launch_bounds__(1024)
 select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int32_t *budget_dev, int budget_scalar,
               const int32_t *n_recent_dev, int32_t *ret_idx, int32_t *target, int32_t *ev_idx, UnitInfo *unit_info,
-              keepkv_stats *stats, const float *__restrict__ select_key) {
+              keepkv_stats *stats, const float *__restrict__ select_key, const int32_t *__restrict__ unit_len) {
   extern __shared__ uint32_t keys[];
   __shared__ int hist[256];
   __shared__ int warp_tot[32];
@@ -29,7 +29,8 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
   const int u = blockIdx.x, b = u / p.H_kv, h = u % p.H_kv, tid = threadIdx.x;
   pdl_wait();
   pdl_trigger();
-  const int len = max(0, min(src.seq_len[b], p.N_cap));
+  // (unit_len: the heads of a sequence differ in length -- only between the two passes of the merge-first compression)
+  const int len = max(0, min(unit_len ? unit_len[u] : src.seq_len[b], p.N_cap));
   int budget = budget_dev ? budget_dev[b] : budget_scalar;
   budget = max(0, min(budget, p.N_cap));
   int n_sink = p.n_sink, n_recent = n_recent_dev ? max(0, n_recent_dev[b]) : p.n_recent;
@@ -262,12 +263,84 @@ constexpr int kMergeInline = 32;   // units with at most this many groups are me
 constexpr int kResolveThreads = 512;
 constexpr int kResolveWarps = kResolveThreads / 32;
 
+// Sorts the M entries to merge of unit u by (slot, position) -- which makes every group contiguous and ascending --,
+// publishes the sorted members and the start of every group, and merges the groups itself when there are few.
+// Called by a whole CTA of kResolveThreads threads.  keys: where the M keys are now (key_smem when `single`, else gk).
+template <int D>
+__device__ __forceinline__ void group_and_merge(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
+                                                int u, size_t base, int n_ev, int M, bool single, uint32_t *key_smem,
+                                                int smem_keys, uint32_t *gk, const int32_t *__restrict__ ret_idx,
+                                                const int32_t *__restrict__ ev_idx, int32_t *target, int32_t *grp_head,
+                                                UnitInfo *unit_info, keepkv_stats *stats, int *warp_tot) {
+  const int tid = threadIdx.x, warp = tid >> 5;
+  int Mp = 1;
+  while (Mp < M) Mp <<= 1;
+  uint32_t *keys = (single || Mp <= smem_keys) ? key_smem : gk;
+  if (keys != gk && !single)
+    for (int i = tid; i < M; i += kResolveThreads) keys[i] = __ldcg(&gk[i]);
+  for (int i = M + tid; i < Mp; i += kResolveThreads) keys[i] = 0xFFFFFFFFu;
+  __syncthreads();
+  if (Mp <= kResolveThreads && keys == key_smem) {
+    // few keys (all distinct): every thread finds the rank of its key by counting, one barrier
+    uint32_t mine = 0xFFFFFFFFu;
+    int rank = 0;
+    if (tid < M) {
+      mine = keys[tid];
+      for (int j = 0; j < M; ++j) rank += keys[j] < mine ? 1 : 0;
+    }
+    __syncthreads();
+    if (tid < M) keys[rank] = mine;
+    __syncthreads();
+  } else {
+    // bitonic sort, ascending
+    for (int k = 2; k <= Mp; k <<= 1) {
+      for (int jj = k >> 1; jj > 0; jj >>= 1) {
+        for (int i = tid; i < Mp; i += kResolveThreads) {
+          const int ixj = i ^ jj;
+          if (ixj > i) {
+            const uint32_t a = keys[i], b = keys[ixj];
+            if ((a > b) == ((i & k) == 0)) { keys[i] = b; keys[ixj] = a; }
+          }
+        }
+        __syncthreads();
+      }
+    }
+  }
+  // publish the sorted members and the start of every group
+  int n_groups = 0;
+  for (int i0 = 0; i0 < M; i0 += kResolveThreads) {
+    const int i = i0 + tid;
+    const bool head = i < M && (i == 0 || (keys[i] >> 16) != (keys[i - 1] >> 16));
+    int tot;
+    const int pos = n_groups + block_excl_count(head, warp_tot, tot);
+    if (head) grp_head[base + pos] = i;
+    if (i < M && keys != gk) gk[i] = keys[i];
+    n_groups += tot;
+  }
+  if (tid == 0) {
+    grp_head[base + n_groups] = M;
+    unit_info[u].n_groups = n_groups <= kMergeInline ? 0 : n_groups;
+    stats[u].n_below_T = n_ev - M;
+  }
+  if (n_groups <= kMergeInline) {
+    // few groups (every steady-state compression): merge them here, one warp per group
+    __syncthreads();   // the keys and group starts written above are visible to the whole CTA
+    for (int g = warp; g < n_groups; g += kResolveWarps) {
+      const int beg = grp_head[base + g], n = grp_head[base + g + 1] - beg;
+      const int c = (int)(gk[beg] >> 16);
+      merge_group<D>(p, src, dst, c, ret_idx[base + c], [&](int t) { return ev_idx[base + (gk[beg + t] & 0xFFFFu)]; }, n,
+                     target + base, base, stats + u);
+    }
+  }
+}
+
+
 template <int D>
 __global__ void __launch_bounds__(kResolveThreads)
 resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_t *__restrict__ ev_idx,
                UnitInfo *unit_info, const float4 *__restrict__ nom_v, const int32_t *__restrict__ nom_si,
                const int32_t *__restrict__ sched, int C_max, const int32_t *__restrict__ ret_idx, int32_t *target,
-               uint32_t *grp_key, int key_stride, int32_t *grp_head, keepkv_stats *stats, int smem_keys) {
+               uint32_t *grp_key, int key_stride, int32_t *grp_head, keepkv_stats *stats, int smem_keys, int decide_only) {
   extern __shared__ uint32_t key_smem[];
   __shared__ float ke_s[kResolveWarps][D];
   __shared__ float kc_s[kResolveWarps][2][D];
@@ -290,7 +363,7 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
   // (every steady-state compression) needs no exchange through global memory.
   const int n_cta = min((int)gridDim.x, (ui.n_ev + kResolveThreads - 1) / kResolveThreads);
   if ((int)blockIdx.x >= n_cta) return;
-  const bool single = ui.n_ev <= kResolveThreads;
+  const bool single = ui.n_ev <= kResolveThreads && !decide_only;
   if (tid == 0) { s_nq[0] = s_nq[1] = 0; s_base = 0; }
   __syncthreads();
 
@@ -343,6 +416,10 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
     }
     __syncthreads();
     if (kind) { slot = res_slot[tid]; merge = res_merge[tid] != 0; }
+    if (decide_only) {   // the caller pairs the entries itself (merge-first policy): the partner above T, or -1
+      if (valid) target[base + e] = merge ? slot : -1;
+      continue;
+    }
     // ---- record the decision; entries to merge go to the unit's key list (any order: it is sorted below)
     int tot;
     const int off = block_excl_count(merge, warp_tot, tot);
@@ -362,6 +439,7 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
       if (merge) gk[s_base + off] = ((uint32_t)slot << 16) | (uint32_t)j;
     }
   }
+  if (decide_only) return;
   int M;
   if (single) {
     M = s_base;
@@ -375,65 +453,8 @@ resolve_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_
     __threadfence();
     M = *reinterpret_cast<volatile int *>(&unit_info[u].n_keys);
   }
-  int Mp = 1;
-  while (Mp < M) Mp <<= 1;
-  uint32_t *keys = (single || Mp <= smem_keys) ? key_smem : gk;
-  if (keys != gk && !single)
-    for (int i = tid; i < M; i += kResolveThreads) keys[i] = __ldcg(&gk[i]);
-  for (int i = M + tid; i < Mp; i += kResolveThreads) keys[i] = 0xFFFFFFFFu;
-  __syncthreads();
-  if (Mp <= kResolveThreads && keys == key_smem) {
-    // few keys (all distinct): every thread finds the rank of its key by counting, one barrier
-    uint32_t mine = 0xFFFFFFFFu;
-    int rank = 0;
-    if (tid < M) {
-      mine = keys[tid];
-      for (int j = 0; j < M; ++j) rank += keys[j] < mine ? 1 : 0;
-    }
-    __syncthreads();
-    if (tid < M) keys[rank] = mine;
-    __syncthreads();
-  } else {
-    // bitonic sort, ascending
-    for (int k = 2; k <= Mp; k <<= 1) {
-      for (int jj = k >> 1; jj > 0; jj >>= 1) {
-        for (int i = tid; i < Mp; i += kResolveThreads) {
-          const int ixj = i ^ jj;
-          if (ixj > i) {
-            const uint32_t a = keys[i], b = keys[ixj];
-            if ((a > b) == ((i & k) == 0)) { keys[i] = b; keys[ixj] = a; }
-          }
-        }
-        __syncthreads();
-      }
-    }
-  }
-  // publish the sorted members and the start of every group
-  int n_groups = 0;
-  for (int i0 = 0; i0 < M; i0 += kResolveThreads) {
-    const int i = i0 + tid;
-    const bool head = i < M && (i == 0 || (keys[i] >> 16) != (keys[i - 1] >> 16));
-    int tot;
-    const int pos = n_groups + block_excl_count(head, warp_tot, tot);
-    if (head) grp_head[base + pos] = i;
-    if (i < M && keys != gk) gk[i] = keys[i];
-    n_groups += tot;
-  }
-  if (tid == 0) {
-    grp_head[base + n_groups] = M;
-    unit_info[u].n_groups = n_groups <= kMergeInline ? 0 : n_groups;
-    stats[u].n_below_T = ui.n_ev - M;
-  }
-  if (n_groups <= kMergeInline) {
-    // few groups (every steady-state compression): merge them here, one warp per group
-    __syncthreads();   // the keys and group starts written above are visible to the whole CTA
-    for (int g = warp; g < n_groups; g += kResolveWarps) {
-      const int beg = grp_head[base + g], n = grp_head[base + g + 1] - beg;
-      const int c = (int)(gk[beg] >> 16);
-      merge_group<D>(p, src, dst, c, ret_idx[base + c], [&](int t) { return ev_idx[base + (gk[beg + t] & 0xFFFFu)]; }, n,
-                     target + base, base, stats + u);
-    }
-  }
+  group_and_merge<D>(p, src, dst, u, base, ui.n_ev, M, single, key_smem, smem_keys, gk, ret_idx, ev_idx, target, grp_head,
+                     unit_info, stats, warp_tot);
 }
 
 // ------------------------------------------------------------------ merge
@@ -493,23 +514,282 @@ static void launch_compress_t(const keepkv_params &p, const keepkv_cache &src, c
     return;
   }
   launch_pdl(select_kernel, dim3(U), dim3(512), sel_smem, ctx.stream, p, src, dst.seq_len, budget_dev, budget_scalar,
-             n_recent_dev, ret_idx, target, ev_idx, ui, stats, select_key);
+             n_recent_dev, ret_idx, target, ev_idx, ui, stats, select_key, (const int32_t *)nullptr);
   KEEPKV_CHECK_LAUNCH(ctx);
   if (ret_bound <= 0) return;   // nothing is kept: every entry is dropped, which select has recorded
   const int cgx = (ret_bound + 63) / 64 < 32 ? (ret_bound + 63) / 64 : 32;   // the retained count is only known on the device
   launch_pdl(compact_kernel<D>, dim3(cgx, U), dim3(256), 0, ctx.stream, p, src, dst, ret_idx, ui,
              inv_norm);
   KEEPKV_CHECK_LAUNCH(ctx);
+  // T = +inf: no cosine can exceed it, nothing merges -- the eviction strategy alone (what follows a merge-first pass)
+  if (isinf(p.merge_threshold) && p.merge_threshold > 0.f) return;
   launch_nominate(p, src, dst, ev_idx, ui, inv_norm, sched, nom_v, nom_si, L.nom_chunks, status_dev, ctx);
   launch_pdl(resolve_kernel<D>, dim3(L.nom_chunks, U), dim3(kResolveThreads), (size_t)smem_keys * 4, ctx.stream,
       p, src, dst, ev_idx, ui, nom_v, nom_si, sched, L.nom_chunks, ret_idx, target, grp_key, L.key_stride, grp_head,
-      stats, smem_keys);
+      stats, smem_keys, 0);
   KEEPKV_CHECK_LAUNCH(ctx);
   int gx = 4096 / U;
   gx = gx < 1 ? 1 : (gx > 32 ? 32 : gx);
   launch_pdl(merge_kernel<D>, dim3(gx, U), dim3(256), 0, ctx.stream, p, src, dst, ret_idx, ev_idx, target, ui, grp_key,
              L.key_stride, grp_head, stats);
   KEEPKV_CHECK_LAUNCH(ctx);
+}
+
+
+// ------------------------------------------------------------------ prefill merge-first policy (Section 3.4; App. B, Table 3)
+// keepkv_merge_similar: before any eviction, every entry whose most similar OTHER key exceeds T is merged into that
+// entry, provided the partner is earlier in the cache and is not itself merged away (the earlier of two entries is
+// the target; no entry is both target and member).  The similarity search is the compression's own
+// (nominate_kernel + resolve_kernel) with rows and columns both running over all entries of the unit and the
+// diagonal masked; what is new is the pairing rule, which needs every entry's partner before any entry can be
+// placed:
+//   mf_prepare  -> inverse norms of all keys, the identity row list, the unit's sizes
+//   nominate    -> two best cosines per entry over all other entries
+//   resolve     -> partner above T per entry, exact where the ranking is close       (decide_only)
+//   mf_mark     -> members, kept entries and their slots, targets, the key list of the groups
+//   compact     -> kept rows to dst
+//   group       -> keys sorted into groups, few groups merged at once
+//   merge       -> Eq. A.3 for units with many groups
+template <int D>
+__global__ void __launch_bounds__(256)
+mf_prepare_kernel(keepkv_params p, keepkv_cache src, int32_t *ev_idx, UnitInfo *unit_info, float *__restrict__ inv_norm) {
+  constexpr int CH = D / 8;
+  pdl_wait();
+  pdl_trigger();
+  const int u = blockIdx.y, b = u / p.H_kv;
+  const int len = max(0, min(src.seq_len[b], p.N_cap));
+  const size_t base = (size_t)u * p.N_cap;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    UnitInfo ui{len, len, len, 0, 0, 0, 0, 0};
+    unit_info[u] = ui;
+  }
+  const uint4 *sK = reinterpret_cast<const uint4 *>(src.K);
+  const int lane = threadIdx.x & 31, ch = lane & 15, sub = lane >> 4, warp = threadIdx.x >> 5;
+  for (int r0 = blockIdx.x * 16; r0 < len; r0 += gridDim.x * 16) {   // sixteen lanes per row, two rows per warp
+    const int i = r0 + warp * 2 + sub;
+    uint4 kv = make_uint4(0, 0, 0, 0);
+    if (i < len && ch < CH) kv = sK[(base + i) * CH + ch];
+    float ss = 0.f;
+    const uint32_t w[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) { const float a = bf16_lo(w[q]), bb = bf16_hi(w[q]); ss = fmaf(a, a, ss); ss = fmaf(bb, bb, ss); }
+    ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+    ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+    ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+    ss += __shfl_xor_sync(0xffffffffu, ss, 8);
+    if (i < len && ch == 0) { inv_norm[base + i] = rsqrtf(ss); ev_idx[base + i] = i; }
+  }
+}
+
+// One CTA per unit.  partner[e] (in `target`): the entry e would merge into, or -1.  Writes the kept list (ret_idx),
+// the member list (ev_idx), target[e] = slot of the partner for a member / -2 for a kept entry, the group keys
+// (slot << 16 | position among the members), sizes and the initial statistics.  slot_of: scratch [N] per unit.
+__global__ void __launch_bounds__(1024)
+mf_mark_kernel(keepkv_params p, int32_t *unit_len, int32_t *ret_idx, int32_t *target, int32_t *ev_idx, int32_t *slot_of,
+               uint32_t *grp_key, int key_stride, UnitInfo *unit_info, keepkv_stats *stats) {
+  __shared__ int warp_tot[32];
+  pdl_wait();
+  pdl_trigger();
+  const int u = blockIdx.x, tid = threadIdx.x, nthr = blockDim.x, nw = nthr >> 5;
+  const int len = unit_info[u].len;
+  const size_t base = (size_t)u * p.N_cap;
+  int32_t *tg = target + base;
+  uint32_t *gk = grp_key + (size_t)u * key_stride;
+  auto wants = [&](int e) { const int t = tg[e]; return t >= 0 && t < e; };
+  // pass 1: kept entries and their slots (a thread owns a run of consecutive entries)
+  constexpr int RUN = 4;
+  int n_keep = 0;
+  for (int start = 0; start < len; start += nthr * RUN) {
+    const int i0 = start + tid * RUN;
+    bool mem[RUN];
+    int n_k = 0;
+#pragma unroll
+    for (int r = 0; r < RUN; ++r) {
+      const int e = i0 + r;
+      mem[r] = e < len && wants(e) && !wants(tg[e]);   // its partner stays: e is a member
+      n_k += (e < len && !mem[r]) ? 1 : 0;
+    }
+    int tot;
+    int slot = n_keep + block_excl_sum(n_k, warp_tot, tot, nw);
+#pragma unroll
+    for (int r = 0; r < RUN; ++r) {
+      const int e = i0 + r;
+      if (e < len) {
+        if (mem[r]) {
+          ev_idx[base + (e - slot)] = e;
+          slot_of[base + e] = -1 - (e - slot);   // a member: its position among the members
+        } else {
+          ret_idx[base + slot] = e;
+          slot_of[base + e] = slot;
+          ++slot;
+        }
+      }
+    }
+    n_keep += tot;
+  }
+  __syncthreads();   // (block scope: the global writes above are visible to the whole CTA)
+  // pass 2: members look up the slot of their partner (partners are read before any target is overwritten:
+  // a member's partner is a kept entry, and kept entries' targets are rewritten to -2 only after the barrier below)
+  for (int e = tid; e < len; e += nthr) {
+    const int so = slot_of[base + e];
+    if (so < 0) {
+      const int pos = -1 - so, slot = slot_of[base + tg[e]];
+      gk[pos] = ((uint32_t)slot << 16) | (uint32_t)pos;
+      slot_of[base + e] = -0x40000000 + slot;   // remembered for the rewrite below
+    }
+  }
+  __syncthreads();
+  for (int e = tid; e < len; e += nthr) {
+    const int so = slot_of[base + e];
+    tg[e] = so < 0 ? so + 0x40000000 : -2;
+  }
+  if (tid == 0) {
+    const int n_ev = len - n_keep;
+    UnitInfo ui{len, n_keep, n_ev, 0, n_ev, 0, 0, 0};   // n_keys: every member is an entry to merge
+    unit_info[u] = ui;
+    unit_len[u] = n_keep;
+    keepkv_stats st;
+    st.n_retained = n_keep; st.n_evicted = n_ev; st.n_merged = 0; st.n_below_T = 0;
+    st.n_guard_groups = 0; st.n_groups = 0; st.max_group = 0; st.reserved = 0;
+    stats[u] = st;
+  }
+}
+
+// One CTA per unit: the unit's key list (in global memory) sorted into groups; few groups are merged here.
+template <int D>
+__global__ void __launch_bounds__(kResolveThreads)
+group_kernel(keepkv_params p, keepkv_cache src, keepkv_cache dst, const int32_t *__restrict__ ret_idx,
+             const int32_t *__restrict__ ev_idx, int32_t *target, UnitInfo *unit_info, uint32_t *grp_key, int key_stride,
+             int32_t *grp_head, keepkv_stats *stats, int smem_keys) {
+  extern __shared__ uint32_t key_smem[];
+  __shared__ int warp_tot[32];
+  pdl_wait();
+  pdl_trigger();
+  const int u = blockIdx.x;
+  const UnitInfo ui = unit_info[u];
+  const size_t base = (size_t)u * p.N_cap;
+  group_and_merge<D>(p, src, dst, u, base, ui.n_ev, ui.n_keys, false, key_smem, smem_keys, grp_key + (size_t)u * key_stride,
+                     ret_idx, ev_idx, target, grp_head, unit_info, stats, warp_tot);
+}
+
+// Budget of each sequence for the eviction pass: the caller's, capped by the sequence's shortest merged head (the
+// heads of a sequence share one seq_len, so they must all end at the same length).
+__global__ void mf_budget_kernel(keepkv_params p, const int32_t *budget_dev, int budget_scalar, const int32_t *unit_len,
+                                 int32_t *eff_budget) {
+  pdl_wait();
+  pdl_trigger();
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= p.B) return;
+  int m = p.N_cap;
+  for (int h = 0; h < p.H_kv; ++h) m = min(m, unit_len[b * p.H_kv + h]);
+  const int budget = max(0, min(budget_dev ? budget_dev[b] : budget_scalar, p.N_cap));
+  eff_budget[b] = min(budget, m);
+}
+
+// What the caller sees of the two passes: the prompt index of every row of the result, and one record of statistics.
+__global__ void mf_compose_kernel(keepkv_params p, const int32_t *seq_len, const int32_t *__restrict__ ret1,
+                                  const int32_t *__restrict__ ret2, int32_t *ret_out, const keepkv_stats *st1,
+                                  const UnitInfo *unit_info, const int32_t *prompt_len, keepkv_stats *stats_out) {
+  pdl_wait();
+  pdl_trigger();
+  const int u = blockIdx.y, b = u / p.H_kv;
+  const size_t base = (size_t)u * p.N_cap;
+  const int n = seq_len[b];
+  if (ret_out)
+    for (int s = blockIdx.x * blockDim.x + threadIdx.x; s < n; s += gridDim.x * blockDim.x)
+      ret_out[base + s] = ret1[base + ret2[base + s]];
+  if (stats_out && blockIdx.x == 0 && threadIdx.x == 0) {
+    keepkv_stats st = st1[u];
+    st.n_evicted = st.n_retained + st.n_evicted - n;   // of the prompt's entries (kept + merged away in the merge pass)
+    st.n_retained = n;
+    st.n_below_T = 0;
+    stats_out[u] = st;
+  }
+}
+
+template <int D>
+static void launch_compress_merge_first_t(const keepkv_params &p, const keepkv_cache &cache, const keepkv_cache &scratch,
+                                          const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
+                                          int32_t *ret_idx_out, keepkv_stats *stats_out, char *ws, const WsLayout &L,
+                                          int32_t *status_dev, LaunchCtx &ctx) {
+  const int U = p.B * p.H_kv;
+  UnitInfo *ui = reinterpret_cast<UnitInfo *>(ws + L.unit_info);
+  int32_t *sched = reinterpret_cast<int32_t *>(ws + L.sched);
+  int32_t *ret1 = reinterpret_cast<int32_t *>(ws + L.ret_idx);      // kept entries of the merge pass
+  int32_t *target = reinterpret_cast<int32_t *>(ws + L.target);
+  int32_t *ev_idx = reinterpret_cast<int32_t *>(ws + L.ev_idx);
+  float *inv_norm = reinterpret_cast<float *>(ws + L.inv_norm);
+  float4 *nom_v = reinterpret_cast<float4 *>(ws + L.nom_v);
+  int32_t *nom_si = reinterpret_cast<int32_t *>(ws + L.nom_si);
+  uint32_t *grp_key = reinterpret_cast<uint32_t *>(ws + L.grp_key);
+  int32_t *grp_head = reinterpret_cast<int32_t *>(ws + L.grp_head);
+  keepkv_stats *st1 = reinterpret_cast<keepkv_stats *>(ws + L.stats2);
+  keepkv_stats *st2 = reinterpret_cast<keepkv_stats *>(ws + L.stats);
+  int32_t *unit_len = reinterpret_cast<int32_t *>(ws + L.unit_len);
+  int32_t *eff_budget = reinterpret_cast<int32_t *>(ws + L.eff_budget);
+  const int smem_keys = L.key_stride < 32768 ? L.key_stride : 32768;
+  static bool attr_done_dev[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (!attr_done_dev[dev & 63]) {
+    cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 49152 * 4);
+    cudaFuncSetAttribute(resolve_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
+    cudaFuncSetAttribute(group_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
+    attr_done_dev[dev & 63] = true;
+  }
+  // ---- pass 1: similar entries merged with each other, cache -> scratch (every head keeps its own length for now)
+  int gx = 2 * sm_count() / U;
+  gx = gx < 1 ? 1 : (gx > 32 ? 32 : gx);
+  launch_pdl(mf_prepare_kernel<D>, dim3(gx, U), dim3(256), 0, ctx.stream, p, cache, ev_idx, ui, inv_norm);
+  KEEPKV_CHECK_LAUNCH(ctx);
+  // rows and columns are the same keys: the "retained" operand of the search is the prompt itself
+  launch_nominate(p, cache, cache, ev_idx, ui, inv_norm, sched, nom_v, nom_si, L.nom_chunks, status_dev, ctx, 1);
+  launch_pdl(resolve_kernel<D>, dim3(L.nom_chunks, U), dim3(kResolveThreads), (size_t)smem_keys * 4, ctx.stream,
+      p, cache, cache, ev_idx, ui, nom_v, nom_si, sched, L.nom_chunks, ret1, target, grp_key, L.key_stride, grp_head,
+      st1, smem_keys, 1);
+  KEEPKV_CHECK_LAUNCH(ctx);
+  launch_pdl(mf_mark_kernel, dim3(U), dim3(1024), 0, ctx.stream, p, unit_len, ret1, target, ev_idx, grp_head, grp_key,
+             L.key_stride, ui, st1);
+  KEEPKV_CHECK_LAUNCH(ctx);
+  const int cgx = (p.N_cap + 63) / 64 < 32 ? (p.N_cap + 63) / 64 : 32;
+  launch_pdl(compact_kernel<D>, dim3(cgx, U), dim3(256), 0, ctx.stream, p, cache, scratch, ret1, ui, inv_norm);
+  KEEPKV_CHECK_LAUNCH(ctx);
+  launch_pdl(group_kernel<D>, dim3(U), dim3(kResolveThreads), (size_t)smem_keys * 4, ctx.stream, p, cache, scratch, ret1,
+             ev_idx, target, ui, grp_key, L.key_stride, grp_head, st1, smem_keys);
+  KEEPKV_CHECK_LAUNCH(ctx);
+  int mgx = 4096 / U;
+  mgx = mgx < 1 ? 1 : (mgx > 32 ? 32 : mgx);
+  launch_pdl(merge_kernel<D>, dim3(mgx, U), dim3(256), 0, ctx.stream, p, cache, scratch, ret1, ev_idx, target, ui, grp_key,
+             L.key_stride, grp_head, st1);
+  KEEPKV_CHECK_LAUNCH(ctx);
+  // ---- pass 2: the eviction strategy alone, scratch -> cache
+  launch_pdl(mf_budget_kernel, dim3((p.B + 127) / 128), dim3(128), 0, ctx.stream, p, budget_dev, budget_scalar, unit_len,
+             eff_budget);
+  KEEPKV_CHECK_LAUNCH(ctx);
+  int32_t *ret2 = grp_head;   // (free again: the groups are merged)
+  launch_pdl(select_kernel, dim3(U), dim3(512), (size_t)p.N_cap * sizeof(uint32_t), ctx.stream, p, scratch, cache.seq_len,
+             (const int32_t *)eff_budget, 0, n_recent_dev, ret2, target, ev_idx, ui, st2, (const float *)nullptr,
+             (const int32_t *)unit_len);
+  KEEPKV_CHECK_LAUNCH(ctx);
+  launch_pdl(compact_kernel<D>, dim3(cgx, U), dim3(256), 0, ctx.stream, p, scratch, cache, ret2, ui, inv_norm);
+  KEEPKV_CHECK_LAUNCH(ctx);
+  if (ret_idx_out || stats_out) {
+    launch_pdl(mf_compose_kernel, dim3(4, U), dim3(256), 0, ctx.stream, p, cache.seq_len, ret1, ret2, ret_idx_out, st1, ui,
+               unit_len, stats_out);
+    KEEPKV_CHECK_LAUNCH(ctx);
+  }
+}
+
+void launch_compress_merge_first(const keepkv_params &p, const keepkv_cache &cache, const keepkv_cache &scratch,
+                                 const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
+                                 int32_t *ret_idx_out, keepkv_stats *stats_out, char *ws, const WsLayout &L,
+                                 int32_t *status_dev, LaunchCtx &ctx) {
+  if (p.d == 128)
+    launch_compress_merge_first_t<128>(p, cache, scratch, budget_dev, budget_scalar, n_recent_dev, ret_idx_out, stats_out, ws,
+                                       L, status_dev, ctx);
+  else
+    launch_compress_merge_first_t<64>(p, cache, scratch, budget_dev, budget_scalar, n_recent_dev, ret_idx_out, stats_out, ws,
+                                      L, status_dev, ctx);
 }
 
 void launch_compress(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,

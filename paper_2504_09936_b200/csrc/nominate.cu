@@ -69,7 +69,7 @@ __global__ void __launch_bounds__(kNomThreads, 1)
 nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const __nv_bfloat16 *__restrict__ srcK,
                 const int32_t *__restrict__ ev_idx, const UnitInfo *__restrict__ unit_info,
                 const float *__restrict__ inv_norm, int32_t *sched, float4 *__restrict__ nom_v,
-                int32_t *__restrict__ nom_si, int C_max, int32_t *status_dev) {
+                int32_t *__restrict__ nom_si, int C_max, int32_t *status_dev, int self_mask) {
   using SL = NomSmem<D>;
   constexpr int KSTEPS = D / 16;
   constexpr uint32_t IDESC = umma_idesc_bf16(kNomM, kNomN);
@@ -312,6 +312,9 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
             tc_fence_after();
             const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + a * kNomN + half * 128;
             const int n_valid = it.n_ret - c0;   // columns of this half that exist
+            // rows and columns are the same entries (self_mask): the column of the row's own key does not count
+            const int diag = self_mask ? m0 + row - c0 : -1;
+            const bool crosses = self_mask && m0 + quarter * 32 < c0 + 128 && c0 <= m0 + quarter * 32 + 31;
 #pragma unroll 1
             for (int jg = 0; jg < 2; ++jg) {
               uint32_t r0[32], r1[32];
@@ -323,7 +326,7 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
                 if (lane == 0) mbar_arrive(bar_t_empty + 8 * a);
               }
               const int cb = jg * 64;
-              const bool ragged = n_valid < cb + 64;   // columns past n_ret hold other rows' data
+              const bool ragged = n_valid < cb + 64 || crosses;   // columns past n_ret hold other rows' data
               // `masked` is a compile-time flag: only the last tile of a row of tiles has columns to mask, and a
               // run-time test inside the unrolled loop would be turned into selects that every group pays for
               auto drain32 = [&](auto test, auto masked, const uint32_t (&r)[32], int off) {
@@ -333,10 +336,10 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
                   float a0 = __uint_as_float(r[i]), a1 = __uint_as_float(r[i + 1]);
                   float a2 = __uint_as_float(r[i + 2]), a3 = __uint_as_float(r[i + 3]);
                   if (decltype(masked)::value) {   // a masked column contributes -inf
-                    if (off + i >= n_valid) { a0 = -CUDART_INF_F; iv.x = 1.f; }
-                    if (off + i + 1 >= n_valid) { a1 = -CUDART_INF_F; iv.y = 1.f; }
-                    if (off + i + 2 >= n_valid) { a2 = -CUDART_INF_F; iv.z = 1.f; }
-                    if (off + i + 3 >= n_valid) { a3 = -CUDART_INF_F; iv.w = 1.f; }
+                    if (off + i >= n_valid || off + i == diag) { a0 = -CUDART_INF_F; iv.x = 1.f; }
+                    if (off + i + 1 >= n_valid || off + i + 1 == diag) { a1 = -CUDART_INF_F; iv.y = 1.f; }
+                    if (off + i + 2 >= n_valid || off + i + 2 == diag) { a2 = -CUDART_INF_F; iv.z = 1.f; }
+                    if (off + i + 3 >= n_valid || off + i + 3 == diag) { a3 = -CUDART_INF_F; iv.w = 1.f; }
                   }
                   offer4<decltype(test)::value>(top, topb, a0, a1, a2, a3, iv, c0 + off + i);
                 }
@@ -404,7 +407,8 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
 template <int D>
 static void launch_nominate_t(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,
                               const int32_t *ev_idx, const UnitInfo *unit_info, const float *inv_norm, int32_t *sched,
-                              float4 *nom_v, int32_t *nom_si, int nom_chunks, int32_t *status_dev, LaunchCtx &ctx) {
+                              float4 *nom_v, int32_t *nom_si, int nom_chunks, int32_t *status_dev, LaunchCtx &ctx,
+                              int self_mask) {
   using SL = NomSmem<D>;
   constexpr size_t smem_bytes = (size_t)SL::kBytes + 1024;
   static bool attr_done_dev[64] = {};
@@ -421,17 +425,17 @@ static void launch_nominate_t(const keepkv_params &p, const keepkv_cache &src, c
   }
   launch_pdl(nominate_kernel<D>, dim3(sm_count()), dim3(kNomThreads), smem_bytes, ctx.stream,
       mapB, p, reinterpret_cast<const __nv_bfloat16 *>(src.K), ev_idx, unit_info, inv_norm, sched, nom_v, nom_si,
-      nom_chunks, status_dev);
+      nom_chunks, status_dev, self_mask);
   KEEPKV_CHECK_LAUNCH(ctx);
 }
 
 void launch_nominate(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst, const int32_t *ev_idx,
                      const UnitInfo *unit_info, const float *inv_norm, int32_t *sched, float4 *nom_v, int32_t *nom_si,
-                     int nom_chunks, int32_t *status_dev, LaunchCtx &ctx) {
+                     int nom_chunks, int32_t *status_dev, LaunchCtx &ctx, int self_mask) {
   if (p.d == 128)
-    launch_nominate_t<128>(p, src, dst, ev_idx, unit_info, inv_norm, sched, nom_v, nom_si, nom_chunks, status_dev, ctx);
+    launch_nominate_t<128>(p, src, dst, ev_idx, unit_info, inv_norm, sched, nom_v, nom_si, nom_chunks, status_dev, ctx, self_mask);
   else
-    launch_nominate_t<64>(p, src, dst, ev_idx, unit_info, inv_norm, sched, nom_v, nom_si, nom_chunks, status_dev, ctx);
+    launch_nominate_t<64>(p, src, dst, ev_idx, unit_info, inv_norm, sched, nom_v, nom_si, nom_chunks, status_dev, ctx, self_mask);
 }
 
 }  // namespace keepkv

@@ -657,3 +657,68 @@ def test_decode_bounded_wait_runs_out_and_the_next_call_is_normal(B, H_kv, n, wi
     ls_after = to_f64(cache.lscore).reshape(B * H_kv, -1)
     for u in range(B * H_kv):
         check_decode_unit(p, u, hc, to_f64(q), to_f64(out), to_f64(lse), ls_after, what="after a timeout")
+
+
+@pytest.mark.parametrize("d,G,T,guard", [(128, 4, 0.8, True), (64, 1, 0.9, False), (128, 8, 0.6, True)])
+def test_prefill_compression_merge_first_policy(d, G, T, guard):
+    """keepkv_compress_merge_first (Section 3.4; App. B, Table 3): clustered keys in random order, exact duplicates
+    (equal cosines: the lower index is the partner), ragged lengths incl. an empty and a one-entry sequence, several
+    row and column tiles per unit.  The oracle runs the two passes per unit -- merge_similar, then the eviction
+    alone (compress with T = +inf) at the sequence's budget capped by its shortest merged head -- and the result
+    must agree: length, the prompt index of every kept row (exact), rows within the bf16 rules, statistics."""
+    B, H_kv = 5, 2
+    n_cap = 1216
+    lens = [1200, 0, 1, 333, 700]
+    budget, n_recent = 200, 100
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=n_cap, period=0, n_sink=4, n_recent=n_recent,
+                       merge_threshold=T, gamma_min=0.0 if guard else -math.inf, gamma_max=4.0 if guard else math.inf)
+    rng = np.random.default_rng(d + G)
+    U = B * H_kv
+    K = np.empty((U, n_cap, d), dtype=np.float32)
+    for u in range(U):
+        n_cl = 40 if u % 2 == 0 else 150            # the two heads of a sequence merge very different numbers of entries
+        centers = rng.standard_normal((n_cl, d)).astype(np.float32) * 3.0
+        K[u] = centers[rng.integers(0, n_cl, n_cap)] + 0.6 * rng.standard_normal((n_cap, d)).astype(np.float32)
+    K[:, 100] = K[:, 7]; K[:, 205] = K[:, 7]; K[:, 206] = K[:, 100]       # duplicates of entry 7
+    cache = random_cache(p, lens, seed=3, vote_max=3, scored_frac=1.0)
+    cache.K.copy_(f32_to_dev_bf16(K).view(B, H_kv, n_cap, d))
+    cache.lscore.mul_(0.25).add_(1.5)              # positive log-scores: few groups near the guard's singular point
+    scratch = kb.Cache.empty(p)
+    ws, st = kb.new_workspace(p), kb.new_status()
+    ret = torch.full((U, n_cap), -7, dtype=torch.int32, device="cuda")
+    stats = torch.zeros(U, 8, dtype=torch.int32, device="cuda")
+    hs = HostCache(cache)
+    kb.keepkv_compress_merge_first(p, cache, scratch, budget, ws, st, retained_idx=ret, stats=stats)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    hd = HostCache(cache)
+    ret, stats = ret.cpu().numpy(), stats.cpu().numpy()
+    # the oracle, pass 1 for every unit; then the budget of each sequence; then pass 2
+    P = oracle_params(p)
+    Pev = oracle_params(_copy_params(p, merge_threshold=math.inf))
+    first = [O.merge_similar(P, *hs.unit(u)) for u in range(U)]
+    assert sum(f["stats"]["n_merged"] for f in first) > 500            # the clusters did merge
+    for b in range(B):
+        eff = min([budget] + [len(first[b * H_kv + h]["ret_idx"]) for h in range(H_kv)])
+        assert int(hd.seq_len[b]) == eff, (b, hd.seq_len[b], eff)
+        for h in range(H_kv):
+            u = b * H_kv + h
+            f = first[u]
+            if any(np.isfinite(g) and min(abs(g - P.gamma_min), abs(g - P.gamma_max)) < 1e-3 * max(1.0, abs(g))
+                   for g in f["gammas"]):
+                continue                            # a group on the edge of the guard: either outcome is right
+            ref = O.compress(Pev, eff, f["K"], f["V"], f["votes"], f["lscore"], sorted_select=True)
+            assert ref["stats"]["n_merged"] == 0
+            want_idx = f["ret_idx"][ref["ret_idx"]]
+            assert np.array_equal(ret[u, :eff], want_idx), f"u={u}: kept rows differ"
+            dK, dV, dvotes, dls = hd.unit(u)
+            assert np.array_equal(dvotes, ref["votes"]), f"u={u}: votes differ"
+            check_close(dK, ref["K"], f"merge-first K u={u}")
+            check_close(dV, ref["V"], f"merge-first V u={u}")
+            check_close(dls, ref["lscore"], f"merge-first lscore u={u}", ulps=None, max_abs=1e-4, mean_rel=1e-5)
+            got = {n: int(stats[u][kb.STATS_FIELDS.index(n)]) for n in kb.STATS_FIELDS}
+            n0 = lens[b]
+            assert got["n_retained"] == eff and got["n_evicted"] == n0 - eff and got["n_below_T"] == 0
+            for n in ("n_merged", "n_groups", "n_guard_groups", "max_group"):
+                assert got[n] == f["stats"][n], (u, n, got, f["stats"])
+    assert hd.seq_len[1] == 0 and hd.seq_len[2] == 1
