@@ -98,7 +98,7 @@ def lib() -> C.CDLL:
         _lib.okv_round_bf16.argtypes = [C.c_double]
         _lib.okv_cosine.restype = C.c_float
         _lib.okv_merge_group.restype = C.c_double
-        for n in ("okv_select", "okv_select_sorted", "okv_compress", "okv_compress_keyed", "okv_merge_similar", "okv_append",
+        for n in ("okv_select", "okv_select_sorted", "okv_compress", "okv_compress_keyed", "okv_merge_similar", "okv_compress_inplace", "okv_append",
                   "okv_num_threads"):
             getattr(_lib, n).restype = C.c_int32
     return _lib
@@ -235,6 +235,24 @@ def compress(P: Params, budget: int, K, V, votes, lscore, sorted_select: bool = 
                                          _pi(target), _p(gam), C.byref(st), C.c_int32(int(sorted_select)))
     return dict(K=dK[:n_ret], V=dV[:n_ret], votes=dv[:n_ret], lscore=dl[:n_ret], ret_idx=ret[:n_ret].copy(),
                 target=target[:n].copy(), gammas=gam[:n_ret],
+                stats={f: getattr(st, f) for f, _ in _Stats._fields_ if f != "pad_"})
+
+
+def compress_inplace(P: Params, budget: int, K, V, votes, lscore, pos):
+    """Algorithm 1 in place for one unit whose rows are not in token order (pos[i] = token position of row i).
+    Returns a dict with the arrays after the call (K, V, votes, lscore, pos: n_ret rows), moved_from [n_ret] (the row
+    each final row came from), target [len] (row of the target before the placement, -1, -2), gammas [len], stats."""
+    K, V, votes, lscore = (_f64(a).copy() for a in (K, V, votes, lscore))
+    pos = np.ascontiguousarray(pos, dtype=np.int32).copy()
+    n = K.shape[0]
+    m = max(n, 1)
+    moved = np.empty(m, dtype=np.int32); target = np.empty(m, dtype=np.int32); gam = np.empty(m, dtype=np.float64)
+    st = _Stats()
+    cp = P.c()
+    n_ret = lib().okv_compress_inplace(C.byref(cp), C.c_int32(n), C.c_int32(budget), _p(K), _p(V), _p(votes), _p(lscore),
+                                       _pi(pos), _pi(moved), _pi(target), _p(gam), C.byref(st))
+    return dict(K=K[:n_ret], V=V[:n_ret], votes=votes[:n_ret], lscore=lscore[:n_ret], pos=pos[:n_ret],
+                moved_from=moved[:n_ret].copy(), target=target[:n].copy(), gammas=gam[:n],
                 stats={f: getattr(st, f) for f, _ in _Stats._fields_ if f != "pad_"})
 
 

@@ -467,6 +467,143 @@ int32_t okv_compress_keyed(const okv_params *P, int32_t len, int32_t budget, con
   return n_ret;
 }
 
+/* ---------------------------------------- Algorithm 1 in place (periodic mode, Section 1) */
+
+/* The compression of Algorithm 1 on a cache whose rows are NOT in token order, done in place: "discard (k_e, v_e),
+ * (k_c, v_c) and insert (k_r, v_r)" taken literally -- a merged entry replaces its target where it sits, an evicted
+ * entry leaves a hole, nothing else moves except what must so that the valid entries end up in rows [0, n_ret).
+ * pos[i] is the token position of row i (distinct per unit); it takes over what row order means elsewhere:
+ *   - sinks: the n_sink smallest positions; recent window: the n_recent largest positions (if the budget cannot hold
+ *     both, the recent window shrinks first, as in okv_select);
+ *   - heavy hitters: the largest kappa among the rest, equal kappa -> lower ROW;
+ *   - match: highest cosine over the retained rows, equal cosines -> lower ROW; merge iff above T;
+ *   - merge: Eq. (A.3) over the target and its members (members in ascending row order, the target first is
+ *     immaterial: the formula is symmetric), guard as in okv_compress; the result overwrites the target's row and
+ *     keeps the target's position;
+ *   - placement: n_ret = min(len, budget).  Retained rows below n_ret stay.  The retained rows at or above n_ret, in
+ *     ascending row order, move into the rows below n_ret that were evicted, in ascending row order.
+ * Arrays are modified in place (capacity >= len rows); moved_from[r] (n_ret entries, may be NULL) receives the row
+ * each final row came from; target [len] as in okv_compress but in ROW numbers before the placement (-1 evicted
+ * without merge, -2 retained); gammas [len] per row (NaN where the row had no group).  Returns n_ret.
+ * What is fixed by the paper here is only that retained entries are untouched unless merged; the tie rules by row
+ * and the placement rule are this oracle's (parity unpinned). */
+int32_t okv_compress_inplace(const okv_params *P, int32_t len, int32_t budget, double *K, double *V, double *votes,
+                             double *lscore, int32_t *pos, int32_t *moved_from, int32_t *target_out, double *gammas,
+                             okv_stats *stats) {
+  const int d = P->d;
+  const int L1 = len > 0 ? len : 1;
+  if (budget < 0) budget = 0;
+  const int n_ret = len < budget ? len : budget;
+  unsigned char *keep = (unsigned char *)calloc((size_t)L1, 1);
+  int32_t *target = (int32_t *)malloc(sizeof(int32_t) * (size_t)L1);
+  okv_stats st;
+  memset(&st, 0, sizeof st);
+  if (budget >= len) {
+    for (int i = 0; i < len; ++i) keep[i] = 1;
+  } else {
+    int n_sink = P->n_sink, n_recent = P->n_recent;
+    if (n_sink > budget) n_sink = budget;
+    if (n_recent > budget - n_sink) n_recent = budget - n_sink;
+    /* rank of every row by position */
+    for (int i = 0; i < len; ++i) {
+      int before = 0;
+      for (int j = 0; j < len; ++j) before += pos[j] < pos[i] ? 1 : 0;
+      if (before < n_sink || before >= len - n_recent) keep[i] = 1;
+    }
+    float *kappa = (float *)malloc(sizeof(float) * (size_t)L1);
+    okv_kappa(len, votes, lscore, kappa);
+    const int n_heavy = budget - n_sink - n_recent;
+    for (int r = 0; r < n_heavy; ++r) {   /* the strict '>' keeps the lowest row on ties */
+      int best = -1;
+      for (int i = 0; i < len; ++i) {
+        if (keep[i]) continue;
+        if (best < 0 || kappa[i] > kappa[best]) best = i;
+      }
+      keep[best] = 1;
+    }
+    free(kappa);
+  }
+  /* match: every evicted row against every retained row */
+  const float T = (float)P->merge_threshold;
+  float *nrm = (float *)malloc(sizeof(float) * (size_t)L1);
+  for (int i = 0; i < len; ++i) nrm[i] = sqrtf(dot_chain(K + (size_t)i * d, K + (size_t)i * d, d));
+  for (int e = 0; e < len; ++e) {
+    if (keep[e]) { target[e] = -2; continue; }
+    float best = -INFINITY;
+    int bi = -1;
+    for (int c = 0; c < len; ++c) {
+      if (!keep[c]) continue;
+      float u = dot_chain(K + (size_t)e * d, K + (size_t)c * d, d) / (nrm[e] * nrm[c]);
+      if (u > best) { best = u; bi = c; }
+    }
+    target[e] = (bi >= 0 && best > T) ? bi : -1;
+    if (target[e] == -1) st.n_below_T++;
+  }
+  free(nrm);
+  st.n_retained = n_ret;
+  st.n_evicted = len - n_ret;
+  /* merge: results are computed from the untouched inputs, then written */
+  int32_t *members = (int32_t *)malloc(sizeof(int32_t) * (size_t)(L1 + 1));
+  double *newK = (double *)malloc(sizeof(double) * (size_t)L1 * d), *newV = (double *)malloc(sizeof(double) * (size_t)L1 * d);
+  double *newp = (double *)malloc(sizeof(double) * (size_t)L1), *newl = (double *)malloc(sizeof(double) * (size_t)L1);
+  unsigned char *rewritten = (unsigned char *)calloc((size_t)L1, 1);
+  for (int c = 0; c < len; ++c) {
+    if (gammas) gammas[c] = NAN;
+    if (!keep[c]) continue;
+    int n = 0;
+    for (int e = 0; e < len; ++e)
+      if (e == c || target[e] == c) members[n++] = e;
+    if (n > 1) {
+      st.n_groups++;
+      double pr, lr, lbar;
+      double gamma = okv_merge_group(d, n, members, K, V, votes, lscore, newK + (size_t)c * d, newV + (size_t)c * d, &pr,
+                                     &lr, &lbar);
+      if (gammas) gammas[c] = gamma;
+      if (gamma > P->gamma_min && gamma <= P->gamma_max && fabs(lbar) >= 1e-6) {
+        for (int j = 0; j < d; ++j) {
+          newK[(size_t)c * d + j] = store_kv(P, newK[(size_t)c * d + j]);
+          newV[(size_t)c * d + j] = store_kv(P, newV[(size_t)c * d + j]);
+        }
+        newp[c] = store_f32(P, pr);
+        newl[c] = store_f32(P, lr);
+        rewritten[c] = 1;
+        st.n_merged += n - 1;
+        if (n - 1 > st.max_group) st.max_group = n - 1;
+      } else {
+        st.n_guard_groups++;
+        for (int t = 0; t < n; ++t)
+          if (members[t] != c) target[members[t]] = -1;
+      }
+    }
+  }
+  for (int c = 0; c < len; ++c)
+    if (rewritten[c]) {
+      memcpy(K + (size_t)c * d, newK + (size_t)c * d, sizeof(double) * (size_t)d);
+      memcpy(V + (size_t)c * d, newV + (size_t)c * d, sizeof(double) * (size_t)d);
+      votes[c] = newp[c];
+      lscore[c] = newl[c];
+    }
+  /* placement */
+  if (moved_from)
+    for (int r = 0; r < n_ret; ++r) moved_from[r] = r;
+  int hole = 0;
+  for (int m = n_ret; m < len; ++m) {
+    if (!keep[m]) continue;
+    while (keep[hole]) ++hole;   /* as many holes below n_ret as retained rows above it */
+    memcpy(K + (size_t)hole * d, K + (size_t)m * d, sizeof(double) * (size_t)d);
+    memcpy(V + (size_t)hole * d, V + (size_t)m * d, sizeof(double) * (size_t)d);
+    votes[hole] = votes[m];
+    lscore[hole] = lscore[m];
+    pos[hole] = pos[m];
+    if (moved_from) moved_from[hole] = m;
+    ++hole;
+  }
+  if (target_out) memcpy(target_out, target, sizeof(int32_t) * (size_t)len);
+  if (stats) *stats = st;
+  free(keep); free(target); free(members); free(newK); free(newV); free(newp); free(newl); free(rewritten);
+  return n_ret;
+}
+
 /* --------------------------- Section 3.4 / App. B.3: prefill "merge first, then evict" */
 
 /* The prefill merge policy of Section 3.4 (App. B, Table 3): before any eviction, entries whose keys are similar

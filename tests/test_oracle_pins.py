@@ -728,3 +728,99 @@ def test_first_observation_initialisation_is_not_the_bias_corrected_mean_after_s
     corrected = ((1 - alpha) * (alpha * s1 + s2)) / (1 - alpha ** 2)
     assert math.isclose(math.exp(ls[0]), plain, rel_tol=1e-12)
     assert abs(plain - corrected) / corrected > 0.05                             # ... and here they do not
+
+
+# ------------------------------------------------ Algorithm 1 in place (periodic mode): position array instead of row order
+
+def _sorted_by_pos(r):
+    o = np.argsort(r["pos"])
+    return r["K"][o], r["V"][o], r["votes"][o], r["lscore"][o], r["pos"][o]
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_inplace_compression_is_the_compression_of_the_token_ordered_cache(seed):
+    """Rows in random order with their token positions: the in-place compression must keep, merge and drop exactly
+    the entries that okv_compress (pinned above) keeps, merges and drops on the same cache laid out in token order
+    -- the cache order is a storage matter, the method is defined on tokens.  (Random scores and keys: no ties,
+    where the two tie rules -- lower row, lower position -- would differ.)"""
+    rng = RNG(900 + seed)
+    n, d = int(rng.integers(12, 70)), int(rng.choice([8, 16]))
+    budget = int(rng.integers(3, n))
+    q, K, V = _rand_unit(rng, n, d, 1)
+    votes = rng.integers(1, 4, n).astype(float); ls = rng.standard_normal(n)
+    P = O.Params(G=1, d=d, n_sink=int(rng.integers(0, 3)), n_recent=int(rng.integers(0, 5)),
+                 merge_threshold=float(rng.choice([-np.inf, 0.0, 0.3])))
+    ref = O.compress(P, budget, K, V, votes, ls)                         # rows = tokens
+    perm = rng.permutation(n)                                            # row i holds token perm[i]
+    got = O.compress_inplace(P, budget, K[perm], V[perm], votes[perm], ls[perm], perm)
+    gK, gV, gp, gl, gpos = _sorted_by_pos(got)
+    assert np.array_equal(gpos, ref["ret_idx"])                          # the same tokens survive
+    assert np.array_equal(gp, ref["votes"])
+    assert np.allclose(gK, ref["K"], rtol=1e-12, atol=1e-13) and np.allclose(gV, ref["V"], rtol=1e-12, atol=1e-13)
+    assert np.allclose(gl, ref["lscore"], rtol=1e-12, atol=1e-13)
+    for f in ("n_retained", "n_evicted", "n_merged", "n_below_T", "n_guard_groups", "n_groups", "max_group"):
+        assert got["stats"][f] == ref["stats"][f], f
+    # attention does not care about the order (Eq. 6 is a sum over entries)
+    o_ref, lse_ref = O.decode(P, q, ref["K"], ref["V"], ref["votes"])
+    o_got, lse_got = O.decode(P, q, got["K"], got["V"], got["votes"])
+    assert np.allclose(o_got, o_ref, atol=1e-12) and np.allclose(lse_got, lse_ref, atol=1e-12)
+
+
+def test_inplace_compression_moves_only_what_it_must():
+    """'Discard (k_e, v_e), (k_c, v_c) and insert (k_r, v_r)' taken literally: a retained row that is not a merge
+    target and sits below the new length keeps its bits and its row; retained rows above the new length fill the
+    holes in ascending order; everything is where moved_from says."""
+    rng = RNG(31)
+    n, d, budget = 40, 8, 30
+    _, K, V = _rand_unit(rng, n, d, 1)
+    votes = np.ones(n); ls = rng.standard_normal(n)
+    pos = rng.permutation(n).astype(np.int32)
+    P = O.Params(G=1, d=d, n_sink=2, n_recent=6, merge_threshold=0.2, gamma_min=-np.inf, gamma_max=np.inf)
+    r = O.compress_inplace(P, budget, K, V, votes, ls, pos)
+    tgt = r["target"]
+    kept = np.nonzero(tgt == -2)[0]
+    holes = [i for i in range(budget) if tgt[i] != -2]
+    movers = [i for i in kept if i >= budget]
+    assert len(holes) == len(movers) and len(kept) == budget
+    merged_targets = set(int(t) for t in tgt if t >= 0)
+    for row in range(budget):
+        src = int(r["moved_from"][row])
+        if row in holes:
+            assert src == movers[holes.index(row)]                       # k-th hole takes the k-th mover
+        else:
+            assert src == row
+        assert r["pos"][row] == pos[src]
+        if src not in merged_targets:                                    # untouched by the merge: the same bits
+            assert np.array_equal(r["K"][row], K[src]) and np.array_equal(r["V"][row], V[src])
+            assert r["votes"][row] == votes[src] and r["lscore"][row] == ls[src]
+        else:
+            assert r["votes"][row] == 1 + np.sum(tgt == src)             # p_r = p_c + sum of its members' votes
+    assert r["stats"]["n_merged"] == np.sum(tgt >= 0) and r["stats"]["n_below_T"] == np.sum(tgt == -1)
+    # a cache within its budget is left alone
+    same = O.compress_inplace(P, n, K, V, votes, ls, pos)
+    assert np.array_equal(same["K"], K) and np.array_equal(same["pos"], pos) and list(same["moved_from"]) == list(range(n))
+
+
+def test_inplace_compression_ties_go_to_the_lower_row_and_theorem_2_holds():
+    """Equal selection keys and equal cosines are decided by the lower ROW (this oracle's rule for a cache without
+    order); and Theorem 2 does not care where rows sit: with s_hat = s^t the output of the step is unchanged."""
+    rng = RNG(32)
+    n, d = 16, 8
+    q, K, V = _rand_unit(rng, n, d, 1)
+    K[9] = K[3]                                                          # two identical keys: equal cosines to anything
+    P = O.Params(G=1, d=d, n_sink=0, n_recent=0, ema_alpha=0.0, merge_threshold=-np.inf, gamma_min=-np.inf,
+                 gamma_max=np.inf)
+    ls = np.zeros(n); ls[[3, 9]] = 5.0; ls[[2, 7, 11]] = 1.0             # rows 3 and 9 kept; 2, 7, 11 tie for the third place
+    pos = np.arange(n)[::-1].copy()                                      # reversed: the lower row is the LATER token
+    r = O.compress_inplace(P, 3, K, V, np.ones(n), ls, pos)
+    assert sorted(np.nonzero(r["target"] == -2)[0]) == [2, 3, 9]         # row 2 wins the tie, not the earlier tokens 7, 11
+    # an evicted row identical in direction to rows 3 and 9 would tie: check with row 12 := 2 * K[3]
+    K2 = K.copy(); K2[12] = 2.0 * K[3]
+    r2 = O.compress_inplace(P, 3, K2, V, np.ones(n), ls, pos)
+    assert r2["target"][12] == 3                                         # equal cosines (1.0): the lower row
+    ls_t = O.score_update(P, q, K, np.full(n, -np.inf))
+    o0, lse0 = O.decode(P, q, K, V, np.ones(n))
+    r3 = O.compress_inplace(P, 5, K, V, np.ones(n), ls_t, pos)
+    if np.nanmax(np.abs(r3["gammas"])) < 1e6:
+        o1, lse1 = O.decode(P, q, r3["K"], r3["V"], r3["votes"])
+        assert np.max(np.abs(o1 - o0)) < 1e-9 and abs(lse1[0] - lse0[0]) < 1e-9
