@@ -33,19 +33,21 @@ if ROOT not in sys.path:
 from paper_2504_09936_b200 import workloads as W  # noqa: E402
 
 METRIC = "decode tokens/s + compress GB/s, fraction of HBM roofline"
-# dram__bytes_read.sum + dram__bytes_write.sum of one steady-state decode launch of workload C2, from the ncu
-# capture summarised in profiles/decode_kernel_C2_steady.md (57.68 MB + 0.61 MB); None for other workloads
-DECODE_TRAFFIC_BYTES = 58.29e6
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the kernel the roofline entry times
+# (keepkv_decode_step in the steady state), per workload, from an ncu capture of that kernel as it stands now;
+# None where no capture of the current kernel exists
+DECODE_TRAFFIC_BYTES = {"C2": None}
 UNIT = "tokens/s"
 
 
 def peaks():
+    """(HBM copy rate in GB/s, sustained dense bf16 rate in TFLOP/s, where they come from)."""
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
             m = json.load(f)
-        return float(m["hbm_gbs"]), "measured"
+        return float(m["hbm_gbs"]), float(m.get("bf16_tflops_sustained", 1400.0)), "measured"
     except Exception:
-        return 6650.0, "fallback"
+        return 6650.0, 1400.0, "fallback"
 
 
 def decode_bytes(w, entries_total):
@@ -149,28 +151,41 @@ def oracle_period_time(w, n_units, n_decode, seed_layer=0):
 def run_reference(args, w, rank):
     if rank != 0:
         return
-    t_all = []
+    # A step is one compression period of ONE layer cache (the oracle has no cache to miss): every decode step of the
+    # period is executed where that stays within a few seconds, else a stated number of them; `timed_s` is what
+    # the clock really measured for one step, `ms_per_step` the period it stands for.
+    n_dec = w.period if w.period * w.U * (w.budget() + w.period) * w.d * w.G <= 2.5e10 else 8
+    t_all, t_meas = [], []
     for _ in range(min(args.warmup, 1)):
-        oracle_period_time(w, w.U, 8)
+        oracle_period_time(w, w.U, n_dec)
     info = None
     for _ in range(args.steps):
-        info = oracle_period_time(w, w.U, 8)
+        t0 = time.perf_counter()
+        info = oracle_period_time(w, w.U, n_dec)
+        t_meas.append(time.perf_counter() - t0)
         t_all.append(info[0])
     period_s = float(np.mean(t_all))
     val = w.B * w.period / period_s
-    cpu = {"value": val, "unit": UNIT, "cores": info[1], "kind": "oracle", "sample": info[2]}
+    cpu = {"value": val, "unit": UNIT, "cores": info[1], "kind": "oracle", "sample": info[2],
+           "timed_s": float(np.mean(t_meas)), "decode_steps_timed": n_dec, "decode_steps_per_period": w.period}
     print(json.dumps({"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
                       "steps": args.steps, "warmup": args.warmup, "ms_per_step": period_s * 1e3,
                       "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-                      "data": "synthetic", "config": config_dict(w, args, "cpu"), "cpu_baseline": cpu,
+                      "data": "synthetic", "config": config_dict(w, args), "cpu_baseline": cpu,
                       "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
                       "gpu_launches": 0}))
 
 
-def config_dict(w, args, l2):
-    return {"workload": f"{w.name}: B={w.B}, {w.H_q}q/{w.H_kv}kv heads, d={w.d}, N={w.N}, budget {w.budget()} "
-                        f"({w.budget_ratio:.0%}), period {w.period}; steady-state compression period",
-            "layers_round_robin": args.layers, "l2": l2, "parallelism": f"replicas x{args.gpus}"}
+def config_dict(w, args):
+    b, P = w.budget(), w.period
+    mb = (w.U * (b + P // 2) * (4 * w.d + 12) + 4 * w.B * w.H_q * w.d) / 1e6
+    return {"workload": f"{w.name}: B={w.B}, {w.H_q}q/{w.H_kv}kv heads, d={w.d}, N={w.N}, budget {b} "
+                        f"({w.budget_ratio:.0%}), period {P}; steady-state compression period",
+            "tokens": "layer-tokens: one token of one sequence attended in one layer cache (B * period * layers per step)",
+            "layers_round_robin": args.layers,
+            "l2": f"each call works on one of {args.layers} distinct layer caches visited round-robin "
+                  f"({args.layers} x {mb:.0f} MB > 126 MB L2)",
+            "parallelism": f"replicas x{args.gpus}"}
 
 
 # --------------------------------------------------------------------------- replicas (N > 1)
@@ -339,9 +354,14 @@ def run_ours(args, w, rank, world):
         with torch.cuda.graph(gd, stream=stream):
             for _ in range(reps):
                 for l in range(L):
-                    kb.keepkv_decode_attention(p, cur[l], q_all[P // 2], out, None, True, ws, st)
+                    kb.keepkv_decode_step(p, cur[l], q_all[P // 2], kn_all[P // 2], vn_all[P // 2], out, None, True, ws, st)
+        lens_keep = [c_.seq_len.clone() for c_ in cur]            # the launch the loop runs appends: put the lengths back
         gd.replay(); stream.synchronize()
+        for c_, n_ in zip(cur, lens_keep):
+            c_.seq_len.copy_(n_)
         e0.record(); gd.replay(); e1.record(); stream.synchronize()
+        for c_, n_ in zip(cur, lens_keep):
+            c_.seq_len.copy_(n_)
         t_decode = e0.elapsed_time(e1) * 1e-3 / (reps * L)
         # ---- compression alone (incremental, budget + P -> budget), as a graph of the L calls
         for t in range(P // 2, P):
@@ -356,6 +376,25 @@ def run_ours(args, w, rank, world):
         e0.record(); gc.replay(); gc.replay(); e1.record(); stream.synchronize()
         t_inc_compress = e0.elapsed_time(e1) * 1e-3 / (2 * L)
         m_inc = float(stats[:, :, 2].sum().item()) / (L * w.U)
+        # ---- the same compression in place (position array; only evicted / merged rows are touched), on copies
+        t_inplace = None
+        if not ragged:
+            ip = [kb.Cache(c_.K.clone(), c_.V.clone(), c_.votes.clone(), c_.lscore.clone(), c_.seq_len.clone()) for c_ in cur[:min(L, 4)]]
+            pos0 = torch.arange(n_cap, dtype=torch.int32, device="cuda").expand(w.B, w.H_kv, n_cap).contiguous()
+            pos_l = [pos0.clone() for _ in ip]
+            plen_l = [c_.seq_len.clone() for c_ in ip]
+            seen_l = [c_.seq_len.clone() for c_ in ip]
+            for c_, a_, b_, s_ in zip(ip, pos_l, plen_l, seen_l):     # warm (loads the kernels); then restore the lengths
+                kb.keepkv_compress_inplace(p, c_, a_, b_, s_, budget_arg, ws, st)
+            stream.synchronize()
+            for c_, b_, src_ in zip(ip, plen_l, cur):
+                c_.seq_len.copy_(src_.seq_len); b_.copy_(src_.seq_len)   # rows beyond the budget count as fresh tokens again
+            e0.record()
+            for c_, a_, b_, s_ in zip(ip, pos_l, plen_l, seen_l):
+                kb.keepkv_compress_inplace(p, c_, a_, b_, s_, budget_arg, ws, st)
+            e1.record(); stream.synchronize()
+            t_inplace = e0.elapsed_time(e1) * 1e-3 / len(ip)
+            del ip, pos_l
         cur, oth = oth, cur                   # the compressed caches are current now
 
         # ---- end to end through the host-buffer entry point: pinned inputs in, outputs back, every step
@@ -402,9 +441,9 @@ def run_ours(args, w, rank, world):
     tokens_per_step = w.B * P * L * world
     value = job_throughput(w.B * P * L, world, args.steps, t_steps)
     e2e_val = job_throughput(w.B * P * L, world, 1, t_e2e)
-    hbm, src = peaks()
+    hbm, tens, src = peaks()
     bud64 = bud.astype(np.int64)
-    entries = int((bud64 + P // 2).sum()) * w.H_kv
+    entries = int((bud64 + P // 2 + 8).sum()) * w.H_kv      # the timed launches append: 16 replays from mid period
     ach = decode_bytes(w, entries) / t_decode / 1e9
     full_dec_gbs = decode_bytes(w, int(lens.astype(np.int64).sum()) * w.H_kv) / t_full_decode / 1e9
 
@@ -423,16 +462,25 @@ def run_ours(args, w, rank, world):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": t_steps / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
-        "config": config_dict(w, args, f"each call works on one of {L} distinct layer caches visited round-robin "
-                                       f"({L} x {decode_bytes(w, entries) / 1e6:.0f} MB > 126 MB L2)"),
+        "config": config_dict(w, args),
         "clocks": clocks, "gpu_launches": launches,
         "e2e": {"value": e2e_val, "unit": UNIT,
                 "h2d_bytes_per_step": int(L * P * (q_all[0].numel() + 2 * kn_all[0].numel()) * 2),
                 "d2h_bytes_per_step": int(L * P * out.numel() * 2), "steps": n_e2e,
                 "note": "keepkv_decode_step_host_layers called once per token for all layers, stream sync after every step"},
-        "roofline": {"bound": "hbm", "kernel": "decode_kernel", "achieved": ach, "peak": hbm, "unit": "GB/s",
-                     "frac": ach / hbm, "peak_source": src, "traffic": DECODE_TRAFFIC_BYTES if w.name == "C2" else None,
+        "roofline": {"bound": "hbm", "kernel": "decode_kernel (keepkv_decode_step, the launch the timed loop runs)",
+                     "achieved": ach, "peak": hbm, "unit": "GB/s", "frac": ach / hbm, "peak_source": src,
+                     "traffic": DECODE_TRAFFIC_BYTES.get(w.name),
                      "bytes_per_launch": decode_bytes(w, entries), "us_per_launch": t_decode * 1e6},
+        "roofline_compress_incremental": {
+            "bound": "hbm", "kernel": "steady_compress_kernel" if steady else "compression pipeline (5 kernels)",
+            "achieved": inc_gbs, "peak": hbm, "unit": "GB/s", "frac": inc_gbs / hbm, "peak_source": src, "traffic": None,
+            "bytes_per_call": inc_bytes, "us_per_call": t_inc_compress * 1e6},
+        "roofline_compress_full": {
+            "bound": "tensor", "kernel": "nominate_kernel (similarity search of the first compression)",
+            "achieved": gemm_flops / t_full_compress / 1e12, "peak": tens, "unit": "TFLOP/s",
+            "frac": gemm_flops / t_full_compress / 1e12 / tens, "peak_source": src + " (sustained bf16)", "traffic": None,
+            "flops_per_call": gemm_flops, "us_per_call": t_full_compress * 1e6},
         "phases": {
             "decode_steady_us": t_decode * 1e6, "decode_steady_gbs": ach, "decode_steady_frac_hbm": ach / hbm,
             "decode_full_cache_us": t_full_decode * 1e6, "decode_full_cache_gbs": full_dec_gbs,
@@ -445,6 +493,8 @@ def run_ours(args, w, rank, world):
             "compress_full_us": t_full_compress * 1e6, "compress_full_gbs": full_gbs,
             "compress_full_frac_hbm": full_gbs / hbm, "merged_per_unit_full": m_full,
             "compress_full_gemm_tflops": gemm_flops / t_full_compress / 1e12,
+            "compress_inplace_us": None if t_inplace is None else t_inplace * 1e6,
+            "compress_inplace_note": "keepkv_compress_inplace on the same caches: rows touched = evicted + merged, not the whole cache",
         },
     }
     if rank == 0:

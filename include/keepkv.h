@@ -56,6 +56,9 @@ typedef enum keepkv_status {
 #define KEEPKV_DEV_NOT_STEADY 4    /* keepkv_compress with KEEPKV_FLAG_COMPRESS_STEADY met a unit  */
                                    /* outside the steady-state limits; it was left untouched     */
 
+#define KEEPKV_DEV_POSITIONS 8     /* keepkv_compress_inplace: a unit's position array does not hold its n_sink first */
+                                   /* and n_recent last tokens; its result is unspecified                         */
+
 typedef struct keepkv_params {
   int32_t B;                /* sequences                                                       */
   int32_t H_q;              /* query heads                                                     */
@@ -185,6 +188,35 @@ int keepkv_compress_scored(const keepkv_params *p, const keepkv_cache *src, cons
                            const float *select_score_or_null, const int32_t *budget_dev, int32_t budget_scalar,
                            const int32_t *n_recent_dev, int32_t *retained_idx_or_null, int32_t *target_or_null,
                            keepkv_stats *stats_or_null, void *ws, size_t ws_bytes, int32_t *status_dev, void *stream);
+
+/* Algorithm 1 in place, for the periodic mode of Section 1 and any loop that compresses every few steps: "discard
+ * (k_e, v_e), (k_c, v_c) and insert (k_r, v_r)" taken literally.  Retained entries stay in their rows, a merged entry
+ * overwrites its target's row, and only the retained rows at or beyond the new length move, into the rows of evicted
+ * entries below it: a steady-state compression touches O(evicted + merged) rows instead of rewriting the cache.  The
+ * price is that the cache is no longer in token order, so the caller keeps three more arrays with it:
+ *   pos      i32 [B, H_kv, N_cap]  token position of every row (valid for rows below pos_len[b])
+ *   pos_len  i32 [B]               rows whose position is recorded; rows [pos_len[b], seq_len[b]) are the tokens
+ *                                  appended since (keepkv_append / keepkv_decode_step), in order
+ *   n_seen   i32 [B]               tokens of the sequence that have a recorded position
+ * The call first gives the appended rows the positions n_seen[b], n_seen[b] + 1, ...; on return pos_len[b] =
+ * seq_len[b] = the new length and n_seen[b] counts them.  To start after keepkv_compress (whose dst is in token
+ * order): pos = its retained_idx output, pos_len = its new length, n_seen = the prompt length.
+ * Per unit, with len = seq_len[b] and the budget as in keepkv_compress:
+ *   1. retained set: the n_sink smallest and the n_recent largest positions, and the largest kappa among the other
+ *      rows, equal keys -> lower ROW; (the first n_sink and last n_recent tokens must all be present, which holds as
+ *      long as the windows are not enlarged between calls: otherwise KEEPKV_DEV_POSITIONS is raised)
+ *   2. every evicted row takes the retained row of highest cosine similarity, equal values -> lower ROW, and is
+ *      merged iff that cosine exceeds merge_threshold (the cosine of keepkv_compress);
+ *   3. every target with members is rewritten in its row by Eq. A.3, guard as in keepkv_compress;
+ *   4. with n = min(len, budget): the retained rows at or above n, in ascending order, move into the evicted rows
+ *      below n, in ascending order (K, V, votes, lscore, pos); seq_len[b] = n.
+ * On a cache in token order without equal keys or cosines the surviving entries are those of keepkv_compress.
+ * Optional outputs: moved_from_or_null i32 [B, H_kv, N_cap] (the row each final row came from), target_or_null
+ * i32 [B, H_kv, N_cap] (per row before step 4: row of its target, -1 dropped, -2 retained), stats_or_null. */
+int keepkv_compress_inplace(const keepkv_params *p, const keepkv_cache *cache, int32_t *pos, int32_t *pos_len,
+                            int32_t *n_seen, const int32_t *budget_dev, int32_t budget_scalar,
+                            const int32_t *n_recent_dev, int32_t *moved_from_or_null, int32_t *target_or_null,
+                            keepkv_stats *stats_or_null, void *ws, size_t ws_bytes, int32_t *status_dev, void *stream);
 
 /* Prefill compression with the merge policy of Section 3.4 (App. B, Table 3): "merge first, then evict".  Before any
  * eviction, entries of the prompt whose keys are similar enough are merged with each other; the eviction strategy

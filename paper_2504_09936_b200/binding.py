@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkeepkv.so")
 
 EXPORTS = ("keepkv_workspace_bytes", "keepkv_workspace_init", "keepkv_append", "keepkv_decode_attention",
-           "keepkv_decode_step", "keepkv_compress", "keepkv_compress_scored", "keepkv_compress_merge_first", "keepkv_prefill_scores", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_debug_decode", "keepkv_status_string", "keepkv_last_cuda_error",
+           "keepkv_decode_step", "keepkv_compress", "keepkv_compress_scored", "keepkv_compress_merge_first", "keepkv_compress_inplace", "keepkv_prefill_scores", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_debug_decode", "keepkv_status_string", "keepkv_last_cuda_error",
            "keepkv_last_launch_count")
 
 
@@ -36,7 +36,7 @@ class keepkv_cache(C.Structure):
 
 
 FLAG_COMPRESS_STEADY = 1   # keepkv_params.flags: the caller promises steady-state units, one kernel compresses them
-DEV_APPEND_FULL, DEV_TIMEOUT, DEV_NOT_STEADY = 1, 2, 4   # bits of *status_dev
+DEV_APPEND_FULL, DEV_TIMEOUT, DEV_NOT_STEADY, DEV_POSITIONS = 1, 2, 4, 8   # bits of *status_dev
 
 STATS_FIELDS = ("n_retained", "n_evicted", "n_merged", "n_below_T", "n_guard_groups", "n_groups", "max_group",
                 "reserved")
@@ -69,6 +69,7 @@ def lib() -> C.CDLL:
         l.keepkv_compress.argtypes = [pp, pc, pc, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         l.keepkv_compress_scored.argtypes = [pp, pc, pc, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         l.keepkv_compress_merge_first.argtypes = [pp, pc, pc, vp, i32, vp, vp, vp, vp, sz, vp, vp]
+        l.keepkv_compress_inplace.argtypes = [pp, pc, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         l.keepkv_decode_step_host.argtypes = [pp, pc] + [vp] * 8 + [C.c_int, vp, sz, vp, vp]
         l.keepkv_decode_step_host_layers.argtypes = [pp, pc, i32] + [vp] * 8 + [C.c_int, vp, sz, vp, vp]
         _lib = l
@@ -194,6 +195,18 @@ def keepkv_compress_scored(p, src: Cache, dst: Cache, select_score, budget, ws, 
                                         bsc, _ptr(n_recent_dev), _ptr(retained_idx), _ptr(target), _ptr(stats),
                                         ws.data_ptr(), ws.numel(), status.data_ptr(), _stream(stream)),
            "keepkv_compress_scored")
+
+
+def keepkv_compress_inplace(p, cache: Cache, pos, pos_len, n_seen, budget, ws, status, n_recent_dev=None, moved_from=None,
+                            target=None, stats=None, stream=None):
+    """Algorithm 1 in place: pos int32 [B, H_kv, N_cap], pos_len and n_seen int32 [B] travel with the cache (see the header)."""
+    for t in (pos, pos_len, n_seen):
+        assert t.dtype == torch.int32 and t.is_cuda and t.is_contiguous()
+    bdev, bsc = (budget.data_ptr(), 0) if isinstance(budget, torch.Tensor) else (None, int(budget))
+    _check(lib().keepkv_compress_inplace(C.byref(p), C.byref(cache.c()), pos.data_ptr(), pos_len.data_ptr(), n_seen.data_ptr(),
+                                         bdev, bsc, _ptr(n_recent_dev), _ptr(moved_from), _ptr(target), _ptr(stats),
+                                         ws.data_ptr(), ws.numel(), status.data_ptr(), _stream(stream)),
+           "keepkv_compress_inplace")
 
 
 def keepkv_compress_merge_first(p, cache: Cache, scratch: Cache, budget, ws, status, n_recent_dev=None,

@@ -41,6 +41,7 @@ WsLayout ws_layout(const keepkv_params &p) {
   L.stats2 = take(U * sizeof(keepkv_stats));
   L.unit_len = take(U * 4);
   L.eff_budget = take((size_t)p.B * 4);
+  L.kept = take(U * N * 4);
   L.total = off;
   return L;
 }
@@ -210,6 +211,30 @@ int keepkv_compress_scored(const keepkv_params *p, const keepkv_cache *src, cons
                   target_or_null ? target_or_null : (int32_t *)(w + L.target),
                   stats_or_null ? stats_or_null : (keepkv_stats *)(w + L.stats), w, L, status_dev, ctx,
                   select_score_or_null);
+  return finish(ctx);
+}
+
+int keepkv_compress_inplace(const keepkv_params *p, const keepkv_cache *cache, int32_t *pos, int32_t *pos_len,
+                            int32_t *n_seen, const int32_t *budget_dev, int32_t budget_scalar,
+                            const int32_t *n_recent_dev, int32_t *moved_from_or_null, int32_t *target_or_null,
+                            keepkv_stats *stats_or_null, void *ws, size_t ws_bytes, int32_t *status_dev, void *stream) {
+  int rc = validate(p);
+  if (rc) return rc;
+  if ((rc = validate_cache(cache))) return rc;
+  if (!pos || !pos_len || !n_seen || !ws || !status_dev || !aligned(ws, 256)) return KEEPKV_ERR_INVALID_ARG;
+  if ((long long)p->B * p->H_kv > kMaxUnits) return KEEPKV_ERR_UNSUPPORTED;
+  if (p->flags & KEEPKV_FLAG_COMPRESS_STEADY) return KEEPKV_ERR_INVALID_ARG;
+  if (!budget_dev) {
+    if (budget_scalar < 0) return KEEPKV_ERR_INVALID_ARG;
+    if (budget_scalar > p->N_cap || (long long)budget_scalar + p->period > p->N_cap) return KEEPKV_ERR_CAPACITY;
+  }
+  WsLayout L = ws_layout(*p);
+  if (ws_bytes < L.total) return KEEPKV_ERR_WORKSPACE;
+  LaunchCtx ctx{(cudaStream_t)stream, 0, cudaSuccess};
+  char *w = (char *)ws;
+  launch_compress_inplace(*p, *cache, pos, pos_len, n_seen, budget_dev, budget_scalar, n_recent_dev, moved_from_or_null,
+                          target_or_null ? target_or_null : (int32_t *)(w + L.target),
+                          stats_or_null ? stats_or_null : (keepkv_stats *)(w + L.stats), w, L, status_dev, ctx);
   return finish(ctx);
 }
 

@@ -38,6 +38,7 @@ struct WsLayout {
   size_t stats2;      // keepkv_stats [U]   merge-first: statistics of the merge pass
   size_t unit_len;    // i32 [U]            merge-first: entries of each unit after the merge pass
   size_t eff_budget;  // i32 [B]            merge-first: budget of each sequence, capped by its shortest head
+  size_t kept;        // i32 [U,N]          in place: the retained rows, ascending
   size_t total;
   size_t decode_bytes;   // the leading part that keepkv_decode_attention uses (counters and partials)
   size_t counter_bytes;  // size of the counters array
@@ -71,6 +72,11 @@ void launch_compress(const keepkv_params &p, const keepkv_cache &src, const keep
 void launch_nominate(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst, const int32_t *ev_idx,
                      const UnitInfo *unit_info, const float *inv_norm, int32_t *sched, float4 *nom_v, int32_t *nom_si,
                      int nom_chunks, int32_t *status_dev, LaunchCtx &ctx, int self_mask = 0);
+// Algorithm 1 in place on a cache with a position array (compress.cu)
+void launch_compress_inplace(const keepkv_params &p, const keepkv_cache &c, int32_t *pos, int32_t *pos_len, int32_t *n_seen,
+                             const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
+                             int32_t *moved_from, int32_t *target, keepkv_stats *stats, char *ws, const WsLayout &L,
+                             int32_t *status_dev, LaunchCtx &ctx);
 // Section 3.4, prefill merge-first policy (compress.cu): cache -> scratch (merge) -> cache (eviction)
 void launch_compress_merge_first(const keepkv_params &p, const keepkv_cache &cache, const keepkv_cache &scratch,
                                  const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,

@@ -20,7 +20,8 @@ constexpr int kWarpSelectMax = 2048;   // candidate sets up to this size are sea
 __global__ void __launch_bounds__(1024)
 select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int32_t *budget_dev, int budget_scalar,
               const int32_t *n_recent_dev, int32_t *ret_idx, int32_t *target, int32_t *ev_idx, UnitInfo *unit_info,
-              keepkv_stats *stats, const float *__restrict__ select_key, const int32_t *__restrict__ unit_len) {
+              keepkv_stats *stats, const float *__restrict__ select_key, const int32_t *__restrict__ unit_len,
+              int32_t *pos, const int32_t *pos_len, const int32_t *n_seen, int32_t *status_dev) {
   extern __shared__ uint32_t keys[];
   __shared__ int hist[256];
   __shared__ int warp_tot[32];
@@ -49,9 +50,34 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
   // Short units need few threads, and every barrier below costs by the warp: the surplus warps leave.
   const int nthr = min((int)blockDim.x, max(128, ((len + 3) / 4 + 31) & ~31)), nw = nthr >> 5;
   if (tid >= nthr) return;
-  for (int i = tid; i < len; i += nthr) {
-    // the caller's scores where given, else kappa = ln p + lscore
-    keys[i] = select_key ? ordered_key(select_key[base + i]) : kappa_key(src.votes[base + i], src.lscore[base + i]);
+  if (pos) {
+    // A cache that is not in token order (in-place compression): sinks and recent window are told by the token
+    // position of a row, not by the row.  Rows from pos_len[b] on are the tokens appended since the last call, in
+    // order: they get their positions here.  A sink or recent row takes key 0, below every real key, so that the
+    // search over all rows ranks the candidates only; what the row order decides elsewhere (equal keys), it
+    // decides here too.
+    const int first_fresh = max(0, min(pos_len[b], len)), n_total = n_seen[b] + (len - first_fresh);
+    const bool all = budget >= len;
+    int n_fixed = 0;
+    for (int i = tid; i < len; i += nthr) {
+      int ps = pos[base + i];
+      if (i >= first_fresh) { ps = n_seen[b] + (i - first_fresh); pos[base + i] = ps; }
+      const bool fixed = all || ps < n_sink || ps >= n_total - n_recent;
+      n_fixed += (!all && fixed) ? 1 : 0;
+      keys[i] = fixed ? 0u : kappa_key(src.votes[base + i], src.lscore[base + i]);
+    }
+    int tot;
+    block_excl_sum(n_fixed, warp_tot, tot, nw);
+    // the n_sink first and the n_recent last tokens must all be present (they are, if the windows never grew faster
+    // than the cache): otherwise positions and ranks disagree and the unit is reported, its result unspecified
+    if (!all && tot != n_sink + n_recent && tid == 0) atomicOr(status_dev, KEEPKV_DEV_POSITIONS);
+    lo = 0;
+    hi = len;
+  } else {
+    for (int i = tid; i < len; i += nthr) {
+      // the caller's scores where given, else kappa = ln p + lscore
+      keys[i] = select_key ? ordered_key(select_key[base + i]) : kappa_key(src.votes[base + i], src.lscore[base + i]);
+    }
   }
   __syncthreads();
 
@@ -129,6 +155,7 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
   // scan per sweep gives the slots.  The rank among keys equal to the threshold is needed only if
   // some of them lose.
   const bool rank_ties = n_heavy > 0 && n_tie < tot_ties;
+  auto valid_key = [&](int i) { return i < len ? keys[i] : 0u; };
   constexpr int RUN = 4;
   int base_tie = 0, base_keep = 0;
   for (int start = 0; start < len; start += nthr * RUN) {
@@ -138,8 +165,8 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
 #pragma unroll
     for (int r = 0; r < RUN; ++r) {
       const int i = i0 + r;
-      const bool valid = i < len, in_mid = valid && i >= lo && i < hi;
-      const uint32_t k = valid ? keys[i] : 0u;
+      const uint32_t k = valid_key(i);
+      const bool valid = i < len, in_mid = valid && i >= lo && i < hi && !(pos && k == 0u);
       tief[r] = false;
       if (!in_mid) {
         keepf[r] = valid;
@@ -179,9 +206,9 @@ select_kernel(keepkv_params p, keepkv_cache src, int32_t *dst_seq_len, const int
     base_keep += tot_keep;
   }
   if (tid == 0) {
-    UnitInfo ui{len, base_keep, len - base_keep, 0, 0, 0, 0, 0};
+    UnitInfo ui{len, base_keep, len - base_keep, 0, 0, 0, base_keep, 0};   // (pad0: the retained count once more, for the in-place path)
     unit_info[u] = ui;
-    if (h == 0) dst_seq_len[b] = base_keep;
+    if (h == 0 && dst_seq_len) dst_seq_len[b] = base_keep;   // (in place: the length changes when the rows have moved)
     keepkv_stats st;
     st.n_retained = base_keep; st.n_evicted = len - base_keep; st.n_merged = 0;
     st.n_below_T = len - base_keep;   // resolve_kernel replaces this once targets are known
@@ -514,7 +541,8 @@ static void launch_compress_t(const keepkv_params &p, const keepkv_cache &src, c
     return;
   }
   launch_pdl(select_kernel, dim3(U), dim3(512), sel_smem, ctx.stream, p, src, dst.seq_len, budget_dev, budget_scalar,
-             n_recent_dev, ret_idx, target, ev_idx, ui, stats, select_key, (const int32_t *)nullptr);
+             n_recent_dev, ret_idx, target, ev_idx, ui, stats, select_key, (const int32_t *)nullptr, (int32_t *)nullptr,
+             (const int32_t *)nullptr, (const int32_t *)nullptr, status_dev);
   KEEPKV_CHECK_LAUNCH(ctx);
   if (ret_bound <= 0) return;   // nothing is kept: every entry is dropped, which select has recorded
   const int cgx = (ret_bound + 63) / 64 < 32 ? (ret_bound + 63) / 64 : 32;   // the retained count is only known on the device
@@ -769,7 +797,7 @@ static void launch_compress_merge_first_t(const keepkv_params &p, const keepkv_c
   int32_t *ret2 = grp_head;   // (free again: the groups are merged)
   launch_pdl(select_kernel, dim3(U), dim3(512), (size_t)p.N_cap * sizeof(uint32_t), ctx.stream, p, scratch, cache.seq_len,
              (const int32_t *)eff_budget, 0, n_recent_dev, ret2, target, ev_idx, ui, st2, (const float *)nullptr,
-             (const int32_t *)unit_len);
+             (const int32_t *)unit_len, (int32_t *)nullptr, (const int32_t *)nullptr, (const int32_t *)nullptr, status_dev);
   KEEPKV_CHECK_LAUNCH(ctx);
   launch_pdl(compact_kernel<D>, dim3(cgx, U), dim3(256), 0, ctx.stream, p, scratch, cache, ret2, ui, inv_norm);
   KEEPKV_CHECK_LAUNCH(ctx);
@@ -790,6 +818,170 @@ void launch_compress_merge_first(const keepkv_params &p, const keepkv_cache &cac
   else
     launch_compress_merge_first_t<64>(p, cache, scratch, budget_dev, budget_scalar, n_recent_dev, ret_idx_out, stats_out, ws,
                                       L, status_dev, ctx);
+}
+
+
+// ------------------------------------------------------------------ Algorithm 1 in place (periodic mode, Section 1)
+// keepkv_compress_inplace: "discard (k_e, v_e), (k_c, v_c) and insert (k_r, v_r)" taken literally.  Retained entries
+// stay where they are, a merged entry overwrites its target's row, and only the retained rows beyond the new
+// length move (into the rows of evicted entries below it), so a compression touches O(evicted + merged) rows
+// instead of rewriting the cache.  The cache is then no longer in token order: a position array tells sinks and
+// recent window (select_kernel in position mode).  The similarity search runs over the cache as it lies: its
+// columns are all rows of the unit, and the rows that are not retained are taken out by a NaN in place of their
+// inverse norm (a NaN never passes the strict comparisons of the search).
+//   select (positions) -> ip_prepare (norms, sizes) -> nominate -> resolve (+ few merges) -> merge -> ip_move
+template <int D>
+__global__ void __launch_bounds__(256)
+ip_prepare_kernel(keepkv_params p, keepkv_cache c, const int32_t *__restrict__ target, int32_t *ident, UnitInfo *unit_info,
+                  float *__restrict__ inv_norm) {
+  constexpr int CH = D / 8;
+  pdl_wait();
+  pdl_trigger();
+  const int u = blockIdx.y;
+  const int len = unit_info[u].len;
+  const size_t base = (size_t)u * p.N_cap;
+  const uint4 *sK = reinterpret_cast<const uint4 *>(c.K);
+  const int lane = threadIdx.x & 31, ch = lane & 15, sub = lane >> 4, warp = threadIdx.x >> 5;
+  for (int r0 = blockIdx.x * 16; r0 < len; r0 += gridDim.x * 16) {   // sixteen lanes per row, two rows per warp
+    const int i = r0 + warp * 2 + sub;
+    const bool kept = i < len && target[base + i] == -2;
+    uint4 kv = make_uint4(0, 0, 0, 0);
+    if (kept && ch < CH) kv = sK[(base + i) * CH + ch];
+    float ss = 0.f;
+    const uint32_t w[4] = {kv.x, kv.y, kv.z, kv.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) { const float a = bf16_lo(w[q]), bb = bf16_hi(w[q]); ss = fmaf(a, a, ss); ss = fmaf(bb, bb, ss); }
+    ss += __shfl_xor_sync(0xffffffffu, ss, 1);
+    ss += __shfl_xor_sync(0xffffffffu, ss, 2);
+    ss += __shfl_xor_sync(0xffffffffu, ss, 4);
+    ss += __shfl_xor_sync(0xffffffffu, ss, 8);
+    if (i < len && ch == 0) {
+      inv_norm[base + i] = kept ? rsqrtf(ss) : __int_as_float(0x7fffffff);   // a row that is not retained is no column
+      ident[base + i] = i;   // the slot of a target is its row
+    }
+  }
+}
+
+// The search's column count is the unit's length (all rows lie in the operand); the rest of the record stays.
+__global__ void ip_columns_kernel(UnitInfo *unit_info, int U, int all_rows) {
+  pdl_wait();
+  pdl_trigger();
+  const int u = blockIdx.x * blockDim.x + threadIdx.x;
+  if (u < U) unit_info[u].n_ret = all_rows ? unit_info[u].len : unit_info[u].pad0;
+}
+
+// One CTA per unit: the retained rows at or above the new length move into the evicted rows below it, both in
+// ascending order (ev_idx is ascending: the holes are its head; kept is ascending: the movers are its tail).  Then
+// the new lengths are published.
+template <int D>
+__global__ void __launch_bounds__(256)
+ip_move_kernel(keepkv_params p, keepkv_cache c, int32_t *pos, int32_t *pos_len, int32_t *n_seen,
+               const int32_t *__restrict__ kept, const int32_t *__restrict__ ev_idx, const UnitInfo *__restrict__ unit_info,
+               int32_t *moved_from) {
+  constexpr int CH = D / 8;
+  __shared__ int s_holes;
+  pdl_wait();
+  pdl_trigger();
+  const int u = blockIdx.x, b = u / p.H_kv, h = u % p.H_kv, tid = threadIdx.x;
+  const UnitInfo ui = unit_info[u];
+  const int n_ret = ui.pad0, n_ev = ui.n_ev;   // pad0: the number of retained rows (n_ret holds the column count of the search)
+  const size_t base = (size_t)u * p.N_cap;
+  if (tid == 0) {   // holes = evicted rows below n_ret: a prefix of the ascending list
+    int lo = 0, hi = n_ev;
+    while (lo < hi) { const int mid = (lo + hi) >> 1; if (ev_idx[base + mid] < n_ret) lo = mid + 1; else hi = mid; }
+    s_holes = lo;
+  }
+  __syncthreads();
+  const int n_holes = s_holes;
+  if (moved_from)
+    for (int r = tid; r < n_ret; r += blockDim.x) moved_from[base + r] = r;
+  __syncthreads();
+  uint4 *K = reinterpret_cast<uint4 *>(c.K), *V = reinterpret_cast<uint4 *>(c.V);
+  for (int idx = tid; idx < n_holes * 2 * CH; idx += blockDim.x) {   // a row pair (K, V) is 2 * CH pieces of 16 bytes
+    const int k = idx / (2 * CH), piece = idx % (2 * CH);
+    const int to = ev_idx[base + k], from = kept[base + (n_ret - n_holes + k)];
+    uint4 *A = piece < CH ? K : V;
+    const int ch = piece < CH ? piece : piece - CH;
+    A[(base + to) * CH + ch] = A[(base + from) * CH + ch];
+  }
+  for (int k = tid; k < n_holes; k += blockDim.x) {
+    const int to = ev_idx[base + k], from = kept[base + (n_ret - n_holes + k)];
+    c.votes[base + to] = c.votes[base + from];
+    c.lscore[base + to] = c.lscore[base + from];
+    pos[base + to] = pos[base + from];
+    if (moved_from) moved_from[base + to] = from;
+  }
+  if (h == 0 && tid == 0) {
+    const int len = ui.len, first_fresh = max(0, min(pos_len[b], len));
+    c.seq_len[b] = n_ret;
+    n_seen[b] += len - first_fresh;
+    pos_len[b] = n_ret;
+  }
+}
+
+template <int D>
+static void launch_compress_inplace_t(const keepkv_params &p, const keepkv_cache &c, int32_t *pos, int32_t *pos_len,
+                                      int32_t *n_seen, const int32_t *budget_dev, int32_t budget_scalar,
+                                      const int32_t *n_recent_dev, int32_t *moved_from, int32_t *target, keepkv_stats *stats,
+                                      char *ws, const WsLayout &L, int32_t *status_dev, LaunchCtx &ctx) {
+  const int U = p.B * p.H_kv;
+  UnitInfo *ui = reinterpret_cast<UnitInfo *>(ws + L.unit_info);
+  int32_t *sched = reinterpret_cast<int32_t *>(ws + L.sched);
+  int32_t *ident = reinterpret_cast<int32_t *>(ws + L.ret_idx);    // slot -> row: the identity here
+  int32_t *kept = reinterpret_cast<int32_t *>(ws + L.kept);        // retained rows, ascending
+  int32_t *ev_idx = reinterpret_cast<int32_t *>(ws + L.ev_idx);
+  float *inv_norm = reinterpret_cast<float *>(ws + L.inv_norm);
+  float4 *nom_v = reinterpret_cast<float4 *>(ws + L.nom_v);
+  int32_t *nom_si = reinterpret_cast<int32_t *>(ws + L.nom_si);
+  uint32_t *grp_key = reinterpret_cast<uint32_t *>(ws + L.grp_key);
+  int32_t *grp_head = reinterpret_cast<int32_t *>(ws + L.grp_head);
+  const int smem_keys = L.key_stride < 32768 ? L.key_stride : 32768;
+  static bool attr_done_dev[64] = {};
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (!attr_done_dev[dev & 63]) {
+    cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 49152 * 4);
+    cudaFuncSetAttribute(resolve_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, 32768 * 4);
+    attr_done_dev[dev & 63] = true;
+  }
+  launch_pdl(select_kernel, dim3(U), dim3(512), (size_t)p.N_cap * sizeof(uint32_t), ctx.stream, p, c, (int32_t *)nullptr,
+             budget_dev, budget_scalar, n_recent_dev, kept, target, ev_idx, ui, stats, (const float *)nullptr,
+             (const int32_t *)nullptr, pos, (const int32_t *)pos_len, (const int32_t *)n_seen, status_dev);
+  KEEPKV_CHECK_LAUNCH(ctx);
+  int gx = 2 * sm_count() / U;
+  gx = gx < 1 ? 1 : (gx > 32 ? 32 : gx);
+  launch_pdl(ip_prepare_kernel<D>, dim3(gx, U), dim3(256), 0, ctx.stream, p, c, (const int32_t *)target, ident, ui, inv_norm);
+  KEEPKV_CHECK_LAUNCH(ctx);
+  const bool merges = !(isinf(p.merge_threshold) && p.merge_threshold > 0.f);
+  if (merges) {
+    launch_pdl(ip_columns_kernel, dim3((U + 127) / 128), dim3(128), 0, ctx.stream, ui, U, 1);
+    KEEPKV_CHECK_LAUNCH(ctx);
+    launch_nominate(p, c, c, ev_idx, ui, inv_norm, sched, nom_v, nom_si, L.nom_chunks, status_dev, ctx);
+    launch_pdl(resolve_kernel<D>, dim3(L.nom_chunks, U), dim3(kResolveThreads), (size_t)smem_keys * 4, ctx.stream,
+        p, c, c, ev_idx, ui, nom_v, nom_si, sched, L.nom_chunks, ident, target, grp_key, L.key_stride, grp_head,
+        stats, smem_keys, 0);
+    KEEPKV_CHECK_LAUNCH(ctx);
+    int mgx = 4096 / U;
+    mgx = mgx < 1 ? 1 : (mgx > 32 ? 32 : mgx);
+    launch_pdl(merge_kernel<D>, dim3(mgx, U), dim3(256), 0, ctx.stream, p, c, c, ident, ev_idx, target, ui, grp_key,
+               L.key_stride, grp_head, stats);
+    KEEPKV_CHECK_LAUNCH(ctx);
+  }
+  launch_pdl(ip_move_kernel<D>, dim3(U), dim3(256), 0, ctx.stream, p, c, pos, pos_len, n_seen, (const int32_t *)kept,
+             (const int32_t *)ev_idx, (const UnitInfo *)ui, moved_from);
+  KEEPKV_CHECK_LAUNCH(ctx);
+}
+
+void launch_compress_inplace(const keepkv_params &p, const keepkv_cache &c, int32_t *pos, int32_t *pos_len, int32_t *n_seen,
+                             const int32_t *budget_dev, int32_t budget_scalar, const int32_t *n_recent_dev,
+                             int32_t *moved_from, int32_t *target, keepkv_stats *stats, char *ws, const WsLayout &L,
+                             int32_t *status_dev, LaunchCtx &ctx) {
+  if (p.d == 128)
+    launch_compress_inplace_t<128>(p, c, pos, pos_len, n_seen, budget_dev, budget_scalar, n_recent_dev, moved_from, target,
+                                   stats, ws, L, status_dev, ctx);
+  else
+    launch_compress_inplace_t<64>(p, c, pos, pos_len, n_seen, budget_dev, budget_scalar, n_recent_dev, moved_from, target,
+                                  stats, ws, L, status_dev, ctx);
 }
 
 void launch_compress(const keepkv_params &p, const keepkv_cache &src, const keepkv_cache &dst,

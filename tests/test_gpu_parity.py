@@ -722,3 +722,144 @@ def test_prefill_compression_merge_first_policy(d, G, T, guard):
             for n in ("n_merged", "n_groups", "n_guard_groups", "max_group"):
                 assert got[n] == f["stats"][n], (u, n, got, f["stats"])
     assert hd.seq_len[1] == 0 and hd.seq_len[2] == 1
+
+
+def _check_inplace_unit(p, u, budget, n_recent, before: HostCache, pos_before, after: HostCache, pos_after, moved, tgt, stats,
+                        what, max_tolerated=0):
+    """One unit of keepkv_compress_inplace against the oracle fed the same rows and positions: targets, moves and
+    positions exact; every row of the result within the bf16 rules (a group on the guard's edge excused)."""
+    P = oracle_params(p, n_recent=n_recent)
+    K, V, votes, ls = before.unit(u)
+    n = K.shape[0]
+    ref = O.compress_inplace(P, budget, K, V, votes, ls, pos_before[u, :n])
+    m = ref["stats"]["n_retained"]
+    assert int(after.seq_len[u // p.H_kv]) == m, f"{what} u={u}: new length"
+    tg, tr = tgt[u, :n], ref["target"]
+    excused = set()
+    diff = np.nonzero(tg != tr)[0]
+    for e in diff:
+        rows = [int(r) for r in (tg[e], tr[e]) if r >= 0]
+        assert len(rows) == 1 or rows[0] == rows[1], f"{what} u={u}: target of row {e}: gpu {tg[e]} oracle {tr[e]}"
+        g = ref["gammas"][rows[0]] if rows else np.nan
+        assert np.isfinite(g) and min(abs(g - P.gamma_min), abs(g - P.gamma_max)) < 1e-3 * max(1.0, abs(g)), \
+            f"{what} u={u}: target of row {e}: gpu {tg[e]} oracle {tr[e]} (not on the guard's edge)"
+        excused.add(rows[0])
+    assert len(diff) <= max_tolerated
+    assert np.array_equal(moved[u, :m], ref["moved_from"]), f"{what} u={u}: rows moved differently"
+    assert np.array_equal(pos_after[u, :m], ref["pos"]), f"{what} u={u}: positions differ"
+    keep = np.array([int(src) not in excused for src in ref["moved_from"]], dtype=bool)
+    dK, dV, dvotes, dls = after.unit(u)
+    assert np.array_equal(dvotes[keep], ref["votes"][keep]), f"{what} u={u}: votes differ"
+    check_close(dK[keep], ref["K"][keep], f"{what} K u={u}")
+    check_close(dV[keep], ref["V"][keep], f"{what} V u={u}")
+    check_close(dls[keep], ref["lscore"][keep], f"{what} lscore u={u}", ulps=None, max_abs=1e-4, mean_rel=1e-5)
+    if not len(diff):
+        for f in ("n_retained", "n_evicted", "n_merged", "n_below_T", "n_guard_groups", "n_groups", "max_group"):
+            assert int(stats[u][kb.STATS_FIELDS.index(f)]) == ref["stats"][f], (what, u, f, stats[u], ref["stats"])
+    return ref
+
+
+def _run_inplace(p, cache, pos, pos_len, n_seen, budget, n_recent_dev=None):
+    U = p.B * p.H_kv
+    ws, st = kb.new_workspace(p), kb.new_status()
+    moved = torch.full((U, p.N_cap), -7, dtype=torch.int32, device="cuda")
+    tgt = torch.full((U, p.N_cap), -7, dtype=torch.int32, device="cuda")
+    stats = torch.zeros(U, 8, dtype=torch.int32, device="cuda")
+    kb.keepkv_compress_inplace(p, cache, pos, pos_len, n_seen, budget, ws, st, n_recent_dev=n_recent_dev, moved_from=moved,
+                               target=tgt, stats=stats)
+    torch.cuda.synchronize()
+    return int(st.item()), moved.cpu().numpy(), tgt.cpu().numpy(), stats.cpu().numpy()
+
+
+@pytest.mark.parametrize("d,G,T", [(128, 4, 0.1), (64, 2, -math.inf), (128, 1, math.inf)])
+def test_compress_inplace_on_scrambled_rows(d, G, T):
+    """keepkv_compress_inplace on caches whose rows are in random order (positions = a random permutation): ragged
+    lengths incl. one within its budget and an empty one, votes > 1, equal selection keys and duplicate keys (the
+    lower row wins), several row tiles of evicted entries; every row of the result against the oracle."""
+    B, H_kv, n_cap, budget, n_recent = 4, 2, 1408, 700, 300
+    lens = [1400, 600, 0, 1000]
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=n_cap, period=0, n_sink=4, n_recent=n_recent, merge_threshold=T)
+    cache = random_cache(p, lens, seed=d + G, vote_max=3, scored_frac=1.0)
+    cache.lscore[:, :, 50:60] = cache.lscore[:, :, 50:51]              # equal keys at the selection threshold, maybe
+    cache.K[:, :, 40] = cache.K[:, :, 10]; cache.K[:, :, 41] = cache.K[:, :, 10]      # equal cosines
+    U = B * H_kv
+    rng = np.random.default_rng(5)
+    pos_np = np.zeros((U, n_cap), dtype=np.int32)
+    for u in range(U):
+        n = lens[u // H_kv]
+        pos_np[u, :n] = rng.permutation(n)
+    pos = torch.from_numpy(pos_np).cuda().view(B, H_kv, n_cap)
+    pos_len = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    n_seen = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    before = HostCache(cache)
+    status, moved, tgt, stats = _run_inplace(p, cache, pos, pos_len, n_seen, budget)
+    assert status == 0
+    after = HostCache(cache)
+    pos_after = pos.cpu().numpy().reshape(U, n_cap)
+    new_len = [min(n, budget) for n in lens]
+    assert after.seq_len.tolist() == new_len and pos_len.tolist() == new_len and n_seen.tolist() == lens
+    merged = 0
+    for u in range(U):
+        ref = _check_inplace_unit(p, u, budget, n_recent, before, pos_np, after, pos_after, moved, tgt, stats,
+                                  what=f"in place d={d} T={T}", max_tolerated=40 if T == -math.inf else 4)
+        merged += ref["stats"]["n_merged"]
+        # rows the call had no reason to touch keep their bits
+        n = lens[u // H_kv]
+        untouched = [r for r in range(min(n, budget)) if tgt[u, r] == -2 and not np.any(tgt[u, :n] == r)]
+        assert np.array_equal(after.K[u, untouched], before.K[u, untouched]) and len(untouched) > 0 or n == 0
+    assert (merged > 0) == (T != math.inf)
+
+
+def test_compress_inplace_periodic_protocol_tracks_positions():
+    """Three periods of the loop the in-place form is for: decode steps append tokens (keepkv_decode_step knows nothing
+    of positions), keepkv_compress_inplace gives the fresh rows their positions, compresses and refills the holes.
+    Every compression is compared with the oracle on the same rows, and with the out-of-place keepkv_compress of the
+    same cache sorted by position: the same tokens survive (no ties in this data)."""
+    B, H_kv, G, d, P_ = 2, 2, 4, 128, 48
+    budget, n_recent, n0 = 256, 150, 700
+    n_cap = 768
+    p = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=n_cap, period=P_, n_sink=4, n_recent=n_recent,
+                       merge_threshold=0.05)
+    prompt = random_cache(p, [n0, n0 - 90], seed=77, scored_frac=1.0)
+    U = B * H_kv
+    # the first compression is out of place: its result is in token order and its retained_idx are the positions
+    cache, ret, _, _ = _run_compress(p, prompt, budget)
+    pos = torch.zeros(B, H_kv, n_cap, dtype=torch.int32, device="cuda")
+    pos[:, :, :budget] = torch.from_numpy(ret[:, :budget].copy()).cuda().view(B, H_kv, budget)
+    pos_len = cache.seq_len.clone()
+    n_seen = prompt.seq_len.clone()
+    ws, st = kb.new_workspace(p), kb.new_status()
+    rng = np.random.default_rng(3)
+    mk = lambda *s: f32_to_dev_bf16(rng.standard_normal(s).astype(np.float32))
+    out = torch.empty(B, H_kv * G, d, dtype=torch.bfloat16, device="cuda")
+    seen = prompt.seq_len.cpu().numpy().copy()
+    for period in range(3):
+        for t in range(P_):
+            kb.keepkv_decode_step(p, cache, mk(B, H_kv * G, d), mk(B, H_kv, d), mk(B, H_kv, d), out, None, True, ws, st)
+        torch.cuda.synchronize()
+        before = HostCache(cache)
+        pos_before = pos.cpu().numpy().reshape(U, n_cap).copy()
+        for u in range(U):                                   # what the call will assign to the fresh rows
+            pos_before[u, budget:budget + P_] = seen[u // H_kv] + np.arange(P_)
+        # the out-of-place compression of the same cache in token order, for the survivors
+        order = np.argsort(pos_before[:, :budget + P_], axis=1)
+        sorted_cache = kb.Cache(cache.K.clone(), cache.V.clone(), cache.votes.clone(), cache.lscore.clone(), cache.seq_len.clone())
+        idx = torch.from_numpy(order).cuda().view(B, H_kv, -1)
+        for tns in (sorted_cache.K, sorted_cache.V):
+            tns[:, :, :budget + P_] = torch.gather(tns[:, :, :budget + P_], 2, idx[..., None].expand(-1, -1, -1, d))
+        for tns in (sorted_cache.votes, sorted_cache.lscore):
+            tns[:, :, :budget + P_] = torch.gather(tns[:, :, :budget + P_], 2, idx)
+        _, ret_oop, _, _ = _run_compress(p, sorted_cache, budget)
+        status, moved, tgt, stats = _run_inplace(p, cache, pos, pos_len, n_seen, budget)
+        assert status == 0
+        seen += P_
+        after = HostCache(cache)
+        pos_after = pos.cpu().numpy().reshape(U, n_cap)
+        assert after.seq_len.tolist() == [budget] * B and pos_len.tolist() == [budget] * B and n_seen.tolist() == seen.tolist()
+        for u in range(U):
+            _check_inplace_unit(p, u, budget, n_recent, before, pos_before, after, pos_after, moved, tgt, stats,
+                                what=f"period {period}", max_tolerated=4)
+            survivors_oop = np.sort(pos_before[u, :budget + P_])[ret_oop[u, :budget]]
+            assert np.array_equal(np.sort(pos_after[u, :budget]), survivors_oop), f"period {period} u={u}: other tokens survive"
+            assert int((moved[u, :budget] != np.arange(budget)).sum()) <= P_      # at most one move per evicted row
+    assert int(st.item()) == 0
