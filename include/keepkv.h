@@ -262,6 +262,22 @@ int keepkv_decode_step_host_layers(const keepkv_params *p, const keepkv_cache *c
                                    void *q_dev, void *k_new_dev, void *v_new_dev, void *out_dev, int update_scores,
                                    void *ws, size_t ws_bytes, int32_t *status_dev, void *stream);
 
+/* The periodic mode of Section 1 keeps the complete KV cache outside the working memory and recompresses from it every
+ * period.  These two calls keep that complete cache in HOST memory (K_host, V_host: bf16 [B, H_kv, N_cap, d],
+ * seq_len_host: i32 [B], all host pointers; pinned memory makes the load asynchronous).
+ * keepkv_complete_append_host is Eq. 2 on the host copy: the step's k_new_host / v_new_host (bf16 [B, H_kv, d]) go
+ * to row seq_len_host[b] of every head and the lengths grow by one; a plain host memcpy, no stream involved;
+ * KEEPKV_ERR_CAPACITY, with nothing written, if a sequence is full.
+ * keepkv_complete_load_host brings the complete cache into a device cache of the same shape, enqueued on `stream`:
+ * the first seq_len_host[b] rows of K and V of every unit (one pitched copy per sequence and array), the lengths, and
+ * the state of a cache nobody has attended to yet (votes 1, lscore -INFINITY).  The host arrays must stay unchanged
+ * until the stream has passed the copies.  What follows is the ordinary path: keepkv_decode_attention with
+ * update_scores on the loaded cache scores it with the current query, keepkv_compress cuts it to the budget. */
+int keepkv_complete_append_host(const keepkv_params *p, void *K_host, void *V_host, int32_t *seq_len_host,
+                                const void *k_new_host, const void *v_new_host);
+int keepkv_complete_load_host(const keepkv_params *p, const void *K_host, const void *V_host,
+                              const int32_t *seq_len_host, const keepkv_cache *dev, void *stream);
+
 /* No counterpart in the paper: the same operation as keepkv_decode_attention for callers that cannot
  * provide a workspace because they cannot allocate device memory where they call this (code running
  * inside another runtime's memory pool, a serving loop whose buffers were all fixed at start-up, a

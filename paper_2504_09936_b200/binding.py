@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkeepkv.so")
 
 EXPORTS = ("keepkv_workspace_bytes", "keepkv_workspace_init", "keepkv_append", "keepkv_decode_attention",
-           "keepkv_decode_step", "keepkv_compress", "keepkv_compress_scored", "keepkv_compress_merge_first", "keepkv_compress_inplace", "keepkv_prefill_scores", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_debug_decode", "keepkv_status_string", "keepkv_last_cuda_error",
+           "keepkv_decode_step", "keepkv_compress", "keepkv_compress_scored", "keepkv_compress_merge_first", "keepkv_compress_inplace", "keepkv_complete_append_host", "keepkv_complete_load_host", "keepkv_prefill_scores", "keepkv_decode_step_host", "keepkv_decode_step_host_layers", "keepkv_decode_attention_static", "keepkv_debug_decode", "keepkv_status_string", "keepkv_last_cuda_error",
            "keepkv_last_launch_count")
 
 
@@ -69,6 +69,8 @@ def lib() -> C.CDLL:
         l.keepkv_compress.argtypes = [pp, pc, pc, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         l.keepkv_compress_scored.argtypes = [pp, pc, pc, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         l.keepkv_compress_merge_first.argtypes = [pp, pc, pc, vp, i32, vp, vp, vp, vp, sz, vp, vp]
+        l.keepkv_complete_append_host.argtypes = [pp, vp, vp, vp, vp, vp]
+        l.keepkv_complete_load_host.argtypes = [pp, vp, vp, vp, pc, vp]
         l.keepkv_compress_inplace.argtypes = [pp, pc, vp, vp, vp, vp, i32, vp, vp, vp, vp, vp, sz, vp, vp]
         l.keepkv_decode_step_host.argtypes = [pp, pc] + [vp] * 8 + [C.c_int, vp, sz, vp, vp]
         l.keepkv_decode_step_host_layers.argtypes = [pp, pc, i32] + [vp] * 8 + [C.c_int, vp, sz, vp, vp]
@@ -195,6 +197,22 @@ def keepkv_compress_scored(p, src: Cache, dst: Cache, select_score, budget, ws, 
                                         bsc, _ptr(n_recent_dev), _ptr(retained_idx), _ptr(target), _ptr(stats),
                                         ws.data_ptr(), ws.numel(), status.data_ptr(), _stream(stream)),
            "keepkv_compress_scored")
+
+
+def keepkv_complete_append_host(p, K_host, V_host, seq_len_host, k_new_host, v_new_host):
+    """Eq. 2 on a complete cache kept in host memory (CPU tensors; seq_len_host int32 [B] is advanced)."""
+    for t in (K_host, V_host, seq_len_host, k_new_host, v_new_host):
+        assert not t.is_cuda and t.is_contiguous()
+    _check(lib().keepkv_complete_append_host(C.byref(p), K_host.data_ptr(), V_host.data_ptr(), seq_len_host.data_ptr(),
+                                             k_new_host.data_ptr(), v_new_host.data_ptr()), "keepkv_complete_append_host")
+
+
+def keepkv_complete_load_host(p, K_host, V_host, seq_len_host, dev: Cache, stream=None):
+    """Loads the host-resident complete cache into a device cache (votes 1, no score history)."""
+    for t in (K_host, V_host, seq_len_host):
+        assert not t.is_cuda and t.is_contiguous()
+    _check(lib().keepkv_complete_load_host(C.byref(p), K_host.data_ptr(), V_host.data_ptr(), seq_len_host.data_ptr(),
+                                           C.byref(dev.c()), _stream(stream)), "keepkv_complete_load_host")
 
 
 def keepkv_compress_inplace(p, cache: Cache, pos, pos_len, n_seen, budget, ws, status, n_recent_dev=None, moved_from=None,

@@ -328,6 +328,49 @@ int keepkv_decode_step_host_layers(const keepkv_params *p, const keepkv_cache *c
   return finish(ctx);
 }
 
+int keepkv_complete_append_host(const keepkv_params *p, void *K_host, void *V_host, int32_t *seq_len_host,
+                                const void *k_new_host, const void *v_new_host) {
+  int rc = validate(p);
+  if (rc) return rc;
+  if (!K_host || !V_host || !seq_len_host || !k_new_host || !v_new_host) return KEEPKV_ERR_INVALID_ARG;
+  for (int b = 0; b < p->B; ++b)
+    if (seq_len_host[b] < 0 || seq_len_host[b] >= p->N_cap) return KEEPKV_ERR_CAPACITY;   // nothing is written
+  const size_t row = (size_t)p->d * 2;
+  for (int b = 0; b < p->B; ++b) {
+    for (int h = 0; h < p->H_kv; ++h) {
+      const size_t u = (size_t)b * p->H_kv + h, at = (u * p->N_cap + seq_len_host[b]) * row;
+      memcpy((char *)K_host + at, (const char *)k_new_host + u * row, row);
+      memcpy((char *)V_host + at, (const char *)v_new_host + u * row, row);
+    }
+    seq_len_host[b] += 1;
+  }
+  return KEEPKV_OK;
+}
+
+int keepkv_complete_load_host(const keepkv_params *p, const void *K_host, const void *V_host,
+                              const int32_t *seq_len_host, const keepkv_cache *dev, void *stream) {
+  int rc = validate(p);
+  if (rc) return rc;
+  if ((rc = validate_cache(dev))) return rc;
+  if (!K_host || !V_host || !seq_len_host) return KEEPKV_ERR_INVALID_ARG;
+  for (int b = 0; b < p->B; ++b)
+    if (seq_len_host[b] < 0 || seq_len_host[b] > p->N_cap) return KEEPKV_ERR_CAPACITY;
+  LaunchCtx ctx{(cudaStream_t)stream, 0, cudaSuccess};
+  const size_t row = (size_t)p->d * 2, pitch = (size_t)p->N_cap * row;
+  auto cp = [&](cudaError_t e) { if (e != cudaSuccess && ctx.err == cudaSuccess) ctx.err = e; };
+  for (int b = 0; b < p->B; ++b) {   // the H_kv units of a sequence have the same length: one pitched copy per array
+    if (seq_len_host[b] == 0) continue;
+    const size_t off = (size_t)b * p->H_kv * pitch, width = (size_t)seq_len_host[b] * row;
+    cp(cudaMemcpy2DAsync((char *)dev->K + off, pitch, (const char *)K_host + off, pitch, width, p->H_kv,
+                         cudaMemcpyHostToDevice, ctx.stream));
+    cp(cudaMemcpy2DAsync((char *)dev->V + off, pitch, (const char *)V_host + off, pitch, width, p->H_kv,
+                         cudaMemcpyHostToDevice, ctx.stream));
+  }
+  cp(cudaMemcpyAsync(dev->seq_len, seq_len_host, (size_t)p->B * 4, cudaMemcpyHostToDevice, ctx.stream));
+  if (ctx.err == cudaSuccess) launch_fresh_state(*p, *dev, ctx);
+  return finish(ctx);
+}
+
 const char *keepkv_status_string(int status) {
   switch (status) {
     case KEEPKV_OK: return "KEEPKV_OK";

@@ -33,6 +33,21 @@ __global__ void __launch_bounds__(128) append_kernel(keepkv_params p, keepkv_cac
   if (threadIdx.x == 0) c.seq_len[b] = pos + 1;
 }
 
+// Fresh state of a cache whose rows were just loaded: one vote per entry, no score history.
+__global__ void fresh_state_kernel(keepkv_params p, keepkv_cache c) {
+  const int u = blockIdx.y, b = u / p.H_kv;
+  const int len = max(0, min(c.seq_len[b], p.N_cap));
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < len; i += gridDim.x * blockDim.x) {
+    c.votes[(size_t)u * p.N_cap + i] = 1.0f;
+    c.lscore[(size_t)u * p.N_cap + i] = -CUDART_INF_F;
+  }
+}
+
+void launch_fresh_state(const keepkv_params &p, const keepkv_cache &c, LaunchCtx &ctx) {
+  fresh_state_kernel<<<dim3(8, p.B * p.H_kv), 256, 0, ctx.stream>>>(p, c);
+  KEEPKV_CHECK_LAUNCH(ctx);
+}
+
 void launch_append(const keepkv_params &p, const keepkv_cache &c, const void *k_new, const void *v_new,
                    int32_t *status_dev, LaunchCtx &ctx) {
   launch_pdl(append_kernel, dim3(p.B), dim3(128), 0, ctx.stream, p, c, reinterpret_cast<const uint4 *>(k_new),

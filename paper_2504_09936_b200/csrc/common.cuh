@@ -60,6 +60,7 @@ int finish_call(LaunchCtx &ctx);
 // launchers (each returns cudaSuccess or the launch error and bumps ctx.launches)
 void launch_append(const keepkv_params &p, const keepkv_cache &c, const void *k_new, const void *v_new,
                    int32_t *status_dev, LaunchCtx &ctx);
+void launch_fresh_state(const keepkv_params &p, const keepkv_cache &c, LaunchCtx &ctx);
 // k_new / v_new: the step's token to append inside the same launch (keepkv_decode_step), or null
 void launch_decode(const keepkv_params &p, const keepkv_cache &c, const void *q, void *out, float *lse,
                    int update_scores, char *ws, const WsLayout &L, int32_t *status_dev, LaunchCtx &ctx,

@@ -312,15 +312,31 @@ __device__ __forceinline__ void merge_group(const keepkv_params &p, const keepkv
     // fetched together and the row loads of the accumulation do not wait on one another
     const int idx = lane == 0 ? ci : (lane <= n ? member(lane - 1) : -1);
     const float pv = idx >= 0 ? votes[idx] : 0.f, lsv = idx >= 0 ? ls[idx] : 0.f;
-    const double a = idx >= 0 ? log((double)pv) + (double)lsv : NEG_INF;
-    const double M = wmax_d(a);
-    const double Z = wsum_d(idx >= 0 ? exp(a - M) : 0.0);
-    Ps = wsum_d((double)pv);
-    const double Lam = M + log(Z);
-    L = Lam - log(Ps);
-    const double omd = idx >= 0 ? exp(a - Lam) : 0.0;
-    lbar = wsum_d(omd * (double)lsv);
-    const float om = (float)omd;
+    // fp32 first: with |L| and |lambda_bar| away from zero its error (about 1e-6 absolute) is far below bf16
+    // resolution in gamma; only a group near the cancellation is evaluated again in fp64 (a warp-uniform choice)
+    float om;
+    {
+      const float a = idx >= 0 ? logf(pv) + lsv : -CUDART_INF_F;
+      const float M = warp_max(a);
+      const float Z = warp_sum(idx >= 0 ? expf(a - M) : 0.f);
+      const float Psf = warp_sum(pv);
+      const float Lam = M + logf(Z);
+      const float Lf = Lam - logf(Psf);
+      om = idx >= 0 ? expf(a - Lam) : 0.f;
+      const float lbf = warp_sum(om * lsv);
+      Ps = (double)Psf; L = (double)Lf; lbar = (double)lbf;
+    }
+    if (!(fabs(L) >= 0.25 && fabs(lbar) >= 0.25)) {
+      const double a = idx >= 0 ? log((double)pv) + (double)lsv : NEG_INF;
+      const double M = wmax_d(a);
+      const double Z = wsum_d(idx >= 0 ? exp(a - M) : 0.0);
+      Ps = wsum_d((double)pv);
+      const double Lam = M + log(Z);
+      L = Lam - log(Ps);
+      const double omd = idx >= 0 ? exp(a - Lam) : 0.0;
+      lbar = wsum_d(omd * (double)lsv);
+      om = (float)omd;
+    }
 #pragma unroll 4
     for (int t = 0; t <= n; ++t) accumulate(__shfl_sync(0xffffffffu, idx, t), __shfl_sync(0xffffffffu, om, t));
   } else {

@@ -7,10 +7,7 @@
 
 namespace keepkv {
 
-// Polls of a bounded mbarrier wait.  Every poll lets the hardware park the thread for up to kSuspendNs, so a wait
-// that is never satisfied gives up after about a second.
-constexpr int kSpinLimit = 1 << 16;
-constexpr uint32_t kSuspendNs = 1u << 14;
+constexpr int kSpinLimit = 1 << 20;   // polls of a bounded mbarrier wait (each poll blocks for a short hardware interval)
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -34,10 +31,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(bar), "r"(parity), "r"(kSuspendNs)
+      : "r"(bar), "r"(parity)
       : "memory");
   return ok != 0;
 }

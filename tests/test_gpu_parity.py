@@ -863,3 +863,49 @@ def test_compress_inplace_periodic_protocol_tracks_positions():
             assert np.array_equal(np.sort(pos_after[u, :budget]), survivors_oop), f"period {period} u={u}: other tokens survive"
             assert int((moved[u, :budget] != np.arange(budget)).sum()) <= P_      # at most one move per evicted row
     assert int(st.item()) == 0
+
+
+def test_periodic_mode_with_the_complete_cache_in_host_memory():
+    """Section 1's periodic mode with the complete cache kept outside the GPU: every step appends to the host copy
+    (keepkv_complete_append_host) and runs on the working cache; every period the complete cache is loaded
+    (keepkv_complete_load_host), scored by the current query, and compressed from scratch.  The loaded cache must
+    be the bits a device-resident complete cache holds, and the working cache must reproduce its output (Theorem 2)."""
+    B, H, d, P_, budget, n_cap = 2, 4, 128, 8, 96, 512
+    p = kb.make_params(B=B, H_q=H, H_kv=H, d=d, N_cap=n_cap, period=P_, n_sink=4, n_recent=40, ema_alpha=0.0,
+                       merge_threshold=-math.inf, gamma_min=-math.inf, gamma_max=math.inf)
+    full_dev = random_cache(p, [400, 250], seed=33, scored_frac=0.0, scale=0.3)
+    full_dev.K.add_(0.5)
+    full_dev.votes.fill_(1.0)
+    Kh, Vh = full_dev.K.cpu().pin_memory(), full_dev.V.cpu().pin_memory()
+    lens_h = full_dev.seq_len.cpu().clone()
+    loaded = kb.Cache.empty(p)
+    ws, st = kb.new_workspace(p), kb.new_status()
+    rng = np.random.default_rng(34)
+    q = torch.full((B, H, d), 0.25, dtype=torch.bfloat16, device="cuda")
+    for period in range(2):
+        kb.keepkv_complete_load_host(p, Kh, Vh, lens_h, loaded)
+        torch.cuda.synchronize()
+        assert torch.equal(loaded.seq_len, full_dev.seq_len)
+        for b in range(B):
+            n = int(lens_h[b])
+            assert torch.equal(loaded.K[b, :, :n].view(torch.int16), full_dev.K[b, :, :n].view(torch.int16))
+            assert torch.equal(loaded.V[b, :, :n].view(torch.int16), full_dev.V[b, :, :n].view(torch.int16))
+            assert torch.all(loaded.votes[b, :, :n] == 1) and torch.all(torch.isinf(loaded.lscore[b, :, :n]))
+        out_full, lse_full = _run_decode(p, loaded, q, True)
+        work, _, _, stats = _run_compress(p, loaded, budget)
+        out_work, lse_work = _run_decode(p, work, q, False)
+        check_close(to_f64(out_work), to_f64(out_full), f"period {period} out", ulps=None, max_abs=2e-2, mean_rel=2e-2)
+        check_close(to_f64(lse_work), to_f64(lse_full), f"period {period} lse", ulps=None, max_abs=2e-2, mean_rel=1e-3)
+        for t in range(P_):
+            kn = f32_to_dev_bf16((rng.standard_normal((B, H, d)) * 0.3 + 0.5).astype(np.float32))
+            vn = f32_to_dev_bf16(rng.standard_normal((B, H, d)).astype(np.float32))
+            o = torch.empty_like(q)
+            kb.keepkv_complete_append_host(p, Kh, Vh, lens_h, kn.cpu(), vn.cpu())
+            kb.keepkv_append(p, full_dev, kn, vn, st)                 # the device-resident twin, for the comparison
+            kb.keepkv_decode_step(p, work, q, kn, vn, o, None, True, ws, st)
+        torch.cuda.synchronize()
+    assert lens_h.tolist() == [400 + 2 * P_, 250 + 2 * P_] and int(st.item()) == 0
+    full = torch.tensor([n_cap, 10], dtype=torch.int32)
+    rc = kb.lib().keepkv_complete_append_host(__import__("ctypes").byref(p), Kh.data_ptr(), Vh.data_ptr(), full.data_ptr(),
+                                              Kh.data_ptr(), Vh.data_ptr())
+    assert rc == -3 and full.tolist() == [n_cap, 10]                  # a full sequence: refused, nothing advanced
