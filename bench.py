@@ -36,7 +36,8 @@ METRIC = "decode tokens/s + compress GB/s, fraction of HBM roofline"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the kernel the roofline entry times
 # (keepkv_decode_step in the steady state), per workload, from an ncu capture of that kernel as it stands now;
 # None where no capture of the current kernel exists
-DECODE_TRAFFIC_BYTES = {"C2": None}
+# (C2: mean of the two launches in profiles/decode_kernel_C2_steady.md)
+DECODE_TRAFFIC_BYTES = {"C2": 60_580_000}
 UNIT = "tokens/s"
 
 
@@ -184,7 +185,8 @@ def config_dict(w, args):
             "tokens": "layer-tokens: one token of one sequence attended in one layer cache (B * period * layers per step)",
             "layers_round_robin": args.layers,
             "l2": f"each call works on one of {args.layers} distinct layer caches visited round-robin "
-                  f"({args.layers} x {mb:.0f} MB > 126 MB L2)",
+                  f"({args.layers} x {mb:.0f} MB = {args.layers * mb:.0f} MB "
+                  f"{'>' if args.layers * mb > 126 else '<= (NOT larger than)'} 126 MB L2)",
             "parallelism": f"replicas x{args.gpus}"}
 
 
