@@ -240,6 +240,11 @@ def run_ours(args, w, rank, world):
     p_inc = kb.make_params(B=w.B, H_q=w.H_q, H_kv=w.H_kv, d=w.d, N_cap=n_cap, period=P, n_sink=w.n_sink,
                            n_recent=w.n_recent(), ema_alpha=0.9, merge_threshold=0.8,
                            flags=kb.FLAG_COMPRESS_STEADY if steady else 0)
+    # The decode steps of the loop visit the layer caches round-robin, so with two layers or more the kernel that
+    # precedes a step on the stream never writes the step's cache: the calls say so and start reading early.
+    p_step = kb.make_params(B=w.B, H_q=w.H_q, H_kv=w.H_kv, d=w.d, N_cap=n_cap, period=P, n_sink=w.n_sink,
+                            n_recent=w.n_recent(), ema_alpha=0.9, merge_threshold=0.8,
+                            flags=kb.FLAG_CACHE_IDLE if L >= 2 else 0)
     nrec_arg = torch.from_numpy(nrec).cuda() if ragged else None
     K0, V0 = dev(Kb).view(w.B, w.H_kv, n_cap, w.d), dev(Vb).view(w.B, w.H_kv, n_cap, w.d)
     del Kb, Vb
@@ -292,6 +297,19 @@ def run_ours(args, w, rank, world):
         e1.record(); stream.synchronize()
         t_full_decode = e0.elapsed_time(e1) * 1e-3 / L
         stats = torch.zeros(L, w.U, 8, dtype=torch.int32, device="cuda")
+        # ---- the prefill compression under the merge-first policy (Section 3.4), on copies of the scored prompt
+        #      caches (it works in place and the phases below need the prompt as it is); Bc serves as its scratch
+        n_mf = min(L, 2)
+        mf = [kb.Cache(A[l].K.clone(), A[l].V.clone(), A[l].votes.clone(), A[l].lscore.clone(), A[l].seq_len.clone())
+              for l in range(n_mf + 1)]
+        kb.keepkv_compress_merge_first(p, mf[n_mf], Bc[0], budget_arg, ws, st, n_recent_dev=nrec_arg)   # loads the kernels
+        stream.synchronize()
+        e0.record()
+        for l in range(n_mf):
+            kb.keepkv_compress_merge_first(p, mf[l], Bc[l], budget_arg, ws, st, n_recent_dev=nrec_arg)
+        e1.record(); stream.synchronize()
+        t_merge_first = e0.elapsed_time(e1) * 1e-3 / n_mf
+        del mf
         kb.keepkv_compress(p, A[0], Bc[0], budget_arg, ws, st, n_recent_dev=nrec_arg, stats=stats[0])   # loads the kernels
         stream.synchronize()
         e0.record()
@@ -306,7 +324,7 @@ def run_ours(args, w, rank, world):
             n = 0
             for t in range(P):
                 for l in range(L):
-                    kb.keepkv_decode_step(p, cur[l], q_all[t + 1], kn_all[t + 1], vn_all[t + 1], out, None, True, ws, st)
+                    kb.keepkv_decode_step(p_step, cur[l], q_all[t + 1], kn_all[t + 1], vn_all[t + 1], out, None, True, ws, st)
                     n += 1
             for l in range(L):
                 kb.keepkv_compress(p_inc, cur[l], oth[l], budget_arg, ws, st, n_recent_dev=nrec_arg,
@@ -349,14 +367,14 @@ def run_ours(args, w, rank, world):
         load_period()
         for t in range(P // 2):              # a real half period with fresh tokens
             for l in range(L):
-                kb.keepkv_decode_step(p, cur[l], q_all[t + 1], kn_all[t + 1], vn_all[t + 1], out, None, True, ws, st)
+                kb.keepkv_decode_step(p_step, cur[l], q_all[t + 1], kn_all[t + 1], vn_all[t + 1], out, None, True, ws, st)
         reps = 16
         gd = torch.cuda.CUDAGraph()
         stream.synchronize()
         with torch.cuda.graph(gd, stream=stream):
             for _ in range(reps):
                 for l in range(L):
-                    kb.keepkv_decode_step(p, cur[l], q_all[P // 2], kn_all[P // 2], vn_all[P // 2], out, None, True, ws, st)
+                    kb.keepkv_decode_step(p_step, cur[l], q_all[P // 2], kn_all[P // 2], vn_all[P // 2], out, None, True, ws, st)
         lens_keep = [c_.seq_len.clone() for c_ in cur]            # the launch the loop runs appends: put the lengths back
         gd.replay(); stream.synchronize()
         for c_, n_ in zip(cur, lens_keep):
@@ -368,7 +386,7 @@ def run_ours(args, w, rank, world):
         # ---- compression alone (incremental, budget + P -> budget), as a graph of the L calls
         for t in range(P // 2, P):
             for l in range(L):
-                kb.keepkv_decode_step(p, cur[l], q_all[t + 1], kn_all[t + 1], vn_all[t + 1], out, None, True, ws, st)
+                kb.keepkv_decode_step(p_step, cur[l], q_all[t + 1], kn_all[t + 1], vn_all[t + 1], out, None, True, ws, st)
         gc = torch.cuda.CUDAGraph()
         stream.synchronize()
         with torch.cuda.graph(gc, stream=stream):
@@ -423,7 +441,7 @@ def run_ours(args, w, rank, world):
             torch.cuda.synchronize()
             t0 = time.perf_counter()
             for t in range(P):
-                kb.keepkv_decode_step_host_layers(p, cur, qh_p[t], knh_p[t], vnh_p[t], oh, qd, kd, vd, od, True, ws, st)
+                kb.keepkv_decode_step_host_layers(p_step, cur, qh_p[t], knh_p[t], vnh_p[t], oh, qd, kd, vd, od, True, ws, st)
                 stream.synchronize()          # the next token's queries depend on this step's output
             for l in range(L):
                 kb.keepkv_compress(p_inc, cur[l], oth[l], budget_arg, ws, st, n_recent_dev=nrec_arg)
@@ -496,6 +514,7 @@ def run_ours(args, w, rank, world):
             "compress_full_frac_hbm": full_gbs / hbm, "merged_per_unit_full": m_full,
             "compress_full_gemm_tflops": gemm_flops / t_full_compress / 1e12,
             "compress_inplace_us": None if t_inplace is None else t_inplace * 1e6,
+            "compress_merge_first_us": t_merge_first * 1e6,
             "compress_inplace_note": "keepkv_compress_inplace on the same caches: rows touched = evicted + merged, not the whole cache",
         },
     }

@@ -85,6 +85,15 @@ typedef struct keepkv_params {
  * KEEPKV_DEV_NOT_STEADY is raised in *status_dev.  Needs budget > 0. */
 #define KEEPKV_FLAG_COMPRESS_STEADY 1
 
+/* keepkv_decode_attention, keepkv_decode_step and their host and static variants: the caller promises that the
+ * kernel which precedes this call on the stream (of this library or not) writes none of the arrays of `cache`
+ * (K, V, votes, lscore, seq_len) -- a model that calls once per layer, each layer with its own cache, knows this.
+ * The launch then reads the lengths and requests its first key / value tiles while that kernel is still
+ * finishing (programmatic dependent launch); the queries, the token to append, the workspace and every write wait
+ * for it as always, so results are bit-identical.  If the promise is broken (e.g. two consecutive calls on one
+ * cache) the call may attend to stale lengths, rows or scores; nothing faults.  Ignored by every other call. */
+#define KEEPKV_FLAG_CACHE_IDLE 2
+
 /* One layer's cache.  Rows [seq_len[b], N_cap) of a unit are unspecified. */
 typedef struct keepkv_cache {
   void *K;                  /* bf16 [B, H_kv, N_cap, d]  keys k_i              (16-byte aligned) */

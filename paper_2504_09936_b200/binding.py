@@ -36,6 +36,7 @@ class keepkv_cache(C.Structure):
 
 
 FLAG_COMPRESS_STEADY = 1   # keepkv_params.flags: the caller promises steady-state units, one kernel compresses them
+FLAG_CACHE_IDLE = 2        # decode calls: the preceding kernel of the stream does not write this cache
 DEV_APPEND_FULL, DEV_TIMEOUT, DEV_NOT_STEADY, DEV_POSITIONS = 1, 2, 4, 8   # bits of *status_dev
 
 STATS_FIELDS = ("n_retained", "n_evicted", "n_merged", "n_below_T", "n_guard_groups", "n_groups", "max_group",

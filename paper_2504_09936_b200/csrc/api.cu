@@ -49,7 +49,7 @@ WsLayout ws_layout(const keepkv_params &p) {
 static int validate(const keepkv_params *p) {
   if (!p) return KEEPKV_ERR_INVALID_ARG;
   if (p->B <= 0 || p->H_q <= 0 || p->H_kv <= 0 || p->N_cap <= 0) return KEEPKV_ERR_INVALID_ARG;
-  if ((p->flags & ~KEEPKV_FLAG_COMPRESS_STEADY) || p->reserved[0] || p->reserved[1]) return KEEPKV_ERR_INVALID_ARG;
+  if ((p->flags & ~(KEEPKV_FLAG_COMPRESS_STEADY | KEEPKV_FLAG_CACHE_IDLE)) || p->reserved[0] || p->reserved[1]) return KEEPKV_ERR_INVALID_ARG;
   if (p->H_q % p->H_kv) return KEEPKV_ERR_UNSUPPORTED;
   const int G = p->H_q / p->H_kv;
   if (!(G == 1 || G == 2 || G == 4 || G == 8)) return KEEPKV_ERR_UNSUPPORTED;

@@ -470,6 +470,75 @@ def test_decode_step_host_layers_matches_per_layer_calls():
     assert int(st.item()) == 0
 
 
+@pytest.mark.parametrize("B,H_kv,G,d,n_cap,base_len,graph", [
+    (8, 8, 4, 128, 2048, 1700, True),     # 64 units: one cluster of four per unit, the launches back to back in a graph
+    (6, 4, 4, 128, 256, 120, False),      # 24 units: clusters of eight, lengths that cross a tile edge
+    (3, 2, 8, 64, 640, 500, True),        # 6 units: no clusters, several CTAs per unit through the partial pool
+])
+def test_decode_step_with_cache_idle_flag_is_bit_identical(B, H_kv, G, d, n_cap, base_len, graph):
+    """KEEPKV_FLAG_CACHE_IDLE: three layer caches visited round-robin, so the launch before each call works on
+    another cache and the promise holds.  Caches, outputs and lse after several steps equal, bit for bit, those
+    of the same loop without the flag, and one unit per layer is compared with the oracle on the last step."""
+    Lr, steps = 3, 5
+    p0 = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=n_cap)
+    p1 = _copy_params(p0, flags=kb.FLAG_CACHE_IDLE)
+    lens = [[base_len + (5 * b + 11 * l) % 9 for b in range(B)] for l in range(Lr)]
+    base = [random_cache(p0, lens[l], seed=70 + l, vote_max=3, scored_frac=0.8) for l in range(Lr)]
+    clone = lambda c: kb.Cache(c.K.clone(), c.V.clone(), c.votes.clone(), c.lscore.clone(), c.seq_len.clone())
+    rng = np.random.default_rng(33)
+    mk = lambda *s: f32_to_dev_bf16(rng.standard_normal(s).astype(np.float32))
+    q, kn, vn = mk(steps, Lr, B, H_kv * G, d), mk(steps, Lr, B, H_kv, d), mk(steps, Lr, B, H_kv, d)
+    results = []
+    before_last = None
+    for p in (p0, p1):
+        caches = [clone(c) for c in base]
+        ws, st = kb.new_workspace(p), kb.new_status()
+        out = torch.zeros(steps, Lr, B, H_kv * G, d, dtype=torch.bfloat16, device="cuda")
+        lse = torch.zeros(steps, Lr, B, H_kv * G, dtype=torch.float32, device="cuda")
+
+        def run(t0, t1):
+            for t in range(t0, t1):
+                for l in range(Lr):
+                    kb.keepkv_decode_step(p, caches[l], q[t, l], kn[t, l], vn[t, l], out[t, l], lse[t, l], True, ws, st)
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            run(0, 1)                       # eager first (loads the kernel outside any capture)
+            if graph:
+                g = torch.cuda.CUDAGraph()
+                stream.synchronize()
+                with torch.cuda.graph(g, stream=stream):
+                    run(1, steps - 1)
+                g.replay()
+            else:
+                run(1, steps - 1)
+            stream.synchronize()
+            if p is p1:
+                before_last = []
+                for l in range(Lr):     # the oracle's input of the last step: the cache with the token appended
+                    c = clone(caches[l])
+                    kb.keepkv_append(p0, c, kn[steps - 1, l], vn[steps - 1, l], st)
+                    stream.synchronize()
+                    before_last.append(HostCache(c))
+            run(steps - 1, steps)
+            stream.synchronize()
+        assert int(st.item()) == 0
+        results.append((caches, out, lse))
+    (ca, oa, la), (cb, ob, lb) = results
+    assert torch.equal(oa.view(torch.int16), ob.view(torch.int16)) and torch.equal(la.view(torch.int32), lb.view(torch.int32))
+    for l in range(Lr):
+        assert torch.equal(ca[l].seq_len, cb[l].seq_len)
+        n = ca[l].seq_len.cpu().numpy()
+        for b in range(B):
+            k = int(n[b])
+            assert torch.equal(ca[l].K[b, :, :k].view(torch.int16), cb[l].K[b, :, :k].view(torch.int16)), (l, b)
+            assert torch.equal(ca[l].V[b, :, :k].view(torch.int16), cb[l].V[b, :, :k].view(torch.int16)), (l, b)
+            assert torch.equal(ca[l].votes[b, :, :k], cb[l].votes[b, :, :k]), (l, b)
+            assert torch.equal(ca[l].lscore[b, :, :k].view(torch.int32), cb[l].lscore[b, :, :k].view(torch.int32)), (l, b)
+        u = (2 * l + 1) % (B * H_kv)
+        check_decode_unit(p0, u, before_last[l], to_f64(q[steps - 1, l]), to_f64(ob[steps - 1, l]), to_f64(lb[steps - 1, l]),
+                          to_f64(cb[l].lscore).reshape(B * H_kv, -1), what=f"layer {l}")
+
+
 def test_decode_is_deterministic():
     p = kb.make_params(B=2, H_q=8, H_kv=2, d=128, N_cap=2048)
     cache = random_cache(p, [2048, 1500], seed=8, vote_max=3)

@@ -71,8 +71,10 @@ def test_flags_and_decode_step_arguments_are_checked_before_any_launch(lib):
     fake2 = kb.keepkv_cache(2560, 5120, 7680, 10240, 12800)
     sz = C.c_size_t()
     # unknown flag bits are rejected by every call that takes the parameters
-    bad = kb.make_params(B=1, H_q=8, H_kv=2, d=64, N_cap=576, period=32, flags=2)
+    bad = kb.make_params(B=1, H_q=8, H_kv=2, d=64, N_cap=576, period=32, flags=4)
     assert lib.keepkv_workspace_bytes(C.byref(bad), C.byref(sz)) == -1
+    idle = kb.make_params(B=1, H_q=8, H_kv=2, d=64, N_cap=576, period=32, flags=kb.FLAG_CACHE_IDLE)
+    assert lib.keepkv_workspace_bytes(C.byref(idle), C.byref(sz)) == 0
     # the steady-state promise needs something to keep
     st = kb.make_params(B=1, H_q=8, H_kv=2, d=64, N_cap=576, period=32, flags=kb.FLAG_COMPRESS_STEADY)
     assert lib.keepkv_workspace_bytes(C.byref(st), C.byref(sz)) == 0
