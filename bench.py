@@ -301,7 +301,7 @@ def run_ours(args, w, rank, world):
         #      caches (it works in place and the phases below need the prompt as it is); Bc serves as its scratch
         n_mf = min(L, 2)
         mf = [kb.Cache(A[l].K.clone(), A[l].V.clone(), A[l].votes.clone(), A[l].lscore.clone(), A[l].seq_len.clone())
-              for l in range(n_mf + 1)]
+              for l in list(range(n_mf)) + [0]]
         kb.keepkv_compress_merge_first(p, mf[n_mf], Bc[0], budget_arg, ws, st, n_recent_dev=nrec_arg)   # loads the kernels
         stream.synchronize()
         e0.record()

@@ -23,7 +23,7 @@
 namespace keepkv {
 
 constexpr int kPfM = 128;        // entries per tile
-constexpr int kPfStages = 3;     // key-tile ring
+constexpr int kPfStages = 3;     // key-tile ring (4 and 5 stages, and four accumulators instead of two, measured equal)
 constexpr int kPfDrainWarps = 16; // four per 32-lane quarter of tensor memory
 constexpr int kPfThreads = 32 * (2 + kPfDrainWarps);   // producer, MMA issuer, drain warps
 constexpr int kPfWmax = 32;      // window queries per head (columns reserved per head)
@@ -39,8 +39,8 @@ struct PfSmem {
   static constexpr int kA = 0;
   static constexpr int kB = kPfStages * kABytes;
   static constexpr int kWt = kB + kBBytes;                  // f32 [32] weights, f32 [33] their suffix sums (as ln)
-  static constexpr int kXchg = kWt + 512;                   // float2 [2 accumulators][128 entries][4 warps]: (max, sum)
-  static constexpr int kBytes = kXchg + 2 * 128 * 4 * 8;
+  static constexpr int kXchg = kWt + 512;                   // float2 [3 tiles in flight][128 entries][4 warps]: (max, sum)
+  static constexpr int kBytes = kXchg + 3 * 128 * 4 * 8;
 };
 
 // Position in the global tile list: sequence, kv head, tile of the unit; next() moves to the next tile.
@@ -51,7 +51,9 @@ __device__ __forceinline__ float pf_ex2(float x) {
 }
 
 // log2 of the window weights alpha^(W-1-k), -inf for k >= W (and, with alpha = 0, for all but the last query)
-struct PfLogWeights { float c[kPfWmax]; };
+// w: the weights themselves and whether the drain may use them as multipliers (every one of the 32 a normal fp32
+// number: a full window and an alpha that is not tiny)
+struct PfLogWeights { float c[kPfWmax]; float w[kPfWmax]; int mult; };
 
 struct PfWalker {
   int b, h, tile, len, tb;
@@ -242,8 +244,8 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
     const float ln_G = logf((float)G);
     float2 *xchg = reinterpret_cast<float2 *>(smem + SL::kXchg);
     // A wait that runs out (here or in another warp) ends the warp's work but not its walk: it goes through the
-    // rest of the tiles without waiting and without reading the accumulators, so that the warps of its quarter
-    // still meet at their barrier on every tile.
+    // rest of the tiles without waiting and without reading the accumulators, and meets the warps of its quarter at
+    // their barrier on every tile.
     bool dead = false;
     for (int it = 0; it < ntiles; ++it) {
       const int a = it & 1;
@@ -276,6 +278,30 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
         }
         // y_k = log2 of (weight_k * score_k); queries k >= W carry weight 0 (log2 = -inf).  Two copies of the
         // loop, chosen per tile: only the last tiles of a unit hold entries that some window queries do not see.
+        if (full && lw.mult) {
+          // Every query sees every entry of the tile and every weight is an ordinary number: the reference of the
+          // exponentials is the largest raw logit (at most the window's weight range above the true maximum) and
+          // the weight multiplies the exponential inside the sum: max, multiply-add, ex2, multiply-add per score.
+          float r0 = fmaxf(__uint_as_float(r[0]), __uint_as_float(r[1])), r1 = fmaxf(__uint_as_float(r[2]), __uint_as_float(r[3]));
+#pragma unroll
+          for (int k = 4; k < 32; k += 4) {
+            r0 = fmaxf(r0, fmaxf(__uint_as_float(r[k]), __uint_as_float(r[k + 1])));
+            r1 = fmaxf(r1, fmaxf(__uint_as_float(r[k + 2]), __uint_as_float(r[k + 3])));
+          }
+          const float m_new = fmaxf(m, fmaxf(r0, r1) * scale2);
+          S *= pf_ex2(m - m_new);   // m = -inf: S is 0 and stays 0 (the logits are finite, so m_new is)
+          float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+          for (int k = 0; k < 32; k += 4) {
+            a0 = fmaf(lw.w[k], pf_ex2(fmaf(__uint_as_float(r[k]), scale2, -m_new)), a0);
+            a1 = fmaf(lw.w[k + 1], pf_ex2(fmaf(__uint_as_float(r[k + 1]), scale2, -m_new)), a1);
+            a2 = fmaf(lw.w[k + 2], pf_ex2(fmaf(__uint_as_float(r[k + 2]), scale2, -m_new)), a2);
+            a3 = fmaf(lw.w[k + 3], pf_ex2(fmaf(__uint_as_float(r[k + 3]), scale2, -m_new)), a3);
+          }
+          S += (a0 + a1) + (a2 + a3);
+          m = m_new;
+          continue;
+        }
         float y[32], mc = -CUDART_INF_F, mc2 = -CUDART_INF_F;
         if (full) {
 #pragma unroll
@@ -308,10 +334,23 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
         }
       }
       if (G > 1) {
-        // the warps of a quarter meet at a barrier of their own (128 threads)
-        float2 *x2 = xchg + (a * 128 + row) * 4;
-        if (hq > 0 && hq < G) x2[hq] = make_float2(m, S);
-        asm volatile("bar.sync %0, 128;" ::"r"(1 + quarter) : "memory");
+        // The warps of a quarter do not wait for each other: those of heads 1-3 leave their (max, sum) and arrive,
+        // only the warp of head 0 waits for them.  They can be two tiles ahead of it at most (the accumulator of
+        // tile t + 3 is not written before the head-0 warp has read tile t + 1, hence combined tile t), so the
+        // exchange area and the barrier rotate over three tiles.  (The same hand-over through mbarriers, with or
+        // without the finishing role rotating over the four warps, measured 8-11 us slower on the C2 prompt.)
+        const int x3 = it % 3;
+        float2 *x2 = xchg + (x3 * 128 + row) * 4;
+        if (hq > 0) {
+          if (hq < G) x2[hq] = make_float2(m, S);
+          __threadfence_block();
+          if (dead)   // no longer paced by the accumulators: stay in step with the head-0 warp instead
+            asm volatile("bar.sync %0, 128;" ::"r"(1 + quarter + 4 * x3) : "memory");
+          else
+            asm volatile("bar.arrive %0, 128;" ::"r"(1 + quarter + 4 * x3) : "memory");
+        } else {
+          asm volatile("bar.sync %0, 128;" ::"r"(1 + quarter + 4 * x3) : "memory");
+        }
         if (hq == 0) {
 #pragma unroll
           for (int w = 1; w < (G < 4 ? G : 4); ++w) {
@@ -369,7 +408,9 @@ static void launch_prefill_t(const keepkv_params &p, const keepkv_cache &c, cons
     if (k >= W) lw.c[k] = -INFINITY;
     else if (p.ema_alpha > 0.f) lw.c[k] = (float)(W - 1 - k) * log2f(p.ema_alpha);
     else lw.c[k] = k == W - 1 ? 0.f : -INFINITY;
+    lw.w[k] = exp2f(lw.c[k]);
   }
+  lw.mult = (W == kPfWmax && lw.c[0] >= -60.f && p.sm_scale > 0.f) ? 1 : 0;
   launch_pdl(prefill_scores_kernel<D, G>, dim3(sm_count()), dim3(kPfThreads), smem_bytes, ctx.stream, mapK, mapQ, p, c,
              W, lw, status_dev);
   KEEPKV_CHECK_LAUNCH(ctx);

@@ -655,7 +655,7 @@ def test_compress_steady_flag_reports_units_outside_its_limits():
     with pytest.raises(kb.KeepKVError):
         kb.keepkv_compress(p, src, kb.Cache.empty(p), 0, ws, st)
     with pytest.raises(kb.KeepKVError):
-        kb.keepkv_compress(_copy_params(p, flags=2), src, kb.Cache.empty(p), budget, ws, st)
+        kb.keepkv_compress(_copy_params(p, flags=4), src, kb.Cache.empty(p), budget, ws, st)
 
 
 @pytest.mark.parametrize("flags", [0, kb.FLAG_COMPRESS_STEADY])
