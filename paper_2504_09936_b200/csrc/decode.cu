@@ -239,11 +239,15 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     TileDesc d;
     d.u = u; d.tile = ptile; d.len = plen;
     d.flags = ((it == 0 || ptile == 0) ? 1 : 0) | ((it == ntiles - 1 || ptile == ptb - 1) ? 2 : 0);
-    d.c_first = (int)(us / chunk);
-    d.nparts = (int)((ue - 1) / chunk) - d.c_first + 1;
     if (aligned) {   // every CTA of the cluster holds a partial (possibly empty) unless the unit is a single tile
       d.c_first = 0;
       d.nparts = ptb == 1 ? 1 : csize;
+    } else if (T < 0x7fffffffLL) {   // (64-bit divisions cost this one thread hundreds of cycles per tile)
+      d.c_first = (int)us / chunk;
+      d.nparts = ((int)ue - 1) / chunk - d.c_first + 1;
+    } else {
+      d.c_first = (int)(us / chunk);
+      d.nparts = (int)((ue - 1) / chunk) - d.c_first + 1;
     }
     d.u_next = -1;
     d.fresh = -1;
@@ -278,11 +282,8 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       return true;
     }
     mbar_expect_tx(bar, SL::kTxBytes);
-#pragma unroll
-    for (int sub = 0; sub < SL::kSub; ++sub) {
-      tma_load_2d(dst + SL::kK + sub * SL::kSubBytes, &mapK, sub * 64, row, bar);
-      tma_load_2d(dst + SL::kV + sub * SL::kSubBytes, &mapV, sub * 64, row, bar);
-    }
+    tma_load_3d(dst + SL::kK, &mapK, 0, row, 0, bar);   // both 64-channel halves of the tile in one copy
+    tma_load_3d(dst + SL::kV, &mapV, 0, row, 0, bar);
     bulk_load_1d(dst + SL::kVotes, c.votes + ubase + (size_t)this_tile * kTile, kTile * 4, bar);
     bulk_load_1d(dst + SL::kLscore, c.lscore + ubase + (size_t)this_tile * kTile, kTile * 4, bar);
     ++pit;
@@ -796,7 +797,7 @@ static bool cached_rows_map(CUtensorMap *out, void *base, uint64_t rows, int D) 
   std::lock_guard<std::mutex> lock(mu);
   for (int i = 0; i < used; ++i)
     if (keys[i].base == base && keys[i].rows == rows && keys[i].D == D) { *out = maps[i]; return true; }
-  if (!make_bf16_rows_map(out, base, rows, D, kTile)) return false;
+  if (!make_bf16_halves_map(out, base, rows, D, kTile)) return false;
   const int slot = used < N ? used++ : (next++ % N);
   keys[slot] = MapKey{base, rows, D};
   maps[slot] = *out;

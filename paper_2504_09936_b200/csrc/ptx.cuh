@@ -52,6 +52,12 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map
       "l"(map), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *map, int x, int y, int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar)
+      : "memory");
+}
 __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
                "l"(src), "r"(bytes), "r"(bar)
@@ -190,6 +196,20 @@ inline EncodeTiledFn tensormap_encode_fn() {
 
 // Tensor map over a row-major [rows, D] bf16 matrix with boxes of box_rows x 64 channels and the
 // 128-byte swizzle; rows past the end read as zero.
+// The same rows as a 3-D tensor (64 channels, rows, D / 64 halves of a row; the half is the slowest box dimension):
+// one copy delivers a whole tile as D / 64 consecutive 128-byte-swizzled sub-tiles of box_rows x 64 channels, the
+// layout two 2-D copies of the map below would produce.
+inline bool make_bf16_halves_map(CUtensorMap *map, void *base, uint64_t rows, int D, int box_rows) {
+  EncodeTiledFn fn = tensormap_encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {64, (cuuint64_t)rows, (cuuint64_t)(D / 64)};
+  cuuint64_t strides[2] = {(cuuint64_t)D * 2, 128};
+  cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)(D / 64)};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
 inline bool make_bf16_rows_map(CUtensorMap *map, void *base, uint64_t rows, int D, int box_rows) {
   EncodeTiledFn fn = tensormap_encode_fn();
   if (!fn) return false;
