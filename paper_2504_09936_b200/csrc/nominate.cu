@@ -11,9 +11,10 @@
 //               dst cache into a 2-stage ring;
 //   warp 1      one thread issues tcgen05.mma (M=128, N=256, K=16, bf16 -> fp32) into one of two
 //               256-column accumulators in tensor memory and commits to the ring / accumulator barriers;
-//   warps 2-9   gather the 128 evicted rows from the src cache into the swizzled A tile, then drain the
-//               accumulators with tcgen05.ld: two warps per 32-lane quarter, one per column half,
-//               scaling by the retained keys' inverse norms and tracking the row's top two.
+//   warps 2-17  gather the 128 evicted rows from the src cache into the swizzled A tile, then drain the
+//               accumulators with tcgen05.ld: four warps per 32-lane quarter, each 64 of a tile's 256 columns
+//               (the drain is a latency chain per warp: with two warps per quarter the issue slots were a third
+//               full), scaling by the retained keys' inverse norms and tracking the row's top two.
 // Every wait is bounded; a wait that runs out raises KEEPKV_DEV_TIMEOUT, the CTA stops issuing work,
 // drains what is in flight, frees its tensor memory and returns.
 #include <type_traits>
@@ -26,7 +27,8 @@ namespace keepkv {
 constexpr int kNomM = 128;        // evicted rows per item (tensor-memory lanes)
 constexpr int kNomN = 256;        // retained columns per tile
 constexpr int kNomStages = 2;     // B ring
-constexpr int kNomThreads = 320;  // 10 warps
+constexpr int kNomDrainWarps = 16; // four per 32-lane quarter of tensor memory, each a quarter of a tile's columns
+constexpr int kNomThreads = 32 * (2 + kNomDrainWarps);
 
 template <int D>
 struct NomSmem {
@@ -35,10 +37,10 @@ struct NomSmem {
   static constexpr int kBBytes = kSub * kNomN * 128;
   static constexpr int kA = 0;
   static constexpr int kB = 2 * kABytes;                  // two A tiles: the next item is gathered while this one is drained
-  static constexpr int kInv = kB + kNomStages * kBBytes;  // f32 [8 warps][128]   inverse norms of the warp's columns
-  static constexpr int kRowInv = kInv + 8 * 128 * 4;      // f32 [2][128]         inverse norms of the staged rows
-  static constexpr int kXchg = kRowInv + 2 * 128 * 4;     // u32 [2][128][5]      column-half exchange
-  static constexpr int kPrefix = kXchg + 2 * 128 * 5 * 4; // i32 [kMaxUnits + 1]  row-tile prefix over units
+  static constexpr int kInv = kB + kNomStages * kBBytes;  // f32 [16 warps][64]   inverse norms of the warp's columns
+  static constexpr int kRowInv = kInv + 16 * 64 * 4;      // f32 [2][128]         inverse norms of the staged rows
+  static constexpr int kXchg = kRowInv + 2 * 128 * 4;     // u32 [2][128][3][3]   exchange between the column quarters
+  static constexpr int kPrefix = kXchg + 2 * 128 * 9 * 4; // i32 [kMaxUnits + 1]  row-tile prefix over units
   static constexpr int kBytes = kPrefix + (kMaxUnits + 1) * 4;
 };
 
@@ -92,11 +94,11 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
 
   if (tid == 0) {
     for (int i = 0; i < 2; ++i) {
-      mbar_init(bar_a_ready + 8 * i, 8);
+      mbar_init(bar_a_ready + 8 * i, kNomDrainWarps);
       mbar_init(bar_b_full + 8 * i, 1);
       mbar_init(bar_b_empty + 8 * i, 1);
       mbar_init(bar_t_full + 8 * i, 1);
-      mbar_init(bar_t_empty + 8 * i, 8);
+      mbar_init(bar_t_empty + 8 * i, kNomDrainWarps);
     }
     mbar_init(bar_drain, 1);
     s_abort = 0;
@@ -199,18 +201,18 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
     }
   } else {
     // ------------------------------------------------------------ A staging + accumulator drain
-    const int ew = warp - 2, quarter = warp & 3, half = ew >> 2;
+    const int ew = warp - 2, quarter = warp & 3, cq = ew >> 2;   // cq: which 64 columns of a tile
     const int row = quarter * 32 + lane;                        // tensor-memory lane = row of the item
-    float *inv_w = reinterpret_cast<float *>(smem + SL::kInv) + ew * 128;
+    float *inv_w = reinterpret_cast<float *>(smem + SL::kInv) + ew * 64;
     float *rowinv = reinterpret_cast<float *>(smem + SL::kRowInv);
     uint32_t *xchg = reinterpret_cast<uint32_t *>(smem + SL::kXchg);
     const size_t n_total = (size_t)U * p.N_cap;
     int acc = 0, n_done = 0;
     bool dead = false, staged = false;
-    // Gathers the 128 evicted rows of an item into swizzled A tile `abuf`, sixteen lanes per row, and
+    // Gathers the 128 evicted rows of an item into swizzled A tile `abuf`, sixteen lanes per row (32 rows per round), and
     // leaves the rows' inverse norms in rowinv[abuf].
     auto stage_rows = [&](const NomItem &si, int abuf) {
-      constexpr int REPS = kNomM / 16;
+      constexpr int REPS = kNomM / 32;
       const size_t sbase_u = (size_t)si.u * p.N_cap;
       const int sm0 = si.m_tile * kNomM;
       const int ch = lane & 15, rsub = ew * 2 + (lane >> 4);
@@ -218,7 +220,7 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
       uint4 val[REPS];
 #pragma unroll
       for (int rep = 0; rep < REPS; ++rep) {
-        const int r = rep * 16 + rsub;
+        const int r = rep * 32 + rsub;
         esrc[rep] = (ch < D / 8 && sm0 + r < si.n_ev) ? ev_idx[sbase_u + sm0 + r] : -1;
       }
 #pragma unroll
@@ -228,7 +230,7 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
       }
 #pragma unroll
       for (int rep = 0; rep < REPS; ++rep) {
-        const int r = rep * 16 + rsub;
+        const int r = rep * 32 + rsub;
         float ss = 0.f;
         const uint32_t w[4] = {val[rep].x, val[rep].y, val[rep].z, val[rep].w};
 #pragma unroll
@@ -254,7 +256,7 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
       Top2 top, topb;   // two trackers over alternate groups of four columns: two independent dependency chains
       top.init(0.f);
       if (it.t0 == it.t1) {   // a chunk without tiles (fewer tiles than chunks): publish an empty result
-        if (half == 0 && m0 + row < it.n_ev) {
+        if (cq == 0 && m0 + row < it.n_ev) {
           const size_t o = (ubase + m0 + row) * C_max + it.chunk;
           nom_v[o] = make_float4(top.best, top.second, 0.f, __int_as_float(-1));
           nom_si[o] = -1;
@@ -269,7 +271,7 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
         }
         // rowinv of this item is visible to every warp, and nobody still reads the other buffer's
         // rowinv (the previous item's results have been published)
-        asm volatile("bar.sync 1, 256;" ::: "memory");
+        asm volatile("bar.sync 1, 512;" ::: "memory");
         // gather the next item's rows into the other A tile now, so that its MMAs can start while this
         // item is drained (the MMAs that last read that tile belong to the item before this one: retired)
         {
@@ -287,13 +289,13 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
 
         for (int t = it.t0; t < it.t1; ++t, ++acc) {
           const int a = acc & 1;
-          const int c0 = t * kNomN + half * 128;
+          const int c0 = t * kNomN + cq * 64;
           {
             const size_t g = ubase + c0 + 4 * lane;
             float4 iv = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (g + 3 < n_total) iv = *reinterpret_cast<const float4 *>(inv_norm + g);
+            if (lane < 16 && g + 3 < n_total) iv = *reinterpret_cast<const float4 *>(inv_norm + g);
             __syncwarp();
-            *reinterpret_cast<float4 *>(inv_w + 4 * lane) = iv;
+            if (lane < 16) *reinterpret_cast<float4 *>(inv_w + 4 * lane) = iv;
             __syncwarp();
           }
           if (!dead) {
@@ -310,23 +312,22 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
           }
           if (!dead && live) {
             tc_fence_after();
-            const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + a * kNomN + half * 128;
-            const int n_valid = it.n_ret - c0;   // columns of this half that exist
+            const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + a * kNomN + cq * 64;
+            const int n_valid = it.n_ret - c0;   // columns of this quarter that exist
             // rows and columns are the same entries (self_mask): the column of the row's own key does not count
             const int diag = self_mask ? m0 + row - c0 : -1;
-            const bool crosses = self_mask && m0 + quarter * 32 < c0 + 128 && c0 <= m0 + quarter * 32 + 31;
+            const bool crosses = self_mask && m0 + quarter * 32 < c0 + 64 && c0 <= m0 + quarter * 32 + 31;
 #pragma unroll 1
-            for (int jg = 0; jg < 2; ++jg) {
-              uint32_t r0[32], r1[32];
-              tmem_ld_32x32(taddr + jg * 64, r0);
-              tmem_ld_32x32(taddr + jg * 64 + 32, r1);
+            for (int jg = 0; jg < 2; ++jg) {   // 32 columns at a time: the register budget of 18 warps
+              uint32_t r0[32];
+              tmem_ld_32x32(taddr + jg * 32, r0);
               tmem_ld_wait();
               if (jg == 1) {   // everything this warp needs from the accumulator is in registers
                 tc_fence_before();
                 if (lane == 0) mbar_arrive(bar_t_empty + 8 * a);
               }
-              const int cb = jg * 64;
-              const bool ragged = n_valid < cb + 64 || crosses;   // columns past n_ret hold other rows' data
+              const int cb = jg * 32;
+              const bool ragged = n_valid < cb + 32 || crosses;   // columns past n_ret hold other rows' data
               // `masked` is a compile-time flag: only the last tile of a row of tiles has columns to mask, and a
               // run-time test inside the unrolled loop would be turned into selects that every group pays for
               auto drain32 = [&](auto test, auto masked, const uint32_t (&r)[32], int off) {
@@ -347,16 +348,12 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
               const bool cold = t == it.t0;   // cold lists: insert everything
               if (cold && ragged) {
                 drain32(std::false_type{}, std::true_type{}, r0, cb);
-                drain32(std::false_type{}, std::true_type{}, r1, cb + 32);
               } else if (cold) {
                 drain32(std::false_type{}, std::false_type{}, r0, cb);
-                drain32(std::false_type{}, std::false_type{}, r1, cb + 32);
               } else if (ragged) {
                 drain32(std::true_type{}, std::true_type{}, r0, cb);
-                drain32(std::true_type{}, std::true_type{}, r1, cb + 32);
               } else {
                 drain32(std::true_type{}, std::false_type{}, r0, cb);
-                drain32(std::true_type{}, std::false_type{}, r1, cb + 32);
               }
               if (cold && jg == 1) top.cut = fmaxf(top.best, topb.best) - top.thr;
             }
@@ -367,15 +364,22 @@ nominate_kernel(const __grid_constant__ CUtensorMap mapB, keepkv_params p, const
       top.insert_any(topb.best, topb.bi);
       top.insert_any(topb.second, topb.si);
       // ---- combine the two column halves of each row and publish the chunk's result
-      uint32_t *x = xchg + (size_t)(buf * 128 + row) * 5;
-      if (half == 1) {
-        x[0] = __float_as_uint(top.best); x[1] = (uint32_t)top.bi; x[2] = __float_as_uint(top.second);
-        x[3] = (uint32_t)top.si;
+      uint32_t *x = xchg + (size_t)(buf * 128 + row) * 9;
+      if (cq > 0) {   // slots are below 65535 (N_cap <= 49152); -1 = none
+        uint32_t *xw = x + (cq - 1) * 3;
+        xw[0] = __float_as_uint(top.best);
+        xw[1] = __float_as_uint(top.second);
+        xw[2] = (uint32_t)(top.bi + 1) | ((uint32_t)(top.si + 1) << 16);
       }
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      if (half == 0) {
-        top.insert(__uint_as_float(x[0]), (int)x[1]);   // the upper half holds higher slots: ties keep the lower half
-        top.insert(__uint_as_float(x[2]), (int)x[3]);
+      asm volatile("bar.sync 1, 512;" ::: "memory");
+      if (cq == 0) {
+#pragma unroll
+        for (int w = 0; w < 3; ++w) {   // ascending columns: a later quarter holds higher slots, ties keep the earlier one
+          const uint32_t *xw = x + w * 3;
+          const uint32_t sl = xw[2];
+          top.insert(__uint_as_float(xw[0]), (int)(sl & 0xffffu) - 1);
+          top.insert(__uint_as_float(xw[1]), (int)(sl >> 16) - 1);
+        }
         if (m0 + row < it.n_ev) {
           const float ri = rowinv[buf * 128 + row];
           const size_t o = (ubase + m0 + row) * C_max + it.chunk;
