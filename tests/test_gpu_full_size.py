@@ -363,3 +363,81 @@ def test_c5_stated_shape_sampled_units():
     lens = W.seq_lens(w, 0)
     b_long, b_short = int(np.argmax(lens)), int(np.argmin(lens))
     assert _protocol_at_stated_shape("C5", [b_long * 8 + 3, b_short * 8 + 6]) is True
+
+
+def test_c2_period_as_the_benchmark_launches_it():
+    """Workload C2 in the launch configuration bench.py times: three layer caches of the full shape visited
+    round-robin, keepkv_decode_step with KEEPKV_FLAG_CACHE_IDLE replayed from a CUDA graph, then the single-kernel
+    steady-state compression.  After 24 steps the caches and outputs equal, bit for bit, those of the unflagged
+    append + attention calls on twin caches; the last step of every layer is compared with the oracle on sampled
+    units, and so is the compression that follows."""
+    w = W.CONFIGS["C2"]
+    Lr, steps = 3, 24
+    p = workload_params(w)
+    p_idle = workload_params(w, flags=kb.FLAG_CACHE_IDLE)
+    p_inc = workload_params(w, flags=kb.FLAG_COMPRESS_STEADY)
+    b = w.budget()
+    units = [5, 38]
+    ws, st = kb.new_workspace(p), kb.new_status()
+    clone = lambda c: kb.Cache(c.K.clone(), c.V.clone(), c.votes.clone(), c.lscore.clone(), c.seq_len.clone())
+    # per layer: prompt of its own seed, scored by one step, compressed to the budget
+    layers = []
+    for l in range(Lr):
+        prompt = workload_cache(w, n_cap=p.N_cap, layer=l)
+        q0 = bits_to_dev(W.make_step_inputs(w, l, 0, 1)[0][0])
+        o0 = torch.empty(w.B, w.H_q, w.d, dtype=torch.bfloat16, device="cuda")
+        kb.keepkv_decode_attention(p, prompt, q0, o0, None, True, ws, st)
+        dst = kb.Cache.empty(p)
+        kb.keepkv_compress(p, prompt, dst, b, ws, st)
+        torch.cuda.synchronize()
+        layers.append(dst)
+        del prompt
+    twins = [clone(c) for c in layers]
+    ins = [W.make_step_inputs(w, l, 1, steps + 1) for l in range(Lr)]
+    q = [[bits_to_dev(ins[l][0][t]) for l in range(Lr)] for t in range(steps)]
+    kn = [[bits_to_dev(ins[l][1][t]) for l in range(Lr)] for t in range(steps)]
+    vn = [[bits_to_dev(ins[l][2][t]) for l in range(Lr)] for t in range(steps)]
+    out = torch.zeros(steps, Lr, w.B, w.H_q, w.d, dtype=torch.bfloat16, device="cuda")
+    lse = torch.zeros(steps, Lr, w.B, w.H_q, dtype=torch.float32, device="cuda")
+    out2, lse2 = torch.zeros_like(out), torch.zeros_like(lse)
+
+    def run(t0, t1):
+        for t in range(t0, t1):
+            for l in range(Lr):
+                kb.keepkv_decode_step(p_idle, layers[l], q[t][l], kn[t][l], vn[t][l], out[t, l], lse[t, l], True, ws, st)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        run(0, 1)
+        g = torch.cuda.CUDAGraph()
+        stream.synchronize()
+        with torch.cuda.graph(g, stream=stream):
+            run(1, steps - 1)
+        g.replay()
+        stream.synchronize()
+        before = [UnitView(c, units) for c in layers]
+        run(steps - 1, steps)
+        stream.synchronize()
+    for t in range(steps):
+        for l in range(Lr):
+            kb.keepkv_append(p, twins[l], kn[t][l], vn[t][l], st)
+            kb.keepkv_decode_attention(p, twins[l], q[t][l], out2[t, l], lse2[t, l], True, ws, st)
+    torch.cuda.synchronize()
+    assert int(st.item()) == 0
+    assert torch.equal(out.view(torch.int16), out2.view(torch.int16)) and torch.equal(lse.view(torch.int32), lse2.view(torch.int32))
+    n = b + steps
+    for l in range(Lr):
+        assert layers[l].seq_len.cpu().tolist() == [n] * w.B == twins[l].seq_len.cpu().tolist()
+        assert torch.equal(layers[l].K[:, :, :n].view(torch.int16), twins[l].K[:, :, :n].view(torch.int16))
+        assert torch.equal(layers[l].V[:, :, :n].view(torch.int16), twins[l].V[:, :, :n].view(torch.int16))
+        assert torch.equal(layers[l].votes[:, :, :n], twins[l].votes[:, :, :n])
+        assert torch.equal(layers[l].lscore[:, :, :n].view(torch.int32), twins[l].lscore[:, :, :n].view(torch.int32))
+        seen = _with_fresh_row(before[l], units, to_f64(kn[steps - 1][l]), to_f64(vn[steps - 1][l]), w.H_kv)
+        _check_decode(p, seen, units, q[steps - 1][l], out[steps - 1, l], layers[l].lscore, f"C2 layer {l} last step",
+                      lse=lse[steps - 1, l])
+    # the steady-state compression of one layer, one kernel
+    src = UnitView(layers[0], units)
+    dst, ret, tgt, stats = _compress(p_inc, layers[0], b)
+    dview = UnitView(dst, units)
+    for u in units:
+        check_compress_unit(p, u, b, p.n_recent, src, dview, ret, tgt, stats, what="C2 steady compress after 24 steps",
+                            max_tolerated=8)
