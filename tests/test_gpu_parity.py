@@ -539,6 +539,46 @@ def test_decode_step_with_cache_idle_flag_is_bit_identical(B, H_kv, G, d, n_cap,
                           to_f64(cb[l].lscore).reshape(B * H_kv, -1), what=f"layer {l}")
 
 
+def test_cache_idle_flag_on_empty_full_and_ragged_sequences():
+    """The idle-cache variant on the shapes that take the less common paths: an empty sequence, one at capacity
+    (its token is dropped and reported), very ragged lengths (no cluster split), attention without an append.
+    Two caches alternate so that the promise holds; everything equals the unflagged calls bit for bit."""
+    B, H_kv, G, d, n_cap = 5, 2, 4, 128, 320
+    p0 = kb.make_params(B=B, H_q=H_kv * G, H_kv=H_kv, d=d, N_cap=n_cap)
+    p1 = _copy_params(p0, flags=kb.FLAG_CACHE_IDLE)
+    lens = [[0, 320, 7, 300, 64], [129, 0, 320, 1, 191]]
+    base = [random_cache(p0, lens[l], seed=90 + l, vote_max=2, scored_frac=0.5) for l in range(2)]
+    clone = lambda c: kb.Cache(c.K.clone(), c.V.clone(), c.votes.clone(), c.lscore.clone(), c.seq_len.clone())
+    rng = np.random.default_rng(44)
+    mk = lambda *s: f32_to_dev_bf16(rng.standard_normal(s).astype(np.float32))
+    steps = 3
+    q, kn, vn = mk(steps, 2, B, H_kv * G, d), mk(steps, 2, B, H_kv, d), mk(steps, 2, B, H_kv, d)
+    res = []
+    for p in (p0, p1):
+        caches = [clone(c) for c in base]
+        ws, st = kb.new_workspace(p), kb.new_status()
+        out = torch.zeros(2 * steps, 2, B, H_kv * G, d, dtype=torch.bfloat16, device="cuda")
+        lse = torch.zeros(2 * steps, 2, B, H_kv * G, dtype=torch.float32, device="cuda")
+        for t in range(steps):
+            for l in range(2):
+                kb.keepkv_decode_step(p, caches[l], q[t, l], kn[t, l], vn[t, l], out[2 * t, l], lse[2 * t, l], True, ws, st)
+            for l in range(2):
+                kb.keepkv_decode_attention(p, caches[l], q[t, l], out[2 * t + 1, l], lse[2 * t + 1, l], t % 2 == 0, ws, st)
+        torch.cuda.synchronize()
+        res.append((caches, out, lse, int(st.item())))
+    (ca, oa, la, sa), (cb, ob, lb, sb) = res
+    assert sa == sb == kb.DEV_APPEND_FULL
+    assert torch.equal(oa.view(torch.int16), ob.view(torch.int16)) and torch.equal(la.view(torch.int32), lb.view(torch.int32))
+    for l in range(2):
+        assert torch.equal(ca[l].seq_len, cb[l].seq_len)
+        n = ca[l].seq_len.cpu().numpy()
+        for b in range(B):
+            k = int(n[b])
+            assert torch.equal(ca[l].K[b, :, :k].view(torch.int16), cb[l].K[b, :, :k].view(torch.int16)), (l, b)
+            assert torch.equal(ca[l].votes[b, :, :k], cb[l].votes[b, :, :k]), (l, b)
+            assert torch.equal(ca[l].lscore[b, :, :k].view(torch.int32), cb[l].lscore[b, :, :k].view(torch.int32)), (l, b)
+
+
 def test_decode_is_deterministic():
     p = kb.make_params(B=2, H_q=8, H_kv=2, d=128, N_cap=2048)
     cache = random_cache(p, [2048, 1500], seed=8, vote_max=3)
