@@ -829,13 +829,15 @@ static void launch_t(const keepkv_params &p, const keepkv_cache &c, const void *
   if (grid > kDecMaxCtas) grid = kDecMaxCtas;
   // Two dozen units to one per SM: one cluster per unit, with as many CTAs per cluster (8, 4 or 2) as two per SM
   // allow -- provided all clusters are resident at once and at least 0.6 of the CTA slots are used (16 units
-  // x 8 = 128 CTAs ran 17.3 us where the equal ranges over the whole list took 15.9 us).
+  // x 8 = 128 CTAs ran 17.3 us where the equal ranges over the whole list took 15.9 us).  The idle-cache variant
+  // takes clusters from 0.2 of the slots on: the slots a small launch leaves free are where the next launch's CTAs
+  // start reading (16 units x 8: 13.3 us against 15.4 us; 8 short units x 8: 8.1 against 11.8 us).
   const int U = p.B * p.H_kv;
   int cs = 1;
   if (2 * U <= grid && p.N_cap / kTile >= 2) {
     static int max_clusters_dev[64][4] = {};   // per device and log2(cluster size); 0 = not asked yet, -1 = none
     for (int c = 8; c > 1 && cs == 1; c >>= 1) {
-      if ((long long)U * c > grid || 5LL * U * c < 3 * grid) continue;
+      if ((long long)U * c > grid || (E ? 5LL * U * c < 1 * grid : 5LL * U * c < 3 * grid)) continue;
       if (c == 8 && 4LL * U * c > 3 * grid) continue;   // 32 clusters of 8 are all resident, yet ran 16.7 us against 14.2 us
       const int li = c == 8 ? 3 : (c == 4 ? 2 : 1);
       int &mc = max_clusters_dev[dev & 63][li];
