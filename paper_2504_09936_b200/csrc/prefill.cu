@@ -23,7 +23,6 @@
 namespace keepkv {
 
 constexpr int kPfM = 128;        // entries per tile
-constexpr int kPfStages = 3;     // key-tile ring (4 and 5 stages, and four accumulators instead of two, measured equal)
 constexpr int kPfDrainWarps = 16; // four per 32-lane quarter of tensor memory
 constexpr int kPfThreads = 32 * (2 + kPfDrainWarps);   // producer, MMA issuer, drain warps
 constexpr int kPfWmax = 32;      // window queries per head (columns reserved per head)
@@ -34,13 +33,18 @@ template <int D, int G>
 struct PfSmem {
   static constexpr int kSub = D / 64;
   static constexpr int kNB = G * kPfWmax;                   // columns of the accumulator
-  static constexpr int kABytes = kSub * kPfM * 128;
+  // Producer, MMA issuer and drain hand a tile over in about a microsecond whatever its size, so up to G = 4 (where
+  // four accumulators fit the 512 columns of tensor memory) a hand-over is a pair of 128-entry tiles.
+  static constexpr int kTP = G <= 4 ? 2 : 1;                // 128-entry tiles per hand-over
+  static constexpr int kRows = kPfM * kTP;                  // entries per hand-over
+  static constexpr int kStages = kTP == 2 ? 2 : 3;          // key ring
+  static constexpr int kABytes = kSub * kRows * 128;
   static constexpr int kBBytes = kSub * kNB * 128;
   static constexpr int kA = 0;
-  static constexpr int kB = kPfStages * kABytes;
+  static constexpr int kB = kStages * kABytes;
   static constexpr int kWt = kB + kBBytes;                  // f32 [32] weights, f32 [33] their suffix sums (as ln)
-  static constexpr int kXchg = kWt + 512;                   // float2 [3 tiles in flight][128 entries][4 warps]: (max, sum)
-  static constexpr int kBytes = kXchg + 3 * 128 * 4 * 8;
+  static constexpr int kXchg = kWt + 512;                   // float2 [3 hand-overs in flight][kRows entries][4 warps]: (max, sum)
+  static constexpr int kBytes = kXchg + 3 * kRows * 4 * 8;
 };
 
 // Position in the global tile list: sequence, kv head, tile of the unit; next() moves to the next tile.
@@ -56,10 +60,10 @@ __device__ __forceinline__ float pf_ex2(float x) {
 struct PfLogWeights { float c[kPfWmax]; float w[kPfWmax]; int mult; };
 
 struct PfWalker {
-  int b, h, tile, len, tb;
+  int b, h, tile, len, tb, rows;   // rows: entries per tile of the list (a hand-over)
   __device__ __forceinline__ void load(const keepkv_params &p, const int32_t *seq_len) {
     len = max(0, min(seq_len[b], p.N_cap));
-    tb = (len + kPfM - 1) / kPfM;
+    tb = (len + rows - 1) / rows;
   }
   __device__ __forceinline__ void next(const keepkv_params &p, const int32_t *seq_len, bool more) {
     if (++tile == tb && more) {
@@ -77,10 +81,10 @@ __global__ void __launch_bounds__(kPfThreads, 1)
 prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapQ,
                       keepkv_params p, keepkv_cache c, int W, const PfLogWeights lw, int32_t *status_dev) {
   using SL = PfSmem<D, G>;
-  constexpr int KSTEPS = D / 16, NB = SL::kNB;
+  constexpr int KSTEPS = D / 16, NB = SL::kNB, TP = SL::kTP, ROWS = SL::kRows, kPfStages = SL::kStages;
   constexpr uint32_t IDESC = umma_idesc_bf16(kPfM, NB);
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * kPfStages + 7];   // a_full[S], a_empty[S], b_full, b_empty, t_full[2], t_empty[2], drain
+  __shared__ __align__(8) uint64_t bars[2 * 3 + 7];   // a_full[S], a_empty[S], b_full, b_empty, t_full[2], t_empty[2], drain
   __shared__ uint32_t s_tmem;
   __shared__ int s_scan[kPfThreads / 32];
   __shared__ int s_start[4];
@@ -137,7 +141,7 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
   pdl_trigger();
 
   // ---- the tile list: every thread sums a block of consecutive sequences, a block scan gives the offsets
-  auto tiles_of = [&](int b) { return (max(0, min(c.seq_len[b], p.N_cap)) + kPfM - 1) / kPfM; };
+  auto tiles_of = [&](int b) { return (max(0, min(c.seq_len[b], p.N_cap)) + ROWS - 1) / ROWS; };
   const int per = (p.B + kPfThreads - 1) / kPfThreads;
   const int b_lo = min(p.B, tid * per), b_hi = min(p.B, b_lo + per);
   int mine = 0;
@@ -177,7 +181,7 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
   __syncthreads();
   const uint32_t tmem = s_tmem;
   PfWalker wk;
-  wk.b = s_start[0]; wk.h = s_start[1]; wk.tile = s_start[2]; wk.len = 0; wk.tb = 1;
+  wk.b = s_start[0]; wk.h = s_start[1]; wk.tile = s_start[2]; wk.len = 0; wk.tb = 1; wk.rows = ROWS;
   if (ntiles > 0) wk.load(p, c.seq_len);
 
   if (warp == 0) {
@@ -202,8 +206,8 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
         mbar_expect_tx(bar_a_full + 8 * s, SL::kABytes);
 #pragma unroll
         for (int sub = 0; sub < SL::kSub; ++sub)
-          tma_load_2d(sbase + SL::kA + s * SL::kABytes + sub * (kPfM * 128), &mapK, sub * 64,
-                      u * p.N_cap + wk.tile * kPfM, bar_a_full + 8 * s);
+          tma_load_2d(sbase + SL::kA + s * SL::kABytes + sub * (ROWS * 128), &mapK, sub * 64,
+                      u * p.N_cap + wk.tile * ROWS, bar_a_full + 8 * s);
         wk.next(p, c.seq_len, it + 1 < ntiles);
       }
     }
@@ -222,10 +226,13 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
         tc_fence_after();
         const uint32_t a_base = sbase + SL::kA + s * SL::kABytes, b_base = sbase + SL::kB;
 #pragma unroll
-        for (int k = 0; k < KSTEPS; ++k) {
-          const uint64_t ad = umma_desc_sw128(a_base + (k >> 2) * (kPfM * 128) + (k & 3) * 32);
-          const uint64_t bd = umma_desc_sw128(b_base + (k >> 2) * (NB * 128) + (k & 3) * 32);
-          umma_bf16(tmem + a * NB, ad, bd, IDESC, k > 0 ? 1u : 0u);
+        for (int hf = 0; hf < TP; ++hf) {   // the 128-entry tiles of the hand-over, each into its own columns
+#pragma unroll
+          for (int k = 0; k < KSTEPS; ++k) {
+            const uint64_t ad = umma_desc_sw128(a_base + (k >> 2) * (ROWS * 128) + hf * (kPfM * 128) + (k & 3) * 32);
+            const uint64_t bd = umma_desc_sw128(b_base + (k >> 2) * (NB * 128) + (k & 3) * 32);
+            umma_bf16(tmem + (a * TP + hf) * NB, ad, bd, IDESC, k > 0 ? 1u : 0u);
+          }
         }
         umma_commit(bar_a_empty + 8 * s);
         umma_commit(bar_t_full + 8 * a);
@@ -256,22 +263,25 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
       }
       tc_fence_after();
       const int row = quarter * 32 + lane;
-      const int i = wk.tile * kPfM + row;                         // this thread's entry
-      const int klo = min(32, max(0, i - wk.len + W));            // first window query that sees it
-      const bool full = wk.tile * kPfM + kPfM - 1 - wk.len + W <= 0;   // the whole tile is seen by every query
-      const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + a * NB;
-      float m = -CUDART_INF_F, S = 0.f;
+      float mH[TP], SH[TP];   // (max, sum) of this thread's entry in each 128-entry tile of the hand-over
       if (g_last < 0 || dead) {   // no head for this warp (or no data any more): the accumulator is not its business
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_t_empty + 8 * a);
       }
+#pragma unroll
+      for (int hf = 0; hf < TP; ++hf) {
+      const int i = wk.tile * ROWS + hf * kPfM + row;             // this thread's entry
+      const int klo = min(32, max(0, i - wk.len + W));            // first window query that sees it
+      const bool full = wk.tile * ROWS + hf * kPfM + kPfM - 1 - wk.len + W <= 0;   // every query sees the whole tile
+      const uint32_t taddr = tmem + ((uint32_t)(quarter * 32) << 16) + (a * TP + hf) * NB;
+      float m = -CUDART_INF_F, S = 0.f;
 #pragma unroll 1
       for (int g = dead ? G : hq; g < G; g += 4) {
         uint32_t r[32];
         tmem_ld_32x32(taddr + g * 32, r);
         tmem_ld_wait();
-        if (g == g_last) {   // this warp's part of the accumulator is in registers: hand it back
+        if (g == g_last && hf == TP - 1) {   // this warp's part of the accumulators is in registers: hand them back
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(bar_t_empty + 8 * a);
@@ -333,6 +343,8 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
           m = m_new;
         }
       }
+      mH[hf] = m; SH[hf] = S;
+      }
       if (G > 1) {
         // The warps of a quarter do not wait for each other: those of heads 1-3 leave their (max, sum) and arrive,
         // only the warp of head 0 waits for them.  They can be two tiles ahead of it at most (the accumulator of
@@ -340,9 +352,12 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
         // exchange area and the barrier rotate over three tiles.  (The same hand-over through mbarriers, with or
         // without the finishing role rotating over the four warps, measured 8-11 us slower on the C2 prompt.)
         const int x3 = it % 3;
-        float2 *x2 = xchg + (x3 * 128 + row) * 4;
+        float2 *x2 = xchg + (x3 * ROWS + row) * 4;   // the entry of tile hf: x2 + hf * 128 * 4
         if (hq > 0) {
-          if (hq < G) x2[hq] = make_float2(m, S);
+          if (hq < G) {
+#pragma unroll
+            for (int hf = 0; hf < TP; ++hf) x2[hf * kPfM * 4 + hq] = make_float2(mH[hf], SH[hf]);
+          }
           __threadfence_block();
           if (dead)   // no longer paced by the accumulators: stay in step with the head-0 warp instead
             asm volatile("bar.sync %0, 128;" ::"r"(1 + quarter + 4 * x3) : "memory");
@@ -353,16 +368,29 @@ prefill_scores_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_con
         }
         if (hq == 0) {
 #pragma unroll
-          for (int w = 1; w < (G < 4 ? G : 4); ++w) {
-            const float2 o = x2[w];
-            const float mm = fmaxf(m, o.x);
-            if (mm > -CUDART_INF_F) S = S * pf_ex2(m - mm) + o.y * pf_ex2(o.x - mm);
-            m = mm;
+          for (int hf = 0; hf < TP; ++hf) {
+            float m = mH[hf], S = SH[hf];
+#pragma unroll
+            for (int w = 1; w < (G < 4 ? G : 4); ++w) {
+              const float2 o = x2[hf * kPfM * 4 + w];
+              const float mm = fmaxf(m, o.x);
+              if (mm > -CUDART_INF_F) S = S * pf_ex2(m - mm) + o.y * pf_ex2(o.x - mm);
+              m = mm;
+            }
+            mH[hf] = m; SH[hf] = S;
           }
         }
       }
-      if (hq == 0 && i < wk.len && !dead)
-        c.lscore[((size_t)(wk.b * p.H_kv + wk.h)) * p.N_cap + i] = (m + log2f(S)) * kPfLn2 - lnwsuf[klo] - ln_G;
+      if (hq == 0 && !dead) {
+#pragma unroll
+        for (int hf = 0; hf < TP; ++hf) {
+          const int i = wk.tile * ROWS + hf * kPfM + row;
+          const int klo = min(32, max(0, i - wk.len + W));
+          if (i < wk.len)
+            c.lscore[((size_t)(wk.b * p.H_kv + wk.h)) * p.N_cap + i] =
+                (mH[hf] + log2f(SH[hf])) * kPfLn2 - lnwsuf[klo] - ln_G;
+        }
+      }
       wk.next(p, c.seq_len, it + 1 < ntiles);
     }
   }
@@ -398,7 +426,7 @@ static void launch_prefill_t(const keepkv_params &p, const keepkv_cache &c, cons
     attr_done_dev[dev & 63] = true;
   }
   CUtensorMap mapK, mapQ;
-  if (!make_bf16_rows_map(&mapK, c.K, (uint64_t)p.B * p.H_kv * p.N_cap, D, kPfM) ||
+  if (!make_bf16_rows_map(&mapK, c.K, (uint64_t)p.B * p.H_kv * p.N_cap, D, SL::kRows) ||
       !make_bf16_rows_map(&mapQ, const_cast<void *>(q_window), (uint64_t)p.B * p.H_q * W, D, W)) {
     if (ctx.err == cudaSuccess) ctx.err = cudaErrorInvalidValue;
     return;
