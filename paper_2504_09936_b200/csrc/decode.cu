@@ -291,10 +291,49 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     s_issued = pit;   // the descriptor of every tile below pit is in place
     return true;
   };
+  // One cluster per unit: tile `it` of this CTA is tile a_tlo + it of the cluster's unit, so its descriptor needs
+  // none of the walk over sequences and heads above (about 400 cycles per tile of this one thread).
+  const int a_u = aligned ? cta / csize : 0;
+  const int a_len = aligned ? len_of(a_u / p.H_kv) : 0;
+  const int a_tlo = aligned ? (int)g0 : 0;
+  int a_fresh_tile = -1, a_fresh_row = -1;
+  if (aligned && k_new) {
+    const int old = old_len(a_u / p.H_kv);
+    if (old >= 0 && old < p.N_cap) { a_fresh_tile = old / kTile; a_fresh_row = old % kTile; }
+  }
+  auto issue_aligned = [&]() -> bool {
+    const int it = pit, stage = it % S;
+    if (!mbar_wait_n(smem_u32(&empty_bar[stage]), ((it / S) & 1) ^ 1, spin_limit)) return false;
+    const int tile = a_tlo + it;
+    TileDesc d;
+    d.u = a_u; d.tile = tile; d.len = a_len;
+    d.flags = (it == 0 ? 1 : 0) | (it == ntiles - 1 ? 2 : 0);
+    d.c_first = 0;
+    d.nparts = tb_unit == 1 ? 1 : csize;
+    d.u_next = -1;
+    d.fresh = tile == a_fresh_tile ? a_fresh_row : -1;
+    *reinterpret_cast<TileDesc *>(smem + stage * SL::kStride + SL::kDesc) = d;
+    if (it != withhold) {   // (test hook: the tile is announced, its copies are never issued)
+      const uint32_t bar = smem_u32(&full_bar[stage]);
+      const uint32_t dst = smem_base + stage * SL::kStride;
+      const size_t ubase = (size_t)a_u * p.N_cap;
+      const int row = (int)ubase + tile * kTile;
+      mbar_expect_tx(bar, SL::kTxBytes);
+      tma_load_3d(dst + SL::kK, &mapK, 0, row, 0, bar);
+      tma_load_3d(dst + SL::kV, &mapV, 0, row, 0, bar);
+      bulk_load_1d(dst + SL::kVotes, c.votes + ubase + (size_t)tile * kTile, kTile * 4, bar);
+      bulk_load_1d(dst + SL::kLscore, c.lscore + ubase + (size_t)tile * kTile, kTile * 4, bar);
+    }
+    ++pit;
+    __threadfence_block();
+    s_issued = pit;
+    return true;
+  };
+  auto issue_next = [&]() -> bool { return aligned ? issue_aligned() : issue_tile(); };
   if (tid == 0) {
     const int first = early ? S : S - 1;   // nothing else to do before the wait: fill the whole ring
     while (pit < ntiles && pit < first)
-      if (!issue_tile()) { s_stop = pit; s_abort = 1; break; }
+      if (!issue_next()) { s_stop = pit; s_abort = 1; break; }
   }
   if (early) {
     pdl_wait();
@@ -364,7 +403,7 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
       const int stage = it % S;
       // keep the ring S-1 tiles ahead: the stage of tile it-1 is free once all four warps have left it
       if (tid == 0 && pit < ntiles && pit <= it + S - 1 && s_stop > pit)
-        if (!issue_tile()) { s_stop = pit; s_abort = 1; }
+        if (!issue_next()) { s_stop = pit; s_abort = 1; }
       __syncwarp();
       if (!dead) {
         int ok = 0;
