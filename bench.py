@@ -425,10 +425,16 @@ def run_ours(args, w, rank, world):
         # host lays a period's inputs out per step and layer beforehand (a serving loop would have produced them
         # there); the timed region is the steps themselves: enqueue, copies, kernels, and the wait for the
         # outputs that the next token depends on.
-        lay = lambda t: torch.empty(P, L, *t.shape[1:], dtype=t.dtype).pin_memory()
-        qh_p, knh_p, vnh_p = lay(qh), lay(knh), lay(vnh)              # [P, L, ...] one period of host inputs
+        # a step's queries, keys and values lie back to back, on the host and in the staging buffer on the device:
+        # the entry point then moves them with one copy
+        nq, nk = L * w.B * w.H_q * w.d, L * w.B * w.H_kv * w.d
+        in_h = torch.empty(P, nq + 2 * nk, dtype=torch.bfloat16).pin_memory()         # one period of host inputs
+        in_d = torch.empty(nq + 2 * nk, dtype=torch.bfloat16, device="cuda")
+        qh_p = in_h[:, :nq].view(P, L, w.B, w.H_q, w.d)
+        knh_p = in_h[:, nq:nq + nk].view(P, L, w.B, w.H_kv, w.d)
+        vnh_p = in_h[:, nq + nk:].view(P, L, w.B, w.H_kv, w.d)
         oh = torch.empty(L, w.B, w.H_q, w.d, dtype=torch.bfloat16).pin_memory()
-        qd, kd, vd = (torch.empty_like(t[0], device="cuda") for t in (qh_p, knh_p, vnh_p))
+        qd, kd, vd = in_d[:nq].view(L, w.B, w.H_q, w.d), in_d[nq:nq + nk].view(L, w.B, w.H_kv, w.d), in_d[nq + nk:].view(L, w.B, w.H_kv, w.d)
         od = torch.empty_like(oh, device="cuda")
 
         def period_e2e(cur, oth):

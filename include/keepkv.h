@@ -265,7 +265,9 @@ int keepkv_decode_step_host(const keepkv_params *p, const keepkv_cache *cache, c
 /* The same step for n_layers independent layer caches of one shape in one call: the host arrays carry the
  * layers back to back (q_host, out_host: bf16 [n_layers, B, H_q, d]; k_new_host, v_new_host: bf16
  * [n_layers, B, H_kv, d]; the device staging buffers have the same shapes), and are moved with one copy
- * each per call instead of one per layer.  caches_host: host array of n_layers keepkv_cache structs. */
+ * each per call instead of one per layer -- with a single copy for all three inputs when k_new_host starts where
+ * q_host ends and v_new_host where k_new_host ends, and the three staging buffers lie the same way.
+ * caches_host: host array of n_layers keepkv_cache structs. */
 int keepkv_decode_step_host_layers(const keepkv_params *p, const keepkv_cache *caches_host, int32_t n_layers,
                                    const void *q_host, const void *k_new_host, const void *v_new_host, void *out_host,
                                    void *q_dev, void *k_new_dev, void *v_new_dev, void *out_dev, int update_scores,

@@ -317,9 +317,16 @@ int keepkv_decode_step_host_layers(const keepkv_params *p, const keepkv_cache *c
     cudaError_t e = cudaMemcpyAsync(dstp, srcp, n, kind, ctx.stream);
     if (e != cudaSuccess && ctx.err == cudaSuccess) ctx.err = e;
   };
-  cp(q_dev, q_host, qb * n_layers, cudaMemcpyHostToDevice);
-  cp(k_new_dev, k_new_host, kb * n_layers, cudaMemcpyHostToDevice);
-  cp(v_new_dev, v_new_host, kb * n_layers, cudaMemcpyHostToDevice);
+  const size_t qn = qb * n_layers, kn = kb * n_layers;
+  const bool packed = (const char *)k_new_host == (const char *)q_host + qn && (const char *)v_new_host == (const char *)k_new_host + kn &&
+                      (char *)k_new_dev == (char *)q_dev + qn && (char *)v_new_dev == (char *)k_new_dev + kn;
+  if (packed) {   // queries, keys and values lie back to back on both sides: one copy instead of three
+    cp(q_dev, q_host, qn + 2 * kn, cudaMemcpyHostToDevice);
+  } else {
+    cp(q_dev, q_host, qn, cudaMemcpyHostToDevice);
+    cp(k_new_dev, k_new_host, kn, cudaMemcpyHostToDevice);
+    cp(v_new_dev, v_new_host, kn, cudaMemcpyHostToDevice);
+  }
   for (int l = 0; l < n_layers && ctx.err == cudaSuccess; ++l) {
     launch_decode(*p, caches_host[l], (const char *)q_dev + qb * l, (char *)out_dev + qb * l, nullptr, update_scores,
                   (char *)ws, L, status_dev, ctx, (const char *)k_new_dev + kb * l, (const char *)v_new_dev + kb * l);

@@ -446,7 +446,9 @@ def test_decode_step_many_sequences():
     assert int(st1.item()) == int(st2.item()) == kb.DEV_APPEND_FULL
 
 
-def test_decode_step_host_layers_matches_per_layer_calls():
+@pytest.mark.parametrize("packed", [False, True])
+def test_decode_step_host_layers_matches_per_layer_calls(packed):
+    """packed: queries, keys and values back to back on the host and in the staging buffer (moved by one copy)."""
     p = kb.make_params(B=2, H_q=8, H_kv=2, d=128, N_cap=256)
     Lr = 3
     base = [random_cache(p, [100 + 7 * l, 200 - 5 * l], seed=40 + l) for l in range(Lr)]
@@ -458,6 +460,13 @@ def test_decode_step_host_layers_matches_per_layer_calls():
     qh, kh, vh = mk(Lr, 2, 8, 128), mk(Lr, 2, 2, 128), mk(Lr, 2, 2, 128)
     oh = torch.empty(Lr, 2, 8, 128, dtype=torch.bfloat16).pin_memory()
     qd, kd, vd, od = (torch.empty_like(t, device="cuda") for t in (qh, kh, vh, oh))
+    if packed:
+        nq, nk = qh.numel(), kh.numel()
+        in_h = torch.empty(nq + 2 * nk, dtype=torch.bfloat16).pin_memory()
+        in_d = torch.empty(nq + 2 * nk, dtype=torch.bfloat16, device="cuda")
+        in_h[:nq].copy_(qh.flatten()); in_h[nq:nq + nk].copy_(kh.flatten()); in_h[nq + nk:].copy_(vh.flatten())
+        qh, kh, vh = in_h[:nq].view_as(qh), in_h[nq:nq + nk].view_as(kh), in_h[nq + nk:].view_as(vh)
+        qd, kd, vd = in_d[:nq].view_as(qh), in_d[nq:nq + nk].view_as(kh), in_d[nq + nk:].view_as(vh)
     kb.keepkv_decode_step_host_layers(p, a, qh, kh, vh, oh, qd, kd, vd, od, True, ws, st)
     torch.cuda.synchronize()
     for l in range(Lr):
