@@ -192,10 +192,17 @@ decode_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ 
     total_b += s_scan[w];
   }
   const long long T = (long long)total_b * p.H_kv;
-  const int chunk = (int)((T + grid - 1) / grid);
+  // Equal ranges of `chunk` tiles per CTA.  When every unit has the same number of tiles and a range holds more than
+  // one unit, the range is rounded up to whole units (if that costs at most an eighth more tiles per CTA): no unit is
+  // then cut between two CTAs, and none of them needs the partial results and the ticket.
+  int chunk = (int)((T + grid - 1) / grid);
   // one cluster per unit, if the launch has them and no sequence is much longer than the average
   const int csize = (int)cluster_nctarank(), crank = (int)cluster_ctarank();
   tb_max = max(max(s_tbmax[0], s_tbmax[1]), max(s_tbmax[2], s_tbmax[3]));
+  if (tb_max > 0 && (long long)tb_max * p.B == total_b && chunk > tb_max) {
+    const int up = (chunk + tb_max - 1) / tb_max * tb_max;
+    if (up * 8 <= chunk * 9) chunk = up;
+  }
   const bool aligned = csize > 1 && grid == U * csize && total_b > 0 && (long long)tb_max * p.B * 4 <= 5LL * total_b;
   long long g0 = min(T, (long long)cta * chunk), g1 = min(T, g0 + chunk);
   int tb_unit = 0;   // aligned: tiles of this cluster's unit
